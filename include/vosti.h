@@ -1,0 +1,200 @@
+/*
+ * vosti.h -- C ABI of libvosti: batch-invariant paged attention for NVIDIA
+ * B200 (sm_100a).
+ *
+ * One attention operation over a prefix-sharing paged KV cache whose output
+ * for a logical (request content, token position, query head) has the same
+ * bits however it is run: alone or co-batched, any prefill chunk size,
+ * multi-token (prefill / speculative) or single-token (decode) query, any
+ * physical page placement, shared or private prefix pages.  This is the
+ * kernel-level contract of the paper's Sec. "Kernel contracts" and App. A
+ * ("Verifying Paged Attention"): equal logical inputs give bitwise-equal
+ * selected outputs across batch, query length, row index and page table.
+ *
+ * Conventions
+ *   - "device" pointers are CUDA device memory of the context's GPU, "host"
+ *     pointers ordinary host memory.  bf16 = 16-bit brain float.
+ *   - Packed rows: [T, H, d] with T = sum of q_lens, request-major,
+ *     token-minor (the paper's packed rows).  Row i of request r stands at
+ *     logical position p = start_pos[r] + i  (Sec. "The causal contract":
+ *     p = k_len - q_len + i) and attends keys 0..p of that request.
+ *   - Logical cache through the page table (App. A):
+ *         K[j,:] = K_phys[ block_table[r][j / P], j mod P, : ]   (V alike)
+ *   - Pool layout:  kv_pool[page][kv_head][0=K,1=V][slot 0..P-1][e 0..d-1]
+ *     bf16, so one (page, kv_head, K|V) chunk is P*d*2 contiguous bytes.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *   - Every call is asynchronous on the given CUDA stream (cudaStream_t
+ *     passed as void*; NULL = the legacy default stream).  Host metadata
+ *     arrays are copied before the call returns and may be reused at once.
+ *   - A context must be driven from one stream at a time: calls that overlap
+ *     on the GPU share the workspace and race.
+ *   - Errors are returned as status codes; nothing aborts, nothing falls
+ *     back to another implementation.  On any error no kernel was launched
+ *     unless the status is VOSTI_ERR_CUDA / VOSTI_ERR_TIMEOUT.
+ *
+ * Numerics are frozen at build time (key tile 64, KV split length 512, the
+ * fold and exponent rules): vosti_fingerprint() hashes them.  Outputs are
+ * comparable bit for bit only under one fingerprint on one GPU model.
+ */
+#ifndef VOSTI_H_
+#define VOSTI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vosti_ctx vosti_ctx;
+
+typedef enum {
+  VOSTI_OK = 0,
+  VOSTI_ERR_INVALID_ARG = 1,        /* null pointer, negative size, bad scale */
+  VOSTI_ERR_UNSUPPORTED_CONFIG = 2, /* geometry outside the frozen set */
+  VOSTI_ERR_OUT_OF_RANGE = 3,       /* lengths / page ids violate the call premises */
+  VOSTI_ERR_WORKSPACE = 4,          /* workspace too small or misaligned */
+  VOSTI_ERR_CUDA = 5,               /* a CUDA runtime / driver call failed */
+  VOSTI_ERR_TIMEOUT = 6             /* a bounded device-side wait gave up */
+} vosti_status;
+
+enum {
+  VOSTI_FLAG_CHECK_WRITE_SLOTS = 1 /* kv_append verifies that write slots are pairwise disjoint */
+};
+
+/* The fixed deployment configuration (Sec. "Fixed kernel choices": tile
+ * parameters are bound at initialisation from model and deployment only; a
+ * configuration outside the supported set is rejected, never auto-tuned).
+ * Supported: head_dim in {64, 128}; page_size 16; n_q_heads a multiple of
+ * n_kv_heads with ratio in {1, 2, 4, 8, 16}. */
+typedef struct {
+  int32_t n_q_heads, n_kv_heads, head_dim, page_size;
+  int64_t num_pages;      /* pages in kv_pool */
+  void* kv_pool;          /* device, caller-owned, 1024-byte aligned, layout above */
+  int32_t max_batch;      /* largest `batch` of any call */
+  int64_t max_total_q;    /* largest sum of q_lens of any call */
+  int64_t max_seq_len;    /* largest seq_len of any request */
+  void* workspace;        /* device, caller-owned, 1024-byte aligned */
+  size_t workspace_bytes; /* >= vosti_workspace_bytes(config) */
+  uint32_t flags;         /* VOSTI_FLAG_* */
+} vosti_config;
+
+/* One unit of scheduled work (App. A: the kernel's parallel loop over query
+ * tiles and heads; the KV split is this library's addition).  Rows of a
+ * request are numbered token*G + head_in_group; row group g holds rows
+ * 16g..16g+15; the item walks KV splits split_begin..split_end-1 of 512 keys
+ * each, for every KV head. */
+typedef struct {
+  int32_t req, row_group, split_begin, split_end;
+} vosti_work_item;
+
+/* Device workspace the configuration needs (host-only; reads no pointer
+ * field).  Returns 0 if the geometry is unsupported. */
+size_t vosti_workspace_bytes(const vosti_config* config);
+
+/* Work planning (host-only, no GPU needed).  Writes up to `cap` items to
+ * `items` (may be NULL with cap 0) and the total count to *n_items; *n_split
+ * receives how many leading items are split-parallel (they emit one partial
+ * (m, z, U) per split, folded later in split order), the rest walk their
+ * splits in order and fold in place; *n_partial_rows the number of partial
+ * rows.  The plan of a request is a pure function of its own
+ * (q_len, start_pos) and the geometry: never of batch size, other requests,
+ * page ids or table width (Sec. "Fixed kernel choices").  Only the order of
+ * items (longest first) depends on the batch; results do not depend on it.
+ * Premises checked: q_len >= 0, start_pos >= 0, start_pos + q_len <= seq_len
+ * <= max_seq_len, batch <= max_batch, sum q_len <= max_total_q. */
+vosti_status vosti_plan(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
+                        const int32_t* seq_lens, int32_t batch, vosti_work_item* items, int64_t cap,
+                        int64_t* n_items, int64_t* n_split, int64_t* n_partial_rows);
+
+/* Create a context on the current CUDA device: checks the geometry, builds
+ * the TMA tensor map of the pool, allocates host staging (the only memory
+ * the library owns) and clears the device status word.  Synchronous. */
+vosti_status vosti_create(vosti_ctx** out, const vosti_config* config);
+vosti_status vosti_destroy(vosti_ctx* ctx);
+
+/* KV write into page slots (Sec. "Separate cache reuse from generation": new
+ * K/V values go to the request's private suffix slots; shared or registered
+ * prefix pages stay immutable -- keeping write slots off shared pages is the
+ * caller's premise).  Token i of request r is written to page
+ * block_tables[r][(start_pos[r]+i) / P], slot (start_pos[r]+i) mod P, for
+ * every KV head.  Bit-exact copy.
+ *   k_new, v_new   device [T, n_kv_heads, d] bf16, 16-byte aligned
+ *   q_lens, start_pos   host [batch]
+ *   block_tables   host [batch, block_table_stride]; only entries that a
+ *                  written position indexes are read
+ * Errors: OUT_OF_RANGE if a position falls outside the table or a page id
+ * outside the pool, or (with VOSTI_FLAG_CHECK_WRITE_SLOTS) two tokens share
+ * a slot. */
+vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_new,
+                             const int32_t* q_lens, const int32_t* start_pos,
+                             const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
+                             void* cuda_stream);
+
+/* Causal GQA attention over the paged cache (App. A, "A Simplified Tile IR":
+ * tiled online softmax with fp32 state (m, z, U), base-two exponent,
+ * weights cast to bf16 before the second product, identity step for rows
+ * that see nothing of a tile, O = U * (z > 0 ? 1/z : 0)).  Reads only the
+ * pool: the chunk's own tokens must have been appended first (that is how
+ * prefill and decode see the same keys).
+ *   q, out        device [T, n_q_heads, d] bf16, 16-byte aligned; every out row is overwritten
+ *   q_lens, start_pos, seq_lens   host [batch]; q_len == 0 skips the request
+ *   block_tables  host [batch, block_table_stride]; only the entries
+ *                 0 .. ceil((start_pos+q_len)/P)-1 of a row are read
+ *   softmax_scale natural-log scale sigma >= 0, finite (scores are sigma * q.k)
+ * Keys j > p are never visible; slots at or beyond start_pos+q_len may hold
+ * anything (they are zero-filled on chip), all other inputs must be finite
+ * (the paper's unchecked finiteness premise).
+ * Errors: OUT_OF_RANGE for violated premises (start_pos+q_len > seq_len,
+ * seq_len > max_seq_len, table too short, page id outside the pool, batch or
+ * total rows above the configured maxima). */
+vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, const int32_t* q_lens,
+                                   const int32_t* start_pos, const int32_t* seq_lens,
+                                   const int32_t* block_tables, int32_t block_table_stride,
+                                   int32_t batch, float softmax_scale, void* cuda_stream);
+
+/* One serving step from HOST buffers: copies q, k_new, v_new to the device,
+ * runs vosti_kv_append then vosti_paged_attention, copies the output back
+ * and waits for it.  Same arithmetic, same kernels; exists so that a caller
+ * (and the end-to-end benchmark) can drive the path without device tensors.
+ *   q_host, out_host     host [T, n_q_heads, d] bf16 (pinned memory makes the copies asynchronous)
+ *   k_new_host, v_new_host   host [T, n_kv_heads, d] bf16
+ * Synchronous: returns after out_host is complete. */
+vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host,
+                             const void* k_new_host, const void* v_new_host, const int32_t* q_lens,
+                             const int32_t* start_pos, const int32_t* seq_lens,
+                             const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
+                             float softmax_scale, void* cuda_stream);
+
+/* Waits for the stream and reads the device status word: VOSTI_OK, or
+ * VOSTI_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is
+ * then undefined).  The word is cleared by the read. */
+vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream);
+
+/* Timing of one kernel of the path with CUDA events recorded on the caller's
+ * stream around each of its launches.  mode: 0 stops recording; 1 times the
+ * split-parallel attention kernel (the decode hot loop, a3-a7), 2 the
+ * sequential attention kernel (long queries), 3 the cross-split combine.
+ * A non-zero mode starts a fresh record.  vosti_profile_read waits for the
+ * recorded events and returns the summed kernel time in milliseconds and the
+ * number of launches timed. */
+vosti_status vosti_profile_enable(vosti_ctx* ctx, int32_t mode);
+vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* kernels_timed);
+
+/* Kernels launched through this context since creation. */
+int64_t vosti_launch_count(const vosti_ctx* ctx);
+
+/* Hash of the frozen numerics (tile size, split length, fold and exponent
+ * rules, library version): the paper's deployment identity W.  ctx may be
+ * NULL. */
+uint64_t vosti_fingerprint(const vosti_ctx* ctx);
+
+/* Frozen constants: key tile B_N, split length L_S, rows per row group. */
+void vosti_constants(int32_t* key_tile, int32_t* split_len, int32_t* rows_per_group);
+
+const char* vosti_status_string(vosti_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VOSTI_H_ */

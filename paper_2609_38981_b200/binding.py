@@ -1,0 +1,259 @@
+"""ctypes binding of libvosti (``include/vosti.h``): argument marshalling only.
+
+Every step of the path runs in the library's CUDA kernels; this module turns
+torch tensors into device pointers and numpy arrays into host pointers.  There
+is no fallback: if the built library is missing, importing this module raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libvosti.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2609_38981_b200.build` "
+        "(nvcc, sm_100a).  There is no CPU or PyTorch fallback.")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+VOSTI_OK, VOSTI_ERR_INVALID_ARG, VOSTI_ERR_UNSUPPORTED_CONFIG, VOSTI_ERR_OUT_OF_RANGE, \
+    VOSTI_ERR_WORKSPACE, VOSTI_ERR_CUDA, VOSTI_ERR_TIMEOUT = range(7)
+VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
+
+EXPORTS = (
+    "vosti_workspace_bytes", "vosti_plan", "vosti_create", "vosti_destroy", "vosti_kv_append",
+    "vosti_paged_attention", "vosti_step_host", "vosti_poll_device_status",
+    "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
+    "vosti_constants", "vosti_status_string",
+)
+
+
+class vosti_config(ctypes.Structure):
+    _fields_ = [
+        ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32), ("page_size", ctypes.c_int32),
+        ("num_pages", ctypes.c_int64), ("kv_pool", ctypes.c_void_p),
+        ("max_batch", ctypes.c_int32), ("max_total_q", ctypes.c_int64),
+        ("max_seq_len", ctypes.c_int64), ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t), ("flags", ctypes.c_uint32),
+    ]
+
+
+class vosti_work_item(ctypes.Structure):
+    _fields_ = [("req", ctypes.c_int32), ("row_group", ctypes.c_int32),
+                ("split_begin", ctypes.c_int32), ("split_end", ctypes.c_int32)]
+
+
+_i32p = ctypes.POINTER(ctypes.c_int32)
+_cfgp = ctypes.POINTER(vosti_config)
+_vp = ctypes.c_void_p
+
+_lib.vosti_workspace_bytes.restype = ctypes.c_size_t
+_lib.vosti_workspace_bytes.argtypes = [_cfgp]
+_lib.vosti_plan.restype = ctypes.c_int
+_lib.vosti_plan.argtypes = [_cfgp, _i32p, _i32p, _i32p, ctypes.c_int32,
+                            ctypes.POINTER(vosti_work_item), ctypes.c_int64,
+                            ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                            ctypes.POINTER(ctypes.c_int64)]
+_lib.vosti_create.restype = ctypes.c_int
+_lib.vosti_create.argtypes = [ctypes.POINTER(_vp), _cfgp]
+_lib.vosti_destroy.restype = ctypes.c_int
+_lib.vosti_destroy.argtypes = [_vp]
+_lib.vosti_kv_append.restype = ctypes.c_int
+_lib.vosti_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, ctypes.c_int32,
+                                 ctypes.c_int32, _vp]
+_lib.vosti_paged_attention.restype = ctypes.c_int
+_lib.vosti_paged_attention.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32,
+                                       ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_step_host.restype = ctypes.c_int
+_lib.vosti_step_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p,
+                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_poll_device_status.restype = ctypes.c_int
+_lib.vosti_poll_device_status.argtypes = [_vp, _vp]
+_lib.vosti_profile_enable.restype = ctypes.c_int
+_lib.vosti_profile_enable.argtypes = [_vp, ctypes.c_int32]
+_lib.vosti_profile_read.restype = ctypes.c_int
+_lib.vosti_profile_read.argtypes = [_vp, ctypes.POINTER(ctypes.c_double),
+                                    ctypes.POINTER(ctypes.c_int64)]
+_lib.vosti_launch_count.restype = ctypes.c_int64
+_lib.vosti_launch_count.argtypes = [_vp]
+_lib.vosti_fingerprint.restype = ctypes.c_uint64
+_lib.vosti_fingerprint.argtypes = [_vp]
+_lib.vosti_constants.restype = None
+_lib.vosti_constants.argtypes = [_i32p, _i32p, _i32p]
+_lib.vosti_status_string.restype = ctypes.c_char_p
+_lib.vosti_status_string.argtypes = [ctypes.c_int]
+
+
+class VostiError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {vosti_status_string(status)} ({status})")
+
+
+def _check(status: int, where: str) -> None:
+    if status != VOSTI_OK:
+        raise VostiError(status, where)
+
+
+def _host_i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _ip(a: np.ndarray):
+    return a.ctypes.data_as(_i32p)
+
+
+def _dev(t) -> int:
+    """Device (or host) address of a contiguous torch tensor, or a raw int."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+def vosti_status_string(status: int) -> str:
+    return _lib.vosti_status_string(int(status)).decode()
+
+
+def vosti_constants():
+    a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    _lib.vosti_constants(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    return {"key_tile": a.value, "split_len": b.value, "rows_per_group": c.value}
+
+
+def make_config(n_q_heads, n_kv_heads, head_dim, page_size, num_pages, max_batch, max_total_q,
+                max_seq_len, kv_pool=0, workspace=0, workspace_bytes=0, flags=0) -> vosti_config:
+    return vosti_config(n_q_heads, n_kv_heads, head_dim, page_size, num_pages, _dev(kv_pool),
+                        max_batch, max_total_q, max_seq_len, _dev(workspace), workspace_bytes, flags)
+
+
+def vosti_workspace_bytes(cfg: vosti_config) -> int:
+    return int(_lib.vosti_workspace_bytes(ctypes.byref(cfg)))
+
+
+def vosti_plan(cfg: vosti_config, q_lens, start_pos, seq_lens):
+    """Host-only planning.  Returns (items [n,4] int32, n_split, n_partial_rows)."""
+    q, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    cnt, nsp, npr = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.vosti_plan(ctypes.byref(cfg), _ip(q), _ip(s), _ip(n), len(q), None, 0,
+                           ctypes.byref(cnt), ctypes.byref(nsp), ctypes.byref(npr)), "vosti_plan")
+    items = (vosti_work_item * max(cnt.value, 1))()
+    _check(_lib.vosti_plan(ctypes.byref(cfg), _ip(q), _ip(s), _ip(n), len(q), items, cnt.value,
+                           ctypes.byref(cnt), ctypes.byref(nsp), ctypes.byref(npr)), "vosti_plan")
+    arr = np.array([[it.req, it.row_group, it.split_begin, it.split_end]
+                    for it in items[:cnt.value]], dtype=np.int32).reshape(-1, 4)
+    return arr, nsp.value, npr.value
+
+
+def vosti_fingerprint(ctx=None) -> int:
+    return int(_lib.vosti_fingerprint(ctx.handle if ctx is not None else None))
+
+
+class Context:
+    """Owns a vosti_ctx handle and keeps the pool / workspace tensors alive."""
+
+    def __init__(self, cfg: vosti_config, keep=()):
+        self.cfg = cfg
+        self._keep = tuple(keep)
+        h = _vp()
+        _check(_lib.vosti_create(ctypes.byref(h), ctypes.byref(cfg)), "vosti_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            _lib.vosti_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def vosti_create(n_q_heads, n_kv_heads, head_dim, page_size, kv_pool, max_batch, max_total_q,
+                 max_seq_len, flags=0, workspace=None) -> Context:
+    """kv_pool: torch uint8/int16/bf16 CUDA tensor holding the whole pool.  The
+    workspace is allocated with torch (device memory is torch's job here)
+    unless one is passed in."""
+    import torch
+    page_bytes = n_kv_heads * 2 * page_size * head_dim * 2
+    num_pages = kv_pool.numel() * kv_pool.element_size() // page_bytes
+    cfg = make_config(n_q_heads, n_kv_heads, head_dim, page_size, num_pages, max_batch,
+                      max_total_q, max_seq_len, flags=flags)
+    need = vosti_workspace_bytes(cfg)
+    if need == 0:
+        raise VostiError(VOSTI_ERR_UNSUPPORTED_CONFIG, "vosti_workspace_bytes")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=kv_pool.device)
+    cfg.kv_pool = kv_pool.data_ptr()
+    cfg.workspace = workspace.data_ptr()
+    cfg.workspace_bytes = workspace.numel() * workspace.element_size()
+    return Context(cfg, keep=(kv_pool, workspace))
+
+
+def vosti_destroy(ctx: Context) -> None:
+    ctx.close()
+
+
+def vosti_kv_append(ctx: Context, k_new, v_new, q_lens, start_pos, block_tables,
+                    stream=None) -> None:
+    q, s = _host_i32(q_lens), _host_i32(start_pos)
+    bt = _host_i32(block_tables)
+    assert bt.ndim == 2 and bt.shape[0] == len(q)
+    _check(_lib.vosti_kv_append(ctx.handle, _dev(k_new), _dev(v_new), _ip(q), _ip(s), _ip(bt),
+                                bt.shape[1], len(q), _stream(stream)), "vosti_kv_append")
+
+
+def vosti_paged_attention(ctx: Context, q, out, q_lens, start_pos, seq_lens, block_tables,
+                          softmax_scale: float, stream=None) -> None:
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    assert bt.ndim == 2 and bt.shape[0] == len(ql)
+    _check(_lib.vosti_paged_attention(ctx.handle, _dev(q), _dev(out), _ip(ql), _ip(s), _ip(n),
+                                      _ip(bt), bt.shape[1], len(ql), float(softmax_scale),
+                                      _stream(stream)), "vosti_paged_attention")
+
+
+def vosti_step_host(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_lens, start_pos,
+                    seq_lens, block_tables, softmax_scale: float, stream=None) -> None:
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    _check(_lib.vosti_step_host(ctx.handle, _dev(q_host), _dev(out_host), _dev(k_new_host),
+                                _dev(v_new_host), _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1],
+                                len(ql), float(softmax_scale), _stream(stream)), "vosti_step_host")
+
+
+def vosti_poll_device_status(ctx: Context, stream=None) -> int:
+    return int(_lib.vosti_poll_device_status(ctx.handle, _stream(stream)))
+
+
+def vosti_profile_enable(ctx: Context, mode: int) -> None:
+    _check(_lib.vosti_profile_enable(ctx.handle, int(mode)), "vosti_profile_enable")
+
+
+def vosti_profile_read(ctx: Context):
+    ms, n = ctypes.c_double(), ctypes.c_int64()
+    _check(_lib.vosti_profile_read(ctx.handle, ctypes.byref(ms), ctypes.byref(n)),
+           "vosti_profile_read")
+    return ms.value, n.value
+
+
+def vosti_launch_count(ctx: Context) -> int:
+    return int(_lib.vosti_launch_count(ctx.handle))

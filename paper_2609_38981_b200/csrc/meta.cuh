@@ -1,0 +1,45 @@
+// Per-call metadata that the host planner writes and the kernels read.
+#pragma once
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/vosti.h"
+
+namespace vosti {
+
+// One request of a call, as the kernels see it.
+struct ReqMeta {
+  int32_t q_row0;     // first packed row of the request
+  int32_t q_len;      // query rows (tokens)
+  int32_t start;      // logical position of row 0
+  int32_t n_pages;    // used pages = ceil((start + q_len) / P)
+  int32_t bt_off;     // offset of the request's page ids in the flat table
+  int32_t n_splits;   // splits touched by the last row: (start + q_len - 1) / L_S + 1
+  int64_t part_base;  // first partial row of the request (split-parallel requests only)
+};
+
+struct AttnParams {
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const ReqMeta* reqs;
+  const vosti_work_item* items;
+  const int32_t* bt_flat;
+  const int2* split_tokens;  // (request, token) of every row the combine kernel finishes
+  float* ws_u;               // partial U rows [rows][D]
+  float2* ws_mz;             // partial (m, z) per row
+  uint32_t* status;
+  int32_t n_workers;         // items of this launch times n_kv_heads
+  int32_t n_split_tokens;
+  int32_t Hq, Hkv, G;
+  float c;                   // sigma * log2(e), rounded once on the host
+};
+
+struct AppendParams {
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  __nv_bfloat16* pool;
+  const int32_t* slot;  // per token: page * P + slot
+  int32_t n_tokens, Hkv;
+};
+
+}  // namespace vosti

@@ -1,0 +1,96 @@
+// The numerical contract: every scalar operation whose rounding decides output
+// bits, written once with explicit round-to-nearest intrinsics so that no two
+// kernels can contract or reassociate it differently.
+//
+// Per (request, position p, query head) the output bits are a function of the
+// query row, the logical keys/values 0..p, the scale and these constants only:
+//   * key tiles are absolute: tile t covers keys [64 t, 64 t + 64) counted from
+//     position 0 of the request (App. A, tile IR: t = 0..N-1, j = t*B_N + b);
+//   * KV splits are absolute too: split k covers [512 k, 512 k + 512); inside a
+//     split the state (m, z, U) starts at (-inf, 0, 0) and is updated tile by
+//     tile in ascending order exactly as in the paper's iteration;
+//   * split results are folded left to right by split index.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace vosti {
+namespace nc {
+
+constexpr int kKeyTile = 64;        // B_N
+constexpr int kSplitLen = 512;      // L_S, a multiple of B_N
+constexpr int kTilesPerSplit = kSplitLen / kKeyTile;
+constexpr int kRowsPerGroup = 16;   // rows packed into one MMA row tile
+constexpr int kSplitRowsMax = 32;   // requests with at most this many rows per KV head run split-parallel
+constexpr int kPageSize = 16;
+constexpr int kPagesPerTile = kKeyTile / kPageSize;
+constexpr int kPagesPerSplit = kSplitLen / kPageSize;
+constexpr uint32_t kVersion = 1;
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// Running maximum in the scaled (base-two) domain.  The raw maximum is taken
+// over visible lanes first; multiplying by c >= 0 is monotone, so this equals
+// the maximum of the scaled scores.
+__device__ __forceinline__ float new_max(float m_old, float raw_max_visible, float c) {
+  return fmaxf(m_old, __fmul_rn(raw_max_visible, c));
+}
+// alpha = 2^(m - m_hat)
+__device__ __forceinline__ float rescale(float m_old, float m_new) {
+  return ex2(__fsub_rn(m_old, m_new));
+}
+// A = 2^(s*c - m_hat), one fused multiply-add then the exponential.
+__device__ __forceinline__ float weight(float s, float c, float neg_m_new) {
+  return ex2(__fmaf_rn(s, c, neg_m_new));
+}
+// z_hat = z*alpha + sum_b A
+__device__ __forceinline__ float z_update(float z, float alpha, float row_sum) {
+  return __fmaf_rn(z, alpha, row_sum);
+}
+__device__ __forceinline__ float u_rescale(float u, float alpha) { return __fmul_rn(u, alpha); }
+
+// sum_b A over the 64 lanes of a tile, order fixed by the lane index b alone:
+// four partial sums, partial q takes the lanes with (b mod 8) / 2 == q in
+// ascending b; total = (s0 + s1) + (s2 + s3).
+__device__ __forceinline__ float quad_partial(const float (&a)[16]) {
+  float s = a[0];
+#pragma unroll
+  for (int i = 1; i < 16; ++i) s = __fadd_rn(s, a[i]);
+  return s;
+}
+__device__ __forceinline__ float quad_total(float s0, float s1, float s2, float s3) {
+  return __fadd_rn(__fadd_rn(s0, s1), __fadd_rn(s2, s3));
+}
+
+// Left fold of split results.  (m_c, z_c, U_c) <- fold((m_c, z_c, U_c), (m_k, z_k, U_k)).
+struct FoldFactors {
+  float a, b;
+};
+__device__ __forceinline__ FoldFactors fold_scalars(float& m_c, float& z_c, float m_k, float z_k) {
+  const float m_star = fmaxf(m_c, m_k);
+  FoldFactors f;
+  f.a = ex2(__fsub_rn(m_c, m_star));
+  f.b = ex2(__fsub_rn(m_k, m_star));
+  z_c = __fmaf_rn(z_c, f.a, __fmul_rn(z_k, f.b));
+  m_c = m_star;
+  return f;
+}
+__device__ __forceinline__ float fold_u(float u_c, float u_k, FoldFactors f) {
+  return __fmaf_rn(u_c, f.a, __fmul_rn(u_k, f.b));
+}
+
+// O = U * select(z > 0, 1/z, 0); adding +0 turns a -0 result into +0 so that
+// the sign of an exactly-zero output cannot depend on which masked lanes a
+// schedule happened to multiply by zero.
+__device__ __forceinline__ float out_scale(float z) { return z > 0.0f ? __frcp_rn(z) : 0.0f; }
+__device__ __forceinline__ float out_value(float u, float inv) {
+  return __fadd_rn(__fmul_rn(u, inv), 0.0f);
+}
+
+}  // namespace nc
+}  // namespace vosti

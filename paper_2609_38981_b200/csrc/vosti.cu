@@ -1,0 +1,612 @@
+// libvosti: C ABI, host-side validation and work planning, kernel launches.
+// Entry points are declared and documented in include/vosti.h.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "attn_warp.cuh"
+
+namespace vosti {
+namespace {
+
+constexpr int kHostSlots = 8;        // ring of pinned staging buffers
+constexpr size_t kAlign = 1024;
+
+size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+
+bool geometry_ok(const vosti_config& c) {
+  if (c.head_dim != 64 && c.head_dim != 128) return false;
+  if (c.page_size != nc::kPageSize) return false;
+  if (c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.n_q_heads % c.n_kv_heads) return false;
+  const int g = c.n_q_heads / c.n_kv_heads;
+  if (g != 1 && g != 2 && g != 4 && g != 8 && g != 16) return false;
+  if (c.num_pages <= 0 || c.max_batch <= 0 || c.max_total_q <= 0 || c.max_seq_len <= 0) return false;
+  // TMA row coordinates are 32-bit: rows = pages * kv_heads * 2 * 16.
+  if (c.num_pages * c.n_kv_heads >= (int64_t{1} << 26)) return false;
+  if (c.max_seq_len >= (int64_t{1} << 30) || c.max_total_q >= (int64_t{1} << 27)) return false;
+  return true;
+}
+
+// Sizes derived from the configuration alone.
+struct Limits {
+  int64_t k_max;         // splits of the longest sequence
+  int64_t pages_max;     // page-table entries one call can carry
+  int64_t items_max;
+  int64_t part_rows_max;
+  size_t meta_bytes;     // one metadata blob (attention or append)
+  // workspace offsets
+  size_t off_status, off_meta, off_part_u, off_part_mz, off_stage_q, off_stage_o, off_stage_k,
+      off_stage_v, total;
+};
+
+Limits limits_of(const vosti_config& c) {
+  Limits L{};
+  const int64_t G = c.n_q_heads / c.n_kv_heads;
+  L.k_max = (c.max_seq_len + nc::kSplitLen - 1) / nc::kSplitLen;
+  L.pages_max = int64_t{c.max_batch} * ((c.max_seq_len + nc::kPageSize - 1) / nc::kPageSize);
+  const int64_t groups_split = (nc::kSplitRowsMax + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+  const int64_t items_split = int64_t{c.max_batch} * groups_split * L.k_max;
+  const int64_t items_seq = (c.max_total_q * G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup + c.max_batch;
+  L.items_max = items_split + items_seq;
+  const int64_t rows_by_batch = int64_t{c.max_batch} * nc::kSplitRowsMax;
+  const int64_t rows_by_total = c.max_total_q * G;
+  L.part_rows_max = std::min(rows_by_batch, rows_by_total) * c.n_kv_heads * L.k_max;
+  const size_t attn_blob = align_up(sizeof(ReqMeta) * c.max_batch, 16) +
+                           align_up(sizeof(vosti_work_item) * L.items_max, 16) +
+                           align_up(sizeof(int32_t) * L.pages_max, 16) +
+                           align_up(sizeof(int2) * c.max_total_q, 16);
+  const size_t append_blob = align_up(sizeof(int32_t) * c.max_total_q, 16);
+  L.meta_bytes = align_up(std::max(attn_blob, append_blob));
+  size_t at = 0;
+  L.off_status = at; at += kAlign;
+  L.off_meta = at; at += L.meta_bytes;
+  L.off_part_u = at; at += align_up(sizeof(float) * L.part_rows_max * c.head_dim);
+  L.off_part_mz = at; at += align_up(sizeof(float2) * L.part_rows_max);
+  const size_t qbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_q_heads * c.head_dim;
+  const size_t kbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_kv_heads * c.head_dim;
+  L.off_stage_q = at; at += align_up(qbytes);
+  L.off_stage_o = at; at += align_up(qbytes);
+  L.off_stage_k = at; at += align_up(kbytes);
+  L.off_stage_v = at; at += align_up(kbytes);
+  L.total = at;
+  return L;
+}
+
+struct Plan {
+  std::vector<vosti_work_item> items;  // split-parallel items first
+  int64_t n_split = 0;
+  int64_t n_partial_rows = 0;
+};
+
+// The plan of one request depends on its own (q_len, start) and the geometry.
+vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const int32_t* start_pos,
+                           const int32_t* seq_lens, int32_t batch, Plan* plan,
+                           std::vector<int64_t>* part_base) {
+  if (batch < 0 || (batch > 0 && (!q_lens || !start_pos || !seq_lens))) return VOSTI_ERR_INVALID_ARG;
+  if (batch > c.max_batch) return VOSTI_ERR_OUT_OF_RANGE;
+  const int G = c.n_q_heads / c.n_kv_heads;
+  int64_t total_q = 0;
+  std::vector<vosti_work_item> split_items, seq_items;
+  if (part_base) part_base->assign(batch, 0);
+  for (int r = 0; r < batch; ++r) {
+    const int64_t q = q_lens[r], st = start_pos[r], n = seq_lens[r];
+    if (q < 0 || st < 0 || st + q > n || n > c.max_seq_len) return VOSTI_ERR_OUT_OF_RANGE;
+    total_q += q;
+    if (q == 0) continue;
+    const int64_t rows = q * G;
+    const int groups = static_cast<int>((rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup);
+    const bool split_parallel = rows <= nc::kSplitRowsMax;
+    if (split_parallel) {
+      if (part_base) (*part_base)[r] = plan->n_partial_rows;
+      const int64_t n_splits = (st + q - 1) / nc::kSplitLen + 1;
+      plan->n_partial_rows += int64_t{c.n_kv_heads} * n_splits * rows;
+    }
+    for (int g = 0; g < groups; ++g) {
+      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{g} * nc::kRowsPerGroup + 15) / G);
+      const int k_g = static_cast<int>((st + last_tok) / nc::kSplitLen + 1);
+      if (split_parallel) {
+        for (int k = 0; k < k_g; ++k) split_items.push_back({r, g, k, k + 1});
+      } else {
+        seq_items.push_back({r, g, 0, k_g});
+      }
+    }
+  }
+  if (total_q > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
+  // Longest first (by key tiles walked); stable, so the order is reproducible.
+  auto tiles_of = [&](const vosti_work_item& it) {
+    const int64_t q = q_lens[it.req], st = start_pos[it.req];
+    const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{it.row_group} * nc::kRowsPerGroup + 15) / G);
+    const int64_t t_end = std::min<int64_t>(int64_t{it.split_end} * nc::kTilesPerSplit,
+                                            (st + last_tok) / nc::kKeyTile + 1);
+    return t_end - int64_t{it.split_begin} * nc::kTilesPerSplit;
+  };
+  auto longer = [&](const vosti_work_item& a, const vosti_work_item& b) { return tiles_of(a) > tiles_of(b); };
+  std::stable_sort(split_items.begin(), split_items.end(), longer);
+  std::stable_sort(seq_items.begin(), seq_items.end(), longer);
+  plan->n_split = static_cast<int64_t>(split_items.size());
+  plan->items = std::move(split_items);
+  plan->items.insert(plan->items.end(), seq_items.begin(), seq_items.end());
+  return VOSTI_OK;
+}
+
+uint64_t fnv1a(uint64_t h, uint64_t x) {
+  for (int i = 0; i < 8; ++i) {
+    h ^= (x >> (8 * i)) & 0xff;
+    h *= 1099511628211ull;
+  }
+  return h;
+}
+
+struct HostSlot {
+  uint8_t* pinned = nullptr;
+  cudaEvent_t copied = nullptr;
+  bool in_flight = false;
+};
+
+}  // namespace
+}  // namespace vosti
+
+using namespace vosti;
+
+struct vosti_ctx {
+  vosti_config cfg;
+  Limits lim;
+  int device = 0;
+  alignas(64) CUtensorMap kv_map;
+  HostSlot slots[kHostSlots];
+  int next_slot = 0;
+  uint8_t* ws = nullptr;
+  int64_t launches = 0;
+  // profiling of the dominant kernel
+  int profile_mode = 0;
+  std::vector<cudaEvent_t> ev_start, ev_stop;
+  size_t ev_used = 0;
+};
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+vosti_status build_kv_map(vosti_ctx* ctx) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn)
+    return VOSTI_ERR_CUDA;
+  const vosti_config& c = ctx->cfg;
+  // The pool as a 2-D bf16 tensor: rows = (page, kv_head, K|V, slot), columns = head_dim.
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(c.head_dim),
+                              static_cast<cuuint64_t>(c.num_pages) * c.n_kv_heads * 2 * c.page_size};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(c.head_dim) * 2};
+  const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(c.page_size)};  // 128 bytes x one page
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiledFn>(fn)(
+      &ctx->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.kv_pool, dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+// Claim the next pinned staging buffer, waiting for its previous copy if needed.
+vosti_status claim_slot(vosti_ctx* ctx, HostSlot** out) {
+  HostSlot* s = &ctx->slots[ctx->next_slot];
+  ctx->next_slot = (ctx->next_slot + 1) % kHostSlots;
+  if (s->in_flight) {
+    if (cudaEventSynchronize(s->copied) != cudaSuccess) return VOSTI_ERR_CUDA;
+    s->in_flight = false;
+  }
+  *out = s;
+  return VOSTI_OK;
+}
+
+vosti_status push_blob(vosti_ctx* ctx, HostSlot* s, size_t bytes, cudaStream_t stream) {
+  if (cudaMemcpyAsync(ctx->ws + ctx->lim.off_meta, s->pinned, bytes, cudaMemcpyHostToDevice, stream) !=
+      cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  if (cudaEventRecord(s->copied, stream) != cudaSuccess) return VOSTI_ERR_CUDA;
+  s->in_flight = true;
+  return VOSTI_OK;
+}
+
+template <int D>
+vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_split, int64_t n_seq,
+                              cudaStream_t stream) {
+  using Cfg = WarpKernelCfg<D>;
+  const int Hkv = ctx->cfg.n_kv_heads;
+  const bool prof = ctx->profile_mode != 0;
+  auto timed = [&](int mode, auto&& launch) {
+    const bool rec = prof && ctx->profile_mode == mode;
+    if (rec) {
+      if (ctx->ev_used == ctx->ev_start.size()) {
+        cudaEvent_t a, b;
+        cudaEventCreate(&a);
+        cudaEventCreate(&b);
+        ctx->ev_start.push_back(a);
+        ctx->ev_stop.push_back(b);
+      }
+      cudaEventRecord(ctx->ev_start[ctx->ev_used], stream);
+    }
+    launch();
+    if (rec) cudaEventRecord(ctx->ev_stop[ctx->ev_used++], stream);
+    ++ctx->launches;
+  };
+  if (n_split > 0) {
+    AttnParams p = base;
+    p.n_workers = static_cast<int32_t>(n_split * Hkv);
+    const int grid = (p.n_workers + kWarpsPerCta - 1) / kWarpsPerCta;
+    timed(1, [&] {
+      attn_warp_kernel<D, false><<<grid, kWarpsPerCta * 32, Cfg::kSmemBytes, stream>>>(ctx->kv_map, p);
+    });
+  }
+  if (n_seq > 0) {
+    AttnParams p = base;
+    p.items = base.items + n_split;
+    p.n_workers = static_cast<int32_t>(n_seq * Hkv);
+    const int grid = (p.n_workers + kWarpsPerCta - 1) / kWarpsPerCta;
+    timed(2, [&] {
+      attn_warp_kernel<D, true><<<grid, kWarpsPerCta * 32, Cfg::kSmemBytes, stream>>>(ctx->kv_map, p);
+    });
+  }
+  if (base.n_split_tokens > 0) {
+    const int warps = base.n_split_tokens * base.Hq;
+    timed(3, [&] { combine_kernel<D><<<(warps + 3) / 4, 128, 0, stream>>>(base); });
+  }
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+template <int D>
+vosti_status set_kernel_attributes() {
+  using Cfg = WarpKernelCfg<D>;
+  if (cudaFuncSetAttribute(attn_warp_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           Cfg::kSmemBytes) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  if (cudaFuncSetAttribute(attn_warp_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           Cfg::kSmemBytes) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  return VOSTI_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* vosti_status_string(vosti_status s) {
+  switch (s) {
+    case VOSTI_OK: return "ok";
+    case VOSTI_ERR_INVALID_ARG: return "invalid argument";
+    case VOSTI_ERR_UNSUPPORTED_CONFIG: return "unsupported configuration";
+    case VOSTI_ERR_OUT_OF_RANGE: return "length or page id out of range";
+    case VOSTI_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case VOSTI_ERR_CUDA: return "CUDA call failed";
+    case VOSTI_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+void vosti_constants(int32_t* key_tile, int32_t* split_len, int32_t* rows_per_group) {
+  if (key_tile) *key_tile = nc::kKeyTile;
+  if (split_len) *split_len = nc::kSplitLen;
+  if (rows_per_group) *rows_per_group = nc::kRowsPerGroup;
+}
+
+uint64_t vosti_fingerprint(const vosti_ctx* ctx) {
+  uint64_t h = 1469598103934665603ull;
+  h = fnv1a(h, nc::kVersion);
+  h = fnv1a(h, nc::kKeyTile);
+  h = fnv1a(h, nc::kSplitLen);
+  h = fnv1a(h, 0x6c656674666f6c64ull);  // left fold by split index
+  h = fnv1a(h, 0x6578322e66746ull);     // ex2.approx.ftz, fused scale-and-shift
+  h = fnv1a(h, 0x6d6d6131363831ull);    // m16n8k16 bf16 chunks of 16, ascending
+  if (ctx) {
+    h = fnv1a(h, static_cast<uint64_t>(ctx->cfg.head_dim));
+    h = fnv1a(h, static_cast<uint64_t>(ctx->cfg.page_size));
+  }
+  return h;
+}
+
+size_t vosti_workspace_bytes(const vosti_config* config) {
+  if (!config || !geometry_ok(*config)) return 0;
+  return limits_of(*config).total;
+}
+
+vosti_status vosti_plan(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
+                        const int32_t* seq_lens, int32_t batch, vosti_work_item* items, int64_t cap,
+                        int64_t* n_items, int64_t* n_split, int64_t* n_partial_rows) {
+  if (!config || cap < 0 || (cap > 0 && !items)) return VOSTI_ERR_INVALID_ARG;
+  if (!geometry_ok(*config)) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  Plan plan;
+  const vosti_status st = plan_requests(*config, q_lens, start_pos, seq_lens, batch, &plan, nullptr);
+  if (st != VOSTI_OK) return st;
+  const int64_t n = static_cast<int64_t>(plan.items.size());
+  for (int64_t i = 0; i < std::min(n, cap); ++i) items[i] = plan.items[i];
+  if (n_items) *n_items = n;
+  if (n_split) *n_split = plan.n_split;
+  if (n_partial_rows) *n_partial_rows = plan.n_partial_rows;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_create(vosti_ctx** out, const vosti_config* config) {
+  if (!out || !config) return VOSTI_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!geometry_ok(*config)) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  if (!config->kv_pool || !config->workspace) return VOSTI_ERR_INVALID_ARG;
+  const Limits lim = limits_of(*config);
+  if (config->workspace_bytes < lim.total || reinterpret_cast<uintptr_t>(config->workspace) % kAlign)
+    return VOSTI_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(config->kv_pool) % kAlign) return VOSTI_ERR_INVALID_ARG;
+  vosti_ctx* ctx = new (std::nothrow) vosti_ctx();
+  if (!ctx) return VOSTI_ERR_INVALID_ARG;
+  ctx->cfg = *config;
+  ctx->lim = lim;
+  ctx->ws = static_cast<uint8_t*>(config->workspace);
+  vosti_status st = VOSTI_OK;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess) st = VOSTI_ERR_CUDA;
+  if (st == VOSTI_OK) st = build_kv_map(ctx);
+  if (st == VOSTI_OK) st = config->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
+  for (int i = 0; st == VOSTI_OK && i < kHostSlots; ++i) {
+    if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->slots[i].pinned), lim.meta_bytes, cudaHostAllocDefault) !=
+            cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->slots[i].copied, cudaEventDisableTiming) != cudaSuccess)
+      st = VOSTI_ERR_CUDA;
+  }
+  if (st == VOSTI_OK && cudaMemset(ctx->ws + lim.off_status, 0, kAlign) != cudaSuccess) st = VOSTI_ERR_CUDA;
+  if (st == VOSTI_OK && cudaDeviceSynchronize() != cudaSuccess) st = VOSTI_ERR_CUDA;
+  if (st != VOSTI_OK) {
+    vosti_destroy(ctx);
+    return st;
+  }
+  *out = ctx;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_destroy(vosti_ctx* ctx) {
+  if (!ctx) return VOSTI_OK;
+  for (auto& s : ctx->slots) {
+    if (s.in_flight) cudaEventSynchronize(s.copied);
+    if (s.copied) cudaEventDestroy(s.copied);
+    if (s.pinned) cudaFreeHost(s.pinned);
+  }
+  for (auto e : ctx->ev_start) cudaEventDestroy(e);
+  for (auto e : ctx->ev_stop) cudaEventDestroy(e);
+  delete ctx;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_new, const int32_t* q_lens,
+                             const int32_t* start_pos, const int32_t* block_tables,
+                             int32_t block_table_stride, int32_t batch, void* cuda_stream) {
+  if (!ctx || batch < 0 || block_table_stride < 0) return VOSTI_ERR_INVALID_ARG;
+  if (batch > 0 && (!q_lens || !start_pos || !block_tables)) return VOSTI_ERR_INVALID_ARG;
+  if (batch > ctx->cfg.max_batch) return VOSTI_ERR_OUT_OF_RANGE;
+  const vosti_config& c = ctx->cfg;
+  int64_t total = 0;
+  for (int r = 0; r < batch; ++r) {
+    if (q_lens[r] < 0 || start_pos[r] < 0) return VOSTI_ERR_OUT_OF_RANGE;
+    total += q_lens[r];
+  }
+  if (total > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
+  if (total == 0) return VOSTI_OK;
+  if (!k_new || !v_new) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) % 16) return VOSTI_ERR_INVALID_ARG;
+  HostSlot* slot = nullptr;
+  vosti_status st = claim_slot(ctx, &slot);
+  if (st != VOSTI_OK) return st;
+  int32_t* dst = reinterpret_cast<int32_t*>(slot->pinned);
+  int64_t t = 0;
+  for (int r = 0; r < batch; ++r) {
+    const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
+    for (int i = 0; i < q_lens[r]; ++i, ++t) {
+      const int64_t p = int64_t{start_pos[r]} + i;
+      const int64_t blk = p / c.page_size;
+      if (blk >= block_table_stride) return VOSTI_ERR_OUT_OF_RANGE;
+      const int64_t page = row[blk];
+      if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
+      dst[t] = static_cast<int32_t>(page * c.page_size + p % c.page_size);
+    }
+  }
+  if (c.flags & VOSTI_FLAG_CHECK_WRITE_SLOTS) {
+    std::vector<int32_t> sorted(dst, dst + total);
+    std::sort(sorted.begin(), sorted.end());
+    if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return VOSTI_ERR_OUT_OF_RANGE;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  st = push_blob(ctx, slot, sizeof(int32_t) * total, stream);
+  if (st != VOSTI_OK) return st;
+  AppendParams p;
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.pool = static_cast<__nv_bfloat16*>(c.kv_pool);
+  p.slot = reinterpret_cast<const int32_t*>(ctx->ws + ctx->lim.off_meta);
+  p.n_tokens = static_cast<int32_t>(total);
+  p.Hkv = c.n_kv_heads;
+  const int64_t warps = total * c.n_kv_heads;
+  const int grid = static_cast<int>((warps + 3) / 4);
+  if (c.head_dim == 128)
+    kv_append_kernel<128><<<grid, 128, 0, stream>>>(p);
+  else
+    kv_append_kernel<64><<<grid, 128, 0, stream>>>(p);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, const int32_t* q_lens,
+                                   const int32_t* start_pos, const int32_t* seq_lens,
+                                   const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
+                                   float softmax_scale, void* cuda_stream) {
+  if (!ctx || batch < 0 || block_table_stride < 0) return VOSTI_ERR_INVALID_ARG;
+  if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
+  if (batch > 0 && !block_tables) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  Plan plan;
+  std::vector<int64_t> part_base;
+  vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, &plan, &part_base);
+  if (st != VOSTI_OK) return st;
+  if (plan.items.empty()) return VOSTI_OK;
+  if (!q || !out) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16) return VOSTI_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(plan.items.size()) > ctx->lim.items_max ||
+      plan.n_partial_rows > ctx->lim.part_rows_max)
+    return VOSTI_ERR_WORKSPACE;
+
+  HostSlot* slot = nullptr;
+  st = claim_slot(ctx, &slot);
+  if (st != VOSTI_OK) return st;
+  // Blob: [ReqMeta x batch][items][flat page ids][split tokens]
+  const int G = c.n_q_heads / c.n_kv_heads;
+  uint8_t* blob = slot->pinned;
+  size_t at = 0;
+  ReqMeta* reqs = reinterpret_cast<ReqMeta*>(blob + at);
+  const size_t off_reqs = at;
+  at += align_up(sizeof(ReqMeta) * batch, 16);
+  const size_t off_items = at;
+  std::memcpy(blob + at, plan.items.data(), sizeof(vosti_work_item) * plan.items.size());
+  at += align_up(sizeof(vosti_work_item) * plan.items.size(), 16);
+  const size_t off_bt = at;
+  int32_t* bt_flat = reinterpret_cast<int32_t*>(blob + at);
+  int64_t bt_used = 0, row0 = 0, n_split_tokens = 0;
+  for (int r = 0; r < batch; ++r) {
+    ReqMeta& m = reqs[r];
+    m.q_row0 = static_cast<int32_t>(row0);
+    m.q_len = q_lens[r];
+    m.start = start_pos[r];
+    m.n_pages = 0;
+    m.bt_off = static_cast<int32_t>(bt_used);
+    m.n_splits = 0;
+    m.part_base = part_base[r];
+    row0 += q_lens[r];
+    if (q_lens[r] == 0) continue;
+    const int64_t n_eff = int64_t{start_pos[r]} + q_lens[r];
+    const int64_t n_pages = (n_eff + c.page_size - 1) / c.page_size;
+    if (n_pages > block_table_stride ||
+        (int64_t{seq_lens[r]} + c.page_size - 1) / c.page_size > block_table_stride)
+      return VOSTI_ERR_OUT_OF_RANGE;
+    const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
+    for (int64_t b = 0; b < n_pages; ++b) {
+      const int32_t page = row[b];
+      if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
+      bt_flat[bt_used + b] = page;
+    }
+    bt_used += n_pages;
+    m.n_pages = static_cast<int32_t>(n_pages);
+    m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1);
+    if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
+  }
+  at += align_up(sizeof(int32_t) * bt_used, 16);
+  const size_t off_tok = at;
+  int2* toks = reinterpret_cast<int2*>(blob + at);
+  {
+    int64_t x = 0;
+    for (int r = 0; r < batch; ++r)
+      if (q_lens[r] > 0 && int64_t{q_lens[r]} * G <= nc::kSplitRowsMax)
+        for (int i = 0; i < q_lens[r]; ++i) toks[x++] = make_int2(r, i);
+  }
+  at += align_up(sizeof(int2) * n_split_tokens, 16);
+
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  st = push_blob(ctx, slot, at, stream);
+  if (st != VOSTI_OK) return st;
+
+  uint8_t* dmeta = ctx->ws + ctx->lim.off_meta;
+  AttnParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.reqs = reinterpret_cast<const ReqMeta*>(dmeta + off_reqs);
+  p.items = reinterpret_cast<const vosti_work_item*>(dmeta + off_items);
+  p.bt_flat = reinterpret_cast<const int32_t*>(dmeta + off_bt);
+  p.split_tokens = reinterpret_cast<const int2*>(dmeta + off_tok);
+  p.ws_u = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_part_u);
+  p.ws_mz = reinterpret_cast<float2*>(ctx->ws + ctx->lim.off_part_mz);
+  p.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status);
+  p.n_workers = 0;
+  p.n_split_tokens = static_cast<int32_t>(n_split_tokens);
+  p.Hq = c.n_q_heads;
+  p.Hkv = c.n_kv_heads;
+  p.G = G;
+  p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
+  const int64_t n_seq = static_cast<int64_t>(plan.items.size()) - plan.n_split;
+  return c.head_dim == 128 ? launch_attention<128>(ctx, p, plan.n_split, n_seq, stream)
+                           : launch_attention<64>(ctx, p, plan.n_split, n_seq, stream);
+}
+
+vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
+                             const void* v_new_host, const int32_t* q_lens, const int32_t* start_pos,
+                             const int32_t* seq_lens, const int32_t* block_tables,
+                             int32_t block_table_stride, int32_t batch, float softmax_scale,
+                             void* cuda_stream) {
+  if (!ctx || batch < 0) return VOSTI_ERR_INVALID_ARG;
+  if (batch > 0 && !q_lens) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  int64_t total = 0;
+  for (int r = 0; r < batch; ++r) {
+    if (q_lens[r] < 0) return VOSTI_ERR_OUT_OF_RANGE;
+    total += q_lens[r];
+  }
+  if (total > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
+  if (total == 0) return VOSTI_OK;
+  if (!q_host || !out_host || !k_new_host || !v_new_host) return VOSTI_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t qbytes = sizeof(__nv_bfloat16) * total * c.n_q_heads * c.head_dim;
+  const size_t kbytes = sizeof(__nv_bfloat16) * total * c.n_kv_heads * c.head_dim;
+  uint8_t* dq = ctx->ws + ctx->lim.off_stage_q;
+  uint8_t* dout = ctx->ws + ctx->lim.off_stage_o;
+  uint8_t* dk = ctx->ws + ctx->lim.off_stage_k;
+  uint8_t* dv = ctx->ws + ctx->lim.off_stage_v;
+  if (cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(dk, k_new_host, kbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v_new_host, kbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  vosti_status st =
+      vosti_kv_append(ctx, dk, dv, q_lens, start_pos, block_tables, block_table_stride, batch, stream);
+  if (st != VOSTI_OK) return st;
+  st = vosti_paged_attention(ctx, dq, dout, q_lens, start_pos, seq_lens, block_tables, block_table_stride,
+                             batch, softmax_scale, stream);
+  if (st != VOSTI_OK) return st;
+  if (cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return VOSTI_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  uint8_t* d = ctx->ws + ctx->lim.off_status;
+  if (cudaMemcpyAsync(&word, d, sizeof word, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemsetAsync(d, 0, sizeof word, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  return (word & kStatusTimeout) ? VOSTI_ERR_TIMEOUT : VOSTI_OK;
+}
+
+vosti_status vosti_profile_enable(vosti_ctx* ctx, int32_t mode) {
+  if (!ctx || mode < 0 || mode > 3) return VOSTI_ERR_INVALID_ARG;
+  ctx->profile_mode = mode;
+  if (mode) ctx->ev_used = 0;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* kernels_timed) {
+  if (!ctx) return VOSTI_ERR_INVALID_ARG;
+  double sum = 0.0;
+  for (size_t i = 0; i < ctx->ev_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(ctx->ev_stop[i]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, ctx->ev_start[i], ctx->ev_stop[i]) != cudaSuccess)
+      return VOSTI_ERR_CUDA;
+    sum += ms;
+  }
+  if (kernel_ms_sum) *kernel_ms_sum = sum;
+  if (kernels_timed) *kernels_timed = static_cast<int64_t>(ctx->ev_used);
+  return VOSTI_OK;
+}
+
+int64_t vosti_launch_count(const vosti_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,73 @@
+"""Helpers for the GPU tests: run call schedules through the C-ABI and collect
+output rows per (request, position); run the same logical requests through the
+CPU oracle."""
+from __future__ import annotations
+
+from typing import Dict, List, Sequence, Tuple
+
+import numpy as np
+import torch
+
+from paper_2609_38981_b200 import inputs
+from paper_2609_38981_b200.harness import DeviceCache, bf16_bits
+
+Call = List[Tuple[int, int, int]]          # (request index, start position, q_len)
+
+
+def run_schedule(cache: DeviceCache, reqs, tables, schedule: Sequence[Call], scale: float,
+                 stride=None, fill=-1, append=True, seq_lens_override=None) -> Dict[int, torch.Tensor]:
+    """Each call appends its tokens then attends.  Returns, per request, an int16
+    tensor [n, Hq, d] with the bf16 bits of every computed row (rows never
+    computed stay at a sentinel)."""
+    geo = cache.geo
+    outs = {i: torch.full((r.n, geo.n_q_heads, geo.head_dim), 0x7FC2, dtype=torch.int16)
+            for i, r in enumerate(reqs)}
+    for call in schedule:
+        idx = [i for i, _, _ in call]
+        starts = [s for _, s, _ in call]
+        qls = [q for _, _, q in call]
+        bt = inputs.block_table_array([tables[i] for i in idx], stride=stride, fill=fill)
+        if append:
+            k = torch.cat([reqs[i].k[s:s + q] for i, s, q in call])
+            v = torch.cat([reqs[i].v[s:s + q] for i, s, q in call])
+            cache.append(k, v, qls, starts, bt)
+        seq = [s + q for s, q in zip(starts, qls)] if seq_lens_override is None else \
+            [seq_lens_override[i] for i in idx]
+        qt = torch.cat([reqs[i].q_rows(s, q) for i, s, q in call])
+        out = bf16_bits(cache.attend(qt, qls, starts, seq, bt, scale))
+        at = 0
+        for i, s, q in call:
+            outs[i][s:s + q] = out[at:at + q]
+            at += q
+    return outs
+
+
+def chunked(n: int, chunk: int, start: int = 0) -> List[Tuple[int, int]]:
+    return [(s, min(chunk, n - s)) for s in range(start, n, chunk)]
+
+
+def oracle_rows(reqs, scale):
+    """Dense fp64 oracle output for every position of every request."""
+    from oracle import oracle
+    return [oracle.attention_dense(inputs.bits(r.q), inputs.bits(r.k), inputs.bits(r.v), r.q0, scale)
+            for r in reqs]
+
+
+def widen_bits(t: torch.Tensor) -> np.ndarray:
+    return t.view(torch.bfloat16).to(torch.float64).numpy()
+
+
+def assert_parity(got_bits: torch.Tensor, ref: np.ndarray, what=""):
+    """The stated tolerance: max abs error <= 1e-2, mean abs error <= 1e-3."""
+    err = np.abs(widen_bits(got_bits) - ref)
+    assert np.isfinite(err).all(), f"{what}: non-finite output"
+    assert err.max() <= 1e-2, f"{what}: max abs err {err.max():.3e}"
+    assert err.mean() <= 1e-3, f"{what}: mean abs err {err.mean():.3e}"
+    return float(err.max()), float(err.mean())
+
+
+def assert_same_bits(a: torch.Tensor, b: torch.Tensor, what=""):
+    if not torch.equal(a, b):
+        bad = (a != b).reshape(a.shape[0], -1).any(dim=1).nonzero().flatten()
+        raise AssertionError(f"{what}: {bad.numel()} of {a.shape[0]} rows differ bitwise, "
+                             f"first at positions {bad[:8].tolist()}")

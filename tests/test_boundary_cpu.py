@@ -1,0 +1,121 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every
+symbol the header declares, and its host-only entry points (planning,
+workspace sizing, constants, status strings) behave as documented."""
+import os
+import re
+import ctypes
+
+import numpy as np
+import pytest
+
+from paper_2609_38981_b200 import build as vbuild
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def vb():
+    vbuild.build()
+    from paper_2609_38981_b200 import binding
+    return binding
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "vosti.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vosti_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(vb):
+    names = declared_functions()
+    assert len(names) >= 14
+    lib = ctypes.CDLL(vb.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in vosti.h but not exported"
+    assert sorted(vb.EXPORTS) == names
+
+
+def test_constants_and_fingerprint(vb):
+    c = vb.vosti_constants()
+    assert c == {"key_tile": 64, "split_len": 512, "rows_per_group": 16}
+    assert vb.vosti_fingerprint() == vb.vosti_fingerprint() != 0
+    assert vb.vosti_status_string(0) == "ok" and "range" in vb.vosti_status_string(3)
+
+
+def cfg(vb, hq=32, hkv=8, d=128, P=16, pages=1000, mb=64, mq=4096, ms=8192):
+    return vb.make_config(hq, hkv, d, P, pages, mb, mq, ms)
+
+
+def test_unsupported_geometry_is_rejected_not_tuned(vb):
+    assert vb.vosti_workspace_bytes(cfg(vb)) > 0
+    for bad in (dict(d=96), dict(P=32), dict(hq=30), dict(hq=24, hkv=8), dict(pages=0)):
+        assert vb.vosti_workspace_bytes(cfg(vb, **bad)) == 0
+        with pytest.raises(vb.VostiError) as e:
+            vb.vosti_plan(cfg(vb, **bad), [1], [0], [1])
+        assert e.value.status == vb.VOSTI_ERR_UNSUPPORTED_CONFIG
+
+
+def test_plan_premises(vb):
+    c = cfg(vb)
+    for q, s, n in (([2], [5], [6]), ([-1], [0], [4]), ([1], [-1], [4]), ([1], [0], [9000]),
+                    ([4097], [0], [4097])):
+        with pytest.raises(vb.VostiError) as e:
+            vb.vosti_plan(c, q, s, n)
+        assert e.value.status == vb.VOSTI_ERR_OUT_OF_RANGE
+    items, n_split, n_part = vb.vosti_plan(c, [0, 0], [0, 3], [0, 3])
+    assert len(items) == 0 and n_split == 0 and n_part == 0
+
+
+def plan_of_request(vb, c, q, s):
+    items, n_split, n_part = vb.vosti_plan(c, [q], [s], [s + q])
+    return sorted(map(tuple, items[:, 1:])), n_split, n_part
+
+
+def test_plan_is_a_pure_function_of_the_request(vb):
+    """Co-batching, batch order and seq_len slack must not change which
+    (row group, split range) items a request gets."""
+    c = cfg(vb)
+    rng = np.random.default_rng(0)
+    reqs = [(1, 511), (1, 512), (1, 4095), (3, 1000), (8, 2047), (9, 100), (512, 0), (512, 7000),
+            (128, 512), (1, 0)]
+    alone = {r: plan_of_request(vb, c, *r) for r in reqs}
+    for _ in range(5):
+        order = rng.permutation(len(reqs))
+        q = [reqs[i][0] for i in order]
+        s = [reqs[i][1] for i in order]
+        n = [a + b + int(rng.integers(0, 50)) for a, b in zip(q, s)]
+        items, n_split, n_part = vb.vosti_plan(c, q, s, n)
+        for slot, i in enumerate(order):
+            mine = sorted(tuple(it[1:]) for it in items if it[0] == slot)
+            assert mine == alone[reqs[i]][0]
+        assert n_split == sum(a[1] for a in alone.values())
+        assert n_part == sum(a[2] for a in alone.values())
+
+
+def test_plan_shapes(vb):
+    c = cfg(vb)          # G = 4, rows per group 16, split 512, split-parallel up to 32 rows
+    # decode at p = 1300: splits 0,1,2, one row group, split-parallel
+    items, n_split, n_part = plan_of_request(vb, c, 1, 1300)
+    assert items == [(0, 0, 1), (0, 1, 2), (0, 2, 3)] and n_split == 3
+    assert n_part == 8 * 3 * 4                      # kv heads x splits x rows
+    # 8 tokens x G=4 = 32 rows: two row groups, still split-parallel
+    items, n_split, _ = plan_of_request(vb, c, 8, 508)   # positions 508..515
+    assert items == [(0, 0, 1), (1, 0, 1), (1, 1, 2)] and n_split == 3
+    # 9 tokens: 36 rows > 32 -> sequential items that walk all their splits
+    items, n_split, n_part = plan_of_request(vb, c, 9, 1020)
+    assert n_split == 0 and n_part == 0
+    assert items == [(0, 0, 2), (1, 0, 3), (2, 0, 3)]
+    # boundaries: position exactly at a split edge
+    assert plan_of_request(vb, c, 1, 511)[0] == [(0, 0, 1)]
+    assert plan_of_request(vb, c, 1, 512)[0] == [(0, 0, 1), (0, 1, 2)]
+
+
+def test_items_are_ordered_longest_first(vb):
+    c = cfg(vb)
+    items, n_split, _ = vb.vosti_plan(c, [1, 1, 1], [100, 4000, 700], [101, 4001, 701])
+    # tiles walked per split-parallel item
+    def tiles(it):
+        p = [100, 4000, 700][it[0]]
+        return min(it[3] * 8, p // 64 + 1) - it[2] * 8
+    t = [tiles(it) for it in items[:n_split]]
+    assert t == sorted(t, reverse=True)
