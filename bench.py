@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the batch-invariant paged-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+One step = one pass of the whole path over one decode-heavy batch:
+vosti_kv_append of the batch's 64 new tokens, then vosti_paged_attention
+(work planning, page gathers, QK^T, online softmax, PV, split partials,
+cross-split combine).  The workload is the decode-heavy recipe: 32 query /
+8 KV heads, head_dim 128, page size 16, batch 64, one query token each,
+contexts uniform in [512, 4096], pages scattered over a 200k-page pool.
+
+Prints ONE JSON line (rank 0).  `value` is KV GB/s with inputs resident in
+HBM; `e2e` is the same metric through vosti_step_host with pinned host
+buffers; `roofline` is the split-parallel attention kernel against the
+measured HBM copy peak; `cpu_baseline` is the fp64 oracle on the host cores.
+With N > 1 every rank runs its own batch (different seed) on its own GPU:
+no collective on the data path, weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import re
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "decode paged-attn KV GB/s"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="vosti", choices=["vosti", "reference"])
+    ap.add_argument("--workload", default="decode_heavy",
+                    choices=["decode_heavy", "prefix_sharing", "long_context_speculative",
+                             "mixed_chunked_prefill"])
+    ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def make_workload(name: str, rank: int):
+    from paper_2609_38981_b200 import inputs
+    fn = getattr(inputs, name)
+    base = {"decode_heavy": 2, "mixed_chunked_prefill": 3, "prefix_sharing": 4,
+            "long_context_speculative": 5}[name]
+    return fn(seed=inputs.BASE_SEED * 10 + base + 1000 * rank)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def ncu_traffic_per_launch(workload: str):
+    """dram bytes per launch of the dominant kernel from the committed ncu summary, if any."""
+    path = os.path.join(ROOT, "profiles", f"attn_split_kernel_{workload}.md")
+    try:
+        m = re.search(r"dram_bytes_per_launch:\s*([0-9.eE+]+)", open(path).read())
+        return float(m.group(1)) if m else None
+    except Exception:
+        return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake",
+        }
+        while not self._halt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, nm in names.items():
+                    if mask & bit:
+                        self.reasons.add(nm)
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def stop(self):
+        self._halt.set()
+        self.join(timeout=2)
+        med = sorted(self.samples)[len(self.samples) // 2] if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def oracle_step_factory(w):
+    """Builds the oracle's view of the workload (a compact host pool holding only
+    the used pages, page ids renumbered) and returns a function running one step."""
+    import numpy as np
+    import torch
+    from oracle import oracle
+    from paper_2609_38981_b200 import inputs
+    geo = w.geo
+    seen, tables = {}, []
+    for tb in w.tables:
+        tables.append([seen.setdefault(p, len(seen)) for p in tb])
+    pool = np.zeros((len(seen), geo.n_kv_heads, 2, geo.page_size, geo.head_dim), dtype=np.uint16)
+    bt = inputs.block_table_array(tables)
+    for r, tb, s in zip(w.requests, tables, w.start_pos):   # cached context, shared pages once
+        oracle.kv_append(pool, inputs.bits(r.k[:s]), inputs.bits(r.v[:s]), [s], [0],
+                         inputs.block_table_array([tb]))
+    q = inputs.bits(w.packed_q())
+    kn, vn = w.packed_new_kv()
+    kn, vn = inputs.bits(kn), inputs.bits(vn)
+    scale = geo.head_dim ** -0.5
+
+    def step():
+        oracle.kv_append(pool, kn, vn, w.q_lens, w.start_pos, bt)
+        return oracle.paged_attention(q, pool, w.q_lens, w.start_pos, w.seq_lens, bt,
+                                      n_kv_heads=geo.n_kv_heads, page_size=geo.page_size,
+                                      scale=scale)
+    return step, oracle.num_threads()
+
+
+def run_reference(args):
+    """The reference arm: the fp64 oracle, as it stands, on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = make_workload(args.workload, 0)
+    step, cores = oracle_step_factory(w)
+    steps = max(1, min(args.steps, 20))
+    warm = max(0, min(args.warmup, 2))
+    for _ in range(warm):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    dt = (time.perf_counter() - t0) / steps
+    val = w.kv_bytes() / dt / 1e9
+    sample = f"full {w.name} step (batch {w.batch}, {sum(w.seq_lens)} cached tokens), {steps} timed steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "geometry": "32q/8kv/d128/page16"},
+        "tokens_per_s": w.total_q / dt,
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import numpy as np
+    import torch
+    from paper_2609_38981_b200 import binding as vb
+    from paper_2609_38981_b200 import inputs
+    from paper_2609_38981_b200.harness import DeviceCache
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    w = make_workload(args.workload, rank)
+    geo = w.geo
+    scale = geo.head_dim ** -0.5
+    max_seq = max(w.seq_lens)
+    cache = DeviceCache(geo, w.num_pages, max_batch=w.batch, max_total_q=max(8192, w.total_q),
+                        max_seq_len=max_seq, device=f"cuda:{local}")
+    cache.upload(w.requests, w.tables, upto=w.start_pos)      # cached context before the step
+    bt = inputs.block_table_array(w.tables)
+    ql, st, sl = (np.asarray(x, dtype=np.int32) for x in (w.q_lens, w.start_pos, w.seq_lens))
+    q_cpu = w.packed_q().contiguous()
+    kn_cpu, vn_cpu = (t.contiguous() for t in w.packed_new_kv())
+    dev = cache.device
+    q, kn, vn = q_cpu.to(dev), kn_cpu.to(dev), vn_cpu.to(dev)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        vb.vosti_kv_append(cache.ctx, kn, vn, ql, st, bt, stream=stream)
+        vb.vosti_paged_attention(cache.ctx, q, out, ql, st, sl, bt, scale, stream=stream)
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
+        step()
+    sync_all()
+    assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_OK
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    vb.vosti_profile_enable(cache.ctx, 1)
+    launches0 = vb.vosti_launch_count(cache.ctx)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    h0 = time.perf_counter()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step()
+    ev1.record(stream)
+    host_enqueue_s = time.perf_counter() - h0
+    sync_all()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop()
+    kernel_ms, kernels_timed = vb.vosti_profile_read(cache.ctx)
+    vb.vosti_profile_enable(cache.ctx, 0)
+    launches = vb.vosti_launch_count(cache.ctx) - launches0
+    assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_OK
+
+    # end to end: host buffers in, host buffer out, every step
+    pin = lambda t: t.pin_memory()
+    qh, knh, vnh = pin(q_cpu), pin(kn_cpu), pin(vn_cpu)
+    outh = torch.empty_like(q_cpu).pin_memory()
+    for _ in range(3):
+        vb.vosti_step_host(cache.ctx, qh, outh, knh, vnh, ql, st, sl, bt, scale, stream=stream)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        vb.vosti_step_host(cache.ctx, qh, outh, knh, vnh, ql, st, sl, bt, scale, stream=stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = max(e0.elapsed_time(e1), (time.perf_counter() - t0) * 1e3) / args.e2e_steps
+    out_match = bool(torch.equal(outh.view(torch.int16), out.cpu().view(torch.int16)))
+
+    kv_bytes = float(w.kv_bytes())
+    t_max, e2e_max, bytes_all, tok_all = elapsed_ms, e2e_ms, kv_bytes, float(w.total_q)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        s = torch.tensor([kv_bytes, float(w.total_q)], device=dev, dtype=torch.float64)
+        dist.all_reduce(s, op=dist.ReduceOp.SUM)
+        t_max, e2e_max = float(t[0]), float(t[1])
+        bytes_all, tok_all = float(s[0]), float(s[1])
+    ms_per_step = t_max / args.steps
+    value = bytes_all / (ms_per_step * 1e-3) / 1e9
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        k_ms = kernel_ms / max(kernels_timed, 1)
+        achieved = kv_bytes / (k_ms * 1e-3) / 1e9 if kernels_timed else None
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {
+                "workload": w.name, "batch": w.batch, "geometry":
+                    f"{geo.n_q_heads}q/{geo.n_kv_heads}kv/d{geo.head_dim}/page{geo.page_size}",
+                "cached_tokens": int(sum(w.seq_lens)), "pool_pages": w.num_pages,
+                "kv_bytes_per_step": int(kv_bytes),
+                "l2": "inputs larger than L2 (KV read per step exceeds 126 MB), no flush",
+                "step": "vosti_kv_append + vosti_paged_attention",
+            },
+            "tokens_per_s": tok_all / (ms_per_step * 1e-3),
+            "pct_of_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,
+            "host_enqueue_us_per_step": host_enqueue_s / args.steps * 1e6,
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "e2e": {"value": bytes_all / (e2e_max * 1e-3) / 1e9, "unit": UNIT,
+                    "h2d_bytes_per_step": int(qh.nbytes + knh.nbytes + vnh.nbytes + bt.nbytes
+                                              + ql.nbytes + st.nbytes + sl.nbytes),
+                    "d2h_bytes_per_step": int(outh.nbytes), "ms_per_step": e2e_max,
+                    "output_equals_device_path": out_match},
+            "roofline": {"bound": "hbm", "kernel": "attn_warp_kernel<128,false>",
+                         "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": (achieved / peak) if achieved else None,
+                         "frac_of_8TBs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
+                         "peak_source": peak_src, "kernel_us": k_ms * 1e3,
+                         "launches_timed": int(kernels_timed),
+                         "traffic": ncu_traffic_per_launch(w.name)},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            ostep, cores = oracle_step_factory(w)
+            ostep()
+            reps = 8
+            c0 = time.perf_counter()
+            for _ in range(reps):
+                ref = ostep()
+            cdt = (time.perf_counter() - c0) / reps
+            got = out.cpu().to(torch.float64).numpy()
+            err = np.abs(got - ref)
+            line["cpu_baseline"] = {
+                "value": kv_bytes / cdt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"the full {w.name} step, {reps} repetitions ({cdt * 1e3:.0f} ms each)"}
+            line["parity"] = {"max_abs_err": float(err.max()), "mean_abs_err": float(err.mean()),
+                              "rows": int(got.shape[0] * got.shape[1])}
+        print(json.dumps(line))
+    cache.close()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
