@@ -1,0 +1,261 @@
+// Split-parallel attention (decode, speculative and other short queries): a
+// persistent kernel, one CTA per SM, four independent warp workers per CTA.
+//
+// A worker draws (item, KV head) tickets from a global counter.  An item is one
+// KV split (512 keys) of one 16-row group of a request; the worker walks its
+// key tiles in ascending order and writes the partial (m, z, U) of the rows
+// that see the split.  Each worker owns a ring of shared-memory stages filled
+// by its own TMA page gathers; the load stream runs ahead of the consumer
+// across item boundaries, so the ring stays full while one item ends and the
+// next begins.  Which worker runs which item, and when, has no effect on the
+// bits: partials are folded later in split order.
+#pragma once
+#include "meta.cuh"
+#include "tile_math.cuh"
+
+namespace vosti {
+
+constexpr uint32_t kStatusTimeout = 1u;
+
+// Eight workers per SM (two per scheduler, so one worker's instruction latency
+// hides behind the other's); each owns kStages stages of 32 keys (K or V).
+template <int D>
+struct SplitKernelCfg {
+  static constexpr int kWarps = 8;
+  static constexpr int kStageKeys = 32;
+  static constexpr int kStages = (D == 128) ? 3 : 6;
+  static constexpr int kSmemBytes =
+      kWarps * kStages * TileCfg<D, kStageKeys>::kStageBytes + kWarps * kStages * 8 + 1024;
+};
+
+template <int D>
+__global__ void __launch_bounds__(SplitKernelCfg<D>::kWarps * 32, 1)
+attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {
+  constexpr int SK = SplitKernelCfg<D>::kStageKeys;
+  using C = TileCfg<D, SK>;
+  constexpr int kWarpsPerCta = SplitKernelCfg<D>::kWarps;
+  constexpr int R = SplitKernelCfg<D>::kStages;
+  constexpr int TPS = nc::kTilesPerSplit;
+  constexpr int LPT = 2 * C::kParts;  // loads per tile: K parts then V parts
+
+  extern __shared__ uint8_t smem_raw[];
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int quad = lane & 3;
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t stage0 = base + warp * R * C::kStageBytes;
+  const uint32_t bar0 = base + kWarpsPerCta * R * C::kStageBytes + warp * R * 8;
+
+  if (lane == 0) {
+    tma_prefetch_desc(&kv_map);
+#pragma unroll
+    for (int s = 0; s < R; ++s) mbar_init(bar0 + s * 8, 1);
+    mbar_fence_init();
+    fence_proxy_async();
+  }
+  __syncwarp();
+
+  const int G = P.G;
+  const float c = P.c;
+
+  // ---- tickets ---------------------------------------------------------------
+  // Producer-side description of an item: enough to issue its loads.
+  struct Desc {
+    uint32_t ticket;
+    int kvh, t_begin, n_loads, n_pages, ids;
+  };
+  auto read_item = [&](uint32_t ticket) -> SplitItem {
+    const int4* src = reinterpret_cast<const int4*>(P.split_items + ticket / P.Hkv);
+    const int4 a = __ldg(src), b = __ldg(src + 1), d = __ldg(src + 2);
+    SplitItem si;
+    si.q_row0 = a.x; si.q_len = a.y; si.start = a.z; si.n_pages = a.w;
+    si.bt_index = b.x; si.split = b.y; si.row_group = b.z; si.n_splits = b.w;
+    si.part_base = (static_cast<int64_t>(static_cast<uint32_t>(d.y)) << 32) | static_cast<uint32_t>(d.x);
+    si.req = d.z; si.pad = d.w;
+    return si;
+  };
+  // The first ticket of worker w is w itself; later ones come from the counter.
+  const uint32_t n_static = gridDim.x * kWarpsPerCta;
+  auto draw = [&](Desc& d, bool first) -> bool {
+    uint32_t t = blockIdx.x * kWarpsPerCta + warp;
+    if (!first) {
+      if (lane == 0) t = n_static + atomicAdd(P.ticket, 1u);
+      t = __shfl_sync(kFullMask, t, 0);
+    }
+    if (t >= static_cast<uint32_t>(P.n_workers)) return false;
+    const SplitItem si = read_item(t);
+    const int last_tok = min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
+    const int t_end = min((si.split + 1) * TPS, (si.start + last_tok) / nc::kKeyTile + 1);
+    d.ticket = t;
+    d.kvh = static_cast<int>(t % P.Hkv);
+    d.t_begin = si.split * TPS;
+    d.n_loads = LPT * (t_end - d.t_begin);
+    d.n_pages = si.n_pages;
+    d.ids = (si.split * nc::kPagesPerSplit + lane < si.n_pages) ? __ldg(P.bt_flat + si.bt_index + lane) : -1;
+    return true;
+  };
+  auto leave = [&]() {
+    if (lane == 0) {
+      __threadfence();
+      const uint32_t d = atomicAdd(P.done, 1u);
+      if (d == gridDim.x * kWarpsPerCta - 1) {  // last worker out resets the counters
+        *P.ticket = 0u;
+        *P.done = 0u;
+        __threadfence();
+      }
+    }
+  };
+
+  Desc cur, nxt;
+  nxt.ticket = 0; nxt.kvh = 0; nxt.t_begin = 0; nxt.n_loads = 0; nxt.n_pages = 0; nxt.ids = -1;
+  if (!draw(cur, true)) {
+    leave();
+    return;
+  }
+  bool has_nxt = true;      // assumed until the second draw says otherwise
+  bool drew_second = false;
+  griddep_wait();           // the pool (appended tokens) and Q come from earlier work in the stream
+
+  // ---- load stream -------------------------------------------------------------
+  uint32_t g_issue = 0, g_cons = 0;  // loads issued / consumed since kernel start
+  int ahead = 0;                     // 0: issuing for cur, 1: for nxt, 2: nxt fully issued
+  int prod_li = 0;                   // next load of the item being issued
+  bool prod_done = false;
+  auto issue_one = [&]() -> bool {
+    if (prod_done || ahead == 2 || g_issue - g_cons >= static_cast<uint32_t>(R)) return false;
+    if (ahead == 1 && !drew_second) return false;  // nxt not drawn yet (first item only)
+    const int kvh = ahead ? nxt.kvh : cur.kvh;
+    const int t_begin = ahead ? nxt.t_begin : cur.t_begin;
+    const int n_loads = ahead ? nxt.n_loads : cur.n_loads;
+    const int n_pages = ahead ? nxt.n_pages : cur.n_pages;
+    const int ids = ahead ? nxt.ids : cur.ids;
+    const int tl = prod_li / LPT;          // tile within the split
+    const int sub = prod_li - tl * LPT;    // 0 .. kParts-1: K parts, then V parts
+    const int is_v = sub >= C::kParts;
+    const int part = sub - is_v * C::kParts;
+    const int first_page = tl * nc::kPagesPerTile + part * C::kPagesPerStage;  // within the split
+    const int stage = g_issue % R;
+    issue_stage_load<D, SK>(&kv_map, stage0 + stage * C::kStageBytes, bar0 + stage * 8, ids, first_page,
+                            max(0, min(C::kPagesPerStage, n_pages - (t_begin * nc::kPagesPerTile + first_page))),
+                            P.Hkv, kvh, is_v, lane);
+    ++g_issue;
+    if (++prod_li == n_loads) {
+      prod_li = 0;
+      ++ahead;
+      if (ahead == 1 && !has_nxt) prod_done = true;
+    }
+    return true;
+  };
+
+  bool timed_out = false;
+  while (true) {
+    while (issue_one()) {
+    }
+    // ---- consumer set-up for `cur` -----------------------------------------------
+    const SplitItem si = read_item(cur.ticket);
+    const int kvh = cur.kvh;
+    const int row_a = si.row_group * nc::kRowsPerGroup + (lane >> 2);
+    const int row_b = row_a + 8;
+    const int tok_a = row_a / G, tok_b = row_b / G;
+    const bool valid_a = tok_a < si.q_len, valid_b = tok_b < si.q_len;
+    RowPair r;
+    r.p_a = valid_a ? si.start + tok_a : -1;
+    r.p_b = valid_b ? si.start + tok_b : -1;
+    r.reset();
+    const int n_eff = si.start + si.q_len;
+    // schedule-only facts about the group: lowest real position, whether rows 8..15 hold real rows
+    const int p_min = si.start + (si.row_group * nc::kRowsPerGroup) / G;
+    const bool upper_rows = (si.row_group * nc::kRowsPerGroup + 8) / G < si.q_len;
+    uint32_t qa[C::KC][4];
+    load_q_frags<D>(qa,
+                    P.q + (static_cast<size_t>(si.q_row0 + tok_a) * P.Hq + kvh * G + row_a % G) * D,
+                    P.q + (static_cast<size_t>(si.q_row0 + tok_b) * P.Hq + kvh * G + row_b % G) * D,
+                    valid_a, valid_b, quad);
+    float u[C::NE][4];
+#pragma unroll
+    for (int e = 0; e < C::NE; ++e) u[e][0] = u[e][1] = u[e][2] = u[e][3] = 0.f;
+    if (!drew_second) {  // first item: its loads are already in flight, now draw the next one
+      drew_second = true;
+      has_nxt = draw(nxt, false);
+      if (ahead == 1 && !has_nxt) prod_done = true;
+    }
+
+    const int n_tiles = cur.n_loads / LPT;
+#pragma unroll 1
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int key0 = (cur.t_begin + tile) * nc::kKeyTile;
+      float s[8][4];
+#pragma unroll
+      for (int part = 0; part < C::kParts; ++part) {
+        const int stage = g_cons % R;
+        if (!__all_sync(kFullMask, mbar_wait_bounded(bar0 + stage * 8, (g_cons / R) & 1))) {
+          timed_out = true;  // warp-uniform: every lane leaves together
+          break;
+        }
+        tile_scores<D, SK>(stage0 + stage * C::kStageBytes, qa, s, part * (SK / 8), lane);
+        __syncwarp();
+        ++g_cons;
+        issue_one();
+      }
+      if (timed_out) break;
+      uint32_t pa[4][4];
+      tile_softmax_dispatch<D>(s, key0, c, r, u, pa, quad, key0 + nc::kKeyTile - 1 <= p_min, upper_rows);
+#pragma unroll
+      for (int part = 0; part < C::kParts; ++part) {
+        const int stage = g_cons % R;
+        if (!__all_sync(kFullMask, mbar_wait_bounded(bar0 + stage * 8, (g_cons / R) & 1))) {
+          timed_out = true;
+          break;
+        }
+        const uint32_t vs = stage0 + stage * C::kStageBytes;
+        const int part_key0 = key0 + part * SK;
+        if (part_key0 + SK > n_eff) zero_value_tail<D, SK>(vs, max(0, n_eff - part_key0), lane);
+        tile_pv<D, SK>(vs, pa, u, part * (SK / 16), lane);
+        __syncwarp();
+        ++g_cons;
+        issue_one();
+      }
+      if (timed_out) break;
+    }
+    if (timed_out) break;
+
+    // ---- partial (m, z, U) of this split for the rows that see it -----------------
+    {
+      const int rows = si.q_len * G;
+      const int64_t slab = si.part_base + (static_cast<int64_t>(kvh) * si.n_splits + si.split) * rows;
+      const int first_key = si.split * nc::kSplitLen;
+      if (valid_a && r.p_a >= first_key) {
+        float* dst = P.ws_u + (slab + row_a) * D + 2 * quad;
+#pragma unroll
+        for (int e = 0; e < C::NE; ++e)
+          *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][0], u[e][1]);
+        if (quad == 0) P.ws_mz[slab + row_a] = make_float2(r.m_a, r.z_a);
+      }
+      if (valid_b && r.p_b >= first_key) {
+        float* dst = P.ws_u + (slab + row_b) * D + 2 * quad;
+#pragma unroll
+        for (int e = 0; e < C::NE; ++e)
+          *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][2], u[e][3]);
+        if (quad == 0) P.ws_mz[slab + row_b] = make_float2(r.m_b, r.z_b);
+      }
+    }
+
+    if (!has_nxt) break;
+    cur = nxt;
+    --ahead;
+    has_nxt = draw(nxt, false);
+    if (ahead == 1 && !has_nxt) prod_done = true;
+  }
+
+  if (timed_out) {
+    if (lane == 0) atomicOr(P.status, kStatusTimeout);
+    // Give copies still in flight a bounded chance to land before the CTA's
+    // shared memory can be handed to another block.
+    const uint64_t t0 = global_timer_ns();
+    while (global_timer_ns() - t0 < 2000000ull) {
+    }
+  }
+  leave();
+}
+
+}  // namespace vosti

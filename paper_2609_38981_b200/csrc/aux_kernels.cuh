@@ -1,0 +1,91 @@
+// Cross-split combine and KV append kernels.
+#pragma once
+#include "meta.cuh"
+#include "nc_math.cuh"
+#include "ptx.cuh"
+
+namespace vosti {
+
+// Cross-split combine for split-parallel rows: one warp per (token, query
+// head) folds the partials of splits 0..floor(p / L_S) left to right, then
+// normalises.  Order depends on the split index only.
+template <int D>
+__global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
+  constexpr int V = D / 32;  // floats per lane
+  const int lane = threadIdx.x & 31;
+  const int widx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (widx >= P.n_split_tokens * P.Hq) return;
+  griddep_wait();  // partials come from the kernel before this one in the stream
+  const int2 rt = P.split_tokens[widx / P.Hq];
+  const int head = widx % P.Hq;
+  const ReqMeta rq = P.reqs[rt.x];
+  const int kvh = head / P.G;
+  const int row = rt.y * P.G + head % P.G;
+  const int rows = rq.q_len * P.G;
+  const int p = rq.start + rt.y;
+  const int n_splits = p / nc::kSplitLen + 1;
+  const int64_t slab0 = rq.part_base + static_cast<int64_t>(kvh) * rq.n_splits * rows + row;
+
+  float uc[V];
+  float mc, zc;
+  {
+    const float2 mz = P.ws_mz[slab0];
+    mc = mz.x;
+    zc = mz.y;
+    const float* src = P.ws_u + slab0 * D + lane * V;
+    if constexpr (V == 4) {
+      const float4 x = *reinterpret_cast<const float4*>(src);
+      uc[0] = x.x; uc[1] = x.y; uc[2] = x.z; uc[3] = x.w;
+    } else {
+      const float2 x = *reinterpret_cast<const float2*>(src);
+      uc[0] = x.x; uc[1] = x.y;
+    }
+  }
+#pragma unroll 4
+  for (int k = 1; k < n_splits; ++k) {
+    const int64_t slab = slab0 + static_cast<int64_t>(k) * rows;
+    const float2 mz = P.ws_mz[slab];
+    float uk[V];
+    const float* src = P.ws_u + slab * D + lane * V;
+    if constexpr (V == 4) {
+      const float4 x = *reinterpret_cast<const float4*>(src);
+      uk[0] = x.x; uk[1] = x.y; uk[2] = x.z; uk[3] = x.w;
+    } else {
+      const float2 x = *reinterpret_cast<const float2*>(src);
+      uk[0] = x.x; uk[1] = x.y;
+    }
+    const nc::FoldFactors f = nc::fold_scalars(mc, zc, mz.x, mz.y);
+#pragma unroll
+    for (int i = 0; i < V; ++i) uc[i] = nc::fold_u(uc[i], uk[i], f);
+  }
+  const float inv = nc::out_scale(zc);
+  __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + rt.y) * P.Hq + head) * D + lane * V;
+#pragma unroll
+  for (int i = 0; i < V; i += 2)
+    *reinterpret_cast<__nv_bfloat162*>(dst + i) =
+        __floats2bfloat162_rn(nc::out_value(uc[i], inv), nc::out_value(uc[i + 1], inv));
+}
+
+// KV append: one warp per (token, KV head); lanes 0-15 copy the K row, lanes
+// 16-31 the V row, 16 bytes (D = 128) or 8 bytes (D = 64) each.
+template <int D>
+__global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams P) {
+  const int lane = threadIdx.x & 31;
+  const int widx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (widx >= P.n_tokens * P.Hkv) return;
+  const int tok = widx / P.Hkv, kvh = widx % P.Hkv;
+  const int slot = P.slot ? P.slot[tok] : P.inline_slot[tok];
+  const int page = slot / nc::kPageSize, within = slot % nc::kPageSize;
+  const int is_v = lane >> 4, part = lane & 15;
+  const __nv_bfloat16* src = (is_v ? P.v_new : P.k_new) + (static_cast<size_t>(tok) * P.Hkv + kvh) * D;
+  __nv_bfloat16* dst = P.pool +
+      ((static_cast<size_t>(page) * P.Hkv + kvh) * 2 + is_v) * (nc::kPageSize * D) +
+      static_cast<size_t>(within) * D;
+  if constexpr (D == 128) {
+    reinterpret_cast<uint4*>(dst)[part] = reinterpret_cast<const uint4*>(src)[part];
+  } else {
+    reinterpret_cast<uint2*>(dst)[part] = reinterpret_cast<const uint2*>(src)[part];
+  }
+}
+
+}  // namespace vosti

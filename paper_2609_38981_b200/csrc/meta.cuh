@@ -18,11 +18,25 @@ struct ReqMeta {
   int64_t part_base;  // first partial row of the request (split-parallel requests only)
 };
 
+// One split-parallel work item, self-contained so that a persistent warp needs
+// a single record per ticket.  48 bytes.
+struct SplitItem {
+  int32_t q_row0, q_len, start, n_pages;
+  int32_t bt_index;  // index in the flat table of the first page of this split
+  int32_t split, row_group, n_splits;
+  int64_t part_base;
+  int32_t req, pad;
+};
+static_assert(sizeof(SplitItem) == 48, "SplitItem is read as three 16-byte words");
+
 struct AttnParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   const ReqMeta* reqs;
-  const vosti_work_item* items;
+  const vosti_work_item* items;    // sequential items
+  const SplitItem* split_items;    // split-parallel items, longest first
+  uint32_t* ticket;                // next split-parallel worker index (self-resetting)
+  uint32_t* done;                  // warps that have left the persistent kernel
   const int32_t* bt_flat;
   const int2* split_tokens;  // (request, token) of every row the combine kernel finishes
   float* ws_u;               // partial U rows [rows][D]
@@ -35,11 +49,13 @@ struct AttnParams {
 };
 
 struct AppendParams {
+  static constexpr int kInlineSlots = 256;
   const __nv_bfloat16* k_new;
   const __nv_bfloat16* v_new;
   __nv_bfloat16* pool;
-  const int32_t* slot;  // per token: page * P + slot
+  const int32_t* slot;  // per token: page * P + slot; nullptr: use inline_slot
   int32_t n_tokens, Hkv;
+  int32_t inline_slot[kInlineSlots];
 };
 
 }  // namespace vosti

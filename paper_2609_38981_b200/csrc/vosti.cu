@@ -5,9 +5,11 @@
 #include <cstdio>
 #include <cstring>
 #include <new>
+#include <utility>
 #include <vector>
 
-#include "attn_warp.cuh"
+#include "attn_seq.cuh"
+#include "aux_kernels.cuh"
 
 namespace vosti {
 namespace {
@@ -55,14 +57,15 @@ Limits limits_of(const vosti_config& c) {
   const int64_t rows_by_total = c.max_total_q * G;
   L.part_rows_max = std::min(rows_by_batch, rows_by_total) * c.n_kv_heads * L.k_max;
   const size_t attn_blob = align_up(sizeof(ReqMeta) * c.max_batch, 16) +
-                           align_up(sizeof(vosti_work_item) * L.items_max, 16) +
+                           align_up(sizeof(SplitItem) * items_split, 16) +
+                           align_up(sizeof(vosti_work_item) * items_seq, 16) +
                            align_up(sizeof(int32_t) * L.pages_max, 16) +
                            align_up(sizeof(int2) * c.max_total_q, 16);
   const size_t append_blob = align_up(sizeof(int32_t) * c.max_total_q, 16);
   L.meta_bytes = align_up(std::max(attn_blob, append_blob));
   size_t at = 0;
   L.off_status = at; at += kAlign;
-  L.off_meta = at; at += L.meta_bytes;
+  L.off_meta = at; at += L.meta_bytes * kHostSlots;  // one region per staging slot
   L.off_part_u = at; at += align_up(sizeof(float) * L.part_rows_max * c.head_dim);
   L.off_part_mz = at; at += align_up(sizeof(float2) * L.part_rows_max);
   const size_t qbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_q_heads * c.head_dim;
@@ -77,58 +80,83 @@ Limits limits_of(const vosti_config& c) {
 
 struct Plan {
   std::vector<vosti_work_item> items;  // split-parallel items first
+  std::vector<std::pair<int64_t, vosti_work_item>> seq_scratch;
   int64_t n_split = 0;
   int64_t n_partial_rows = 0;
 };
 
 // The plan of one request depends on its own (q_len, start) and the geometry.
+// Items are ordered longest first (by key tiles walked): split-parallel items
+// by an 8-bucket counting sort, sequential ones by a stable sort on the
+// precomputed tile count, so the order is reproducible.
 vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const int32_t* start_pos,
-                           const int32_t* seq_lens, int32_t batch, Plan* plan,
-                           std::vector<int64_t>* part_base) {
+                           const int32_t* seq_lens, int32_t batch, Plan* plan, int64_t* part_base) {
   if (batch < 0 || (batch > 0 && (!q_lens || !start_pos || !seq_lens))) return VOSTI_ERR_INVALID_ARG;
   if (batch > c.max_batch) return VOSTI_ERR_OUT_OF_RANGE;
   const int G = c.n_q_heads / c.n_kv_heads;
-  int64_t total_q = 0;
-  std::vector<vosti_work_item> split_items, seq_items;
-  if (part_base) part_base->assign(batch, 0);
+  constexpr int TPS = nc::kTilesPerSplit;
+  int64_t total_q = 0, n_split = 0, n_seq = 0, part_rows = 0;
+  int64_t bucket[TPS + 1] = {0};  // bucket[t] = split items that walk t tiles
+  // pass 1: premises, counts
   for (int r = 0; r < batch; ++r) {
     const int64_t q = q_lens[r], st = start_pos[r], n = seq_lens[r];
     if (q < 0 || st < 0 || st + q > n || n > c.max_seq_len) return VOSTI_ERR_OUT_OF_RANGE;
     total_q += q;
     if (q == 0) continue;
     const int64_t rows = q * G;
-    const int groups = static_cast<int>((rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup);
-    const bool split_parallel = rows <= nc::kSplitRowsMax;
-    if (split_parallel) {
-      if (part_base) (*part_base)[r] = plan->n_partial_rows;
-      const int64_t n_splits = (st + q - 1) / nc::kSplitLen + 1;
-      plan->n_partial_rows += int64_t{c.n_kv_heads} * n_splits * rows;
-    }
-    for (int g = 0; g < groups; ++g) {
-      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{g} * nc::kRowsPerGroup + 15) / G);
-      const int k_g = static_cast<int>((st + last_tok) / nc::kSplitLen + 1);
-      if (split_parallel) {
-        for (int k = 0; k < k_g; ++k) split_items.push_back({r, g, k, k + 1});
-      } else {
-        seq_items.push_back({r, g, 0, k_g});
+    const int64_t groups = (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+    if (rows <= nc::kSplitRowsMax) {
+      if (part_base) part_base[r] = part_rows;
+      part_rows += int64_t{c.n_kv_heads} * ((st + q - 1) / nc::kSplitLen + 1) * rows;
+      for (int64_t g = 0; g < groups; ++g) {
+        const int64_t last_tok = std::min<int64_t>(q - 1, (g * nc::kRowsPerGroup + 15) / G);
+        const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
+        const int64_t k_g = (tiles + TPS - 1) / TPS;
+        bucket[TPS] += k_g - 1;
+        bucket[tiles - (k_g - 1) * TPS] += 1;
+        n_split += k_g;
       }
+    } else {
+      if (part_base) part_base[r] = 0;
+      n_seq += groups;
     }
   }
   if (total_q > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
-  // Longest first (by key tiles walked); stable, so the order is reproducible.
-  auto tiles_of = [&](const vosti_work_item& it) {
-    const int64_t q = q_lens[it.req], st = start_pos[it.req];
-    const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{it.row_group} * nc::kRowsPerGroup + 15) / G);
-    const int64_t t_end = std::min<int64_t>(int64_t{it.split_end} * nc::kTilesPerSplit,
-                                            (st + last_tok) / nc::kKeyTile + 1);
-    return t_end - int64_t{it.split_begin} * nc::kTilesPerSplit;
-  };
-  auto longer = [&](const vosti_work_item& a, const vosti_work_item& b) { return tiles_of(a) > tiles_of(b); };
-  std::stable_sort(split_items.begin(), split_items.end(), longer);
-  std::stable_sort(seq_items.begin(), seq_items.end(), longer);
-  plan->n_split = static_cast<int64_t>(split_items.size());
-  plan->items = std::move(split_items);
-  plan->items.insert(plan->items.end(), seq_items.begin(), seq_items.end());
+  plan->items.resize(static_cast<size_t>(n_split + n_seq));
+  plan->seq_scratch.clear();
+  int64_t at[TPS + 1];
+  {
+    int64_t o = 0;
+    for (int t = TPS; t >= 1; --t) {
+      at[t] = o;
+      o += bucket[t];
+    }
+  }
+  // pass 2: fill
+  vosti_work_item* out = plan->items.data();
+  for (int r = 0; r < batch; ++r) {
+    const int64_t q = q_lens[r], st = start_pos[r];
+    if (q == 0) continue;
+    const int64_t rows = q * G;
+    const int groups = static_cast<int>((rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup);
+    const bool split_parallel = rows <= nc::kSplitRowsMax;
+    for (int g = 0; g < groups; ++g) {
+      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{g} * nc::kRowsPerGroup + 15) / G);
+      const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
+      const int k_g = static_cast<int>((tiles + TPS - 1) / TPS);
+      if (split_parallel) {
+        for (int k = 0; k + 1 < k_g; ++k) out[at[TPS]++] = {r, g, k, k + 1};
+        out[at[tiles - int64_t{k_g - 1} * TPS]++] = {r, g, k_g - 1, k_g};
+      } else {
+        plan->seq_scratch.push_back({tiles, vosti_work_item{r, g, 0, k_g}});
+      }
+    }
+  }
+  std::stable_sort(plan->seq_scratch.begin(), plan->seq_scratch.end(),
+                   [](const auto& a, const auto& b) { return a.first > b.first; });
+  for (size_t i = 0; i < plan->seq_scratch.size(); ++i) out[n_split + i] = plan->seq_scratch[i].second;
+  plan->n_split = n_split;
+  plan->n_partial_rows = part_rows;
   return VOSTI_OK;
 }
 
@@ -140,10 +168,15 @@ uint64_t fnv1a(uint64_t h, uint64_t x) {
   return h;
 }
 
+// One staging slot: a pinned host buffer, its own device metadata region, an
+// event for "copy done" and one for "kernels that read the region are done".
 struct HostSlot {
   uint8_t* pinned = nullptr;
+  uint8_t* device = nullptr;
   cudaEvent_t copied = nullptr;
+  cudaEvent_t released = nullptr;
   bool in_flight = false;
+  bool has_release = false;
 };
 
 }  // namespace
@@ -155,11 +188,15 @@ struct vosti_ctx {
   vosti_config cfg;
   Limits lim;
   int device = 0;
+  int sm_count = 1;
   alignas(64) CUtensorMap kv_map;
   HostSlot slots[kHostSlots];
   int next_slot = 0;
+  cudaStream_t copy_stream = nullptr;  // metadata uploads overlap the previous call's kernels
   uint8_t* ws = nullptr;
   int64_t launches = 0;
+  Plan plan;                       // reused across calls: no allocation in steady state
+  std::vector<int64_t> part_base;
   // profiling of the dominant kernel
   int profile_mode = 0;
   std::vector<cudaEvent_t> ev_start, ev_stop;
@@ -205,19 +242,50 @@ vosti_status claim_slot(vosti_ctx* ctx, HostSlot** out) {
   return VOSTI_OK;
 }
 
+// Upload a slot's blob on the copy stream and make `stream` wait for it.  The
+// copy itself waits until the kernels that last read the slot's device region
+// have finished.
 vosti_status push_blob(vosti_ctx* ctx, HostSlot* s, size_t bytes, cudaStream_t stream) {
-  if (cudaMemcpyAsync(ctx->ws + ctx->lim.off_meta, s->pinned, bytes, cudaMemcpyHostToDevice, stream) !=
-      cudaSuccess)
+  cudaStream_t cs = ctx->copy_stream;
+  if (s->has_release && cudaStreamWaitEvent(cs, s->released, 0) != cudaSuccess) return VOSTI_ERR_CUDA;
+  if (cudaMemcpyAsync(s->device, s->pinned, bytes, cudaMemcpyHostToDevice, cs) != cudaSuccess)
     return VOSTI_ERR_CUDA;
-  if (cudaEventRecord(s->copied, stream) != cudaSuccess) return VOSTI_ERR_CUDA;
+  if (cudaEventRecord(s->copied, cs) != cudaSuccess) return VOSTI_ERR_CUDA;
   s->in_flight = true;
+  if (cudaStreamWaitEvent(stream, s->copied, 0) != cudaSuccess) return VOSTI_ERR_CUDA;
   return VOSTI_OK;
+}
+
+// Mark the point on `stream` after which the slot's device region may be overwritten.
+vosti_status release_slot(HostSlot* s, cudaStream_t stream) {
+  if (cudaEventRecord(s->released, stream) != cudaSuccess) return VOSTI_ERR_CUDA;
+  s->has_release = true;
+  return VOSTI_OK;
+}
+
+// Launch with programmatic stream serialization: the grid may be scheduled
+// while its predecessor in the stream drains; the kernel calls griddep_wait()
+// before touching anything the predecessor wrote.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size_t smem,
+                             cudaStream_t stream, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
 template <int D>
 vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_split, int64_t n_seq,
                               cudaStream_t stream) {
-  using Cfg = WarpKernelCfg<D>;
+  using Cfg = SplitKernelCfg<D>;
   const int Hkv = ctx->cfg.n_kv_heads;
   const bool prof = ctx->profile_mode != 0;
   auto timed = [&](int mode, auto&& launch) {
@@ -239,35 +307,36 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
   if (n_split > 0) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_split * Hkv);
-    const int grid = (p.n_workers + kWarpsPerCta - 1) / kWarpsPerCta;
+    // persistent: one CTA per SM, warps draw (item, KV head) tickets
+    const int grid = std::min((p.n_workers + Cfg::kWarps - 1) / Cfg::kWarps, ctx->sm_count);
     timed(1, [&] {
-      attn_warp_kernel<D, false><<<grid, kWarpsPerCta * 32, Cfg::kSmemBytes, stream>>>(ctx->kv_map, p);
+      launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map, p);
     });
   }
   if (n_seq > 0) {
     AttnParams p = base;
-    p.items = base.items + n_split;
     p.n_workers = static_cast<int32_t>(n_seq * Hkv);
-    const int grid = (p.n_workers + kWarpsPerCta - 1) / kWarpsPerCta;
+    using SeqCfg = SeqKernelCfg<D>;
+    const int grid = (p.n_workers + SeqCfg::kWarps - 1) / SeqCfg::kWarps;
     timed(2, [&] {
-      attn_warp_kernel<D, true><<<grid, kWarpsPerCta * 32, Cfg::kSmemBytes, stream>>>(ctx->kv_map, p);
+      attn_seq_kernel<D><<<grid, SeqCfg::kWarps * 32, SeqCfg::kSmemBytes, stream>>>(ctx->kv_map, p);
     });
   }
   if (base.n_split_tokens > 0) {
     const int warps = base.n_split_tokens * base.Hq;
-    timed(3, [&] { combine_kernel<D><<<(warps + 3) / 4, 128, 0, stream>>>(base); });
+    timed(3, [&] { launch_dependent(combine_kernel<D>, (warps + 3) / 4, 128, 0, stream, base); });
   }
   return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
 }
 
 template <int D>
 vosti_status set_kernel_attributes() {
-  using Cfg = WarpKernelCfg<D>;
-  if (cudaFuncSetAttribute(attn_warp_kernel<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  using Cfg = SplitKernelCfg<D>;
+  if (cudaFuncSetAttribute(attn_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            Cfg::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
-  if (cudaFuncSetAttribute(attn_warp_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           Cfg::kSmemBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_seq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SeqKernelCfg<D>::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   return VOSTI_OK;
 }
@@ -346,13 +415,19 @@ vosti_status vosti_create(vosti_ctx** out, const vosti_config* config) {
   ctx->lim = lim;
   ctx->ws = static_cast<uint8_t*>(config->workspace);
   vosti_status st = VOSTI_OK;
-  if (cudaGetDevice(&ctx->device) != cudaSuccess) st = VOSTI_ERR_CUDA;
+  if (cudaGetDevice(&ctx->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, ctx->device) != cudaSuccess)
+    st = VOSTI_ERR_CUDA;
   if (st == VOSTI_OK) st = build_kv_map(ctx);
   if (st == VOSTI_OK) st = config->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
+  if (st == VOSTI_OK && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+    st = VOSTI_ERR_CUDA;
   for (int i = 0; st == VOSTI_OK && i < kHostSlots; ++i) {
+    ctx->slots[i].device = ctx->ws + lim.off_meta + static_cast<size_t>(i) * lim.meta_bytes;
     if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->slots[i].pinned), lim.meta_bytes, cudaHostAllocDefault) !=
             cudaSuccess ||
-        cudaEventCreateWithFlags(&ctx->slots[i].copied, cudaEventDisableTiming) != cudaSuccess)
+        cudaEventCreateWithFlags(&ctx->slots[i].copied, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->slots[i].released, cudaEventDisableTiming) != cudaSuccess)
       st = VOSTI_ERR_CUDA;
   }
   if (st == VOSTI_OK && cudaMemset(ctx->ws + lim.off_status, 0, kAlign) != cudaSuccess) st = VOSTI_ERR_CUDA;
@@ -370,7 +445,12 @@ vosti_status vosti_destroy(vosti_ctx* ctx) {
   for (auto& s : ctx->slots) {
     if (s.in_flight) cudaEventSynchronize(s.copied);
     if (s.copied) cudaEventDestroy(s.copied);
+    if (s.released) cudaEventDestroy(s.released);
     if (s.pinned) cudaFreeHost(s.pinned);
+  }
+  if (ctx->copy_stream) {
+    cudaStreamSynchronize(ctx->copy_stream);
+    cudaStreamDestroy(ctx->copy_stream);
   }
   for (auto e : ctx->ev_start) cudaEventDestroy(e);
   for (auto e : ctx->ev_stop) cudaEventDestroy(e);
@@ -394,20 +474,27 @@ vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_ne
   if (total == 0) return VOSTI_OK;
   if (!k_new || !v_new) return VOSTI_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) % 16) return VOSTI_ERR_INVALID_ARG;
+  // Few tokens (decode): the slot list rides in the kernel parameters, no upload.
+  const bool inline_slots = total <= AppendParams::kInlineSlots;
+  AppendParams p;
   HostSlot* slot = nullptr;
-  vosti_status st = claim_slot(ctx, &slot);
-  if (st != VOSTI_OK) return st;
-  int32_t* dst = reinterpret_cast<int32_t*>(slot->pinned);
+  vosti_status st = VOSTI_OK;
+  int32_t* dst = p.inline_slot;
+  if (!inline_slots) {
+    st = claim_slot(ctx, &slot);
+    if (st != VOSTI_OK) return st;
+    dst = reinterpret_cast<int32_t*>(slot->pinned);
+  }
   int64_t t = 0;
   for (int r = 0; r < batch; ++r) {
     const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
     for (int i = 0; i < q_lens[r]; ++i, ++t) {
-      const int64_t p = int64_t{start_pos[r]} + i;
-      const int64_t blk = p / c.page_size;
+      const int64_t pos = int64_t{start_pos[r]} + i;
+      const int64_t blk = pos / c.page_size;
       if (blk >= block_table_stride) return VOSTI_ERR_OUT_OF_RANGE;
       const int64_t page = row[blk];
       if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
-      dst[t] = static_cast<int32_t>(page * c.page_size + p % c.page_size);
+      dst[t] = static_cast<int32_t>(page * c.page_size + pos % c.page_size);
     }
   }
   if (c.flags & VOSTI_FLAG_CHECK_WRITE_SLOTS) {
@@ -416,13 +503,14 @@ vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_ne
     if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return VOSTI_ERR_OUT_OF_RANGE;
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  st = push_blob(ctx, slot, sizeof(int32_t) * total, stream);
-  if (st != VOSTI_OK) return st;
-  AppendParams p;
+  if (!inline_slots) {
+    st = push_blob(ctx, slot, sizeof(int32_t) * total, stream);
+    if (st != VOSTI_OK) return st;
+  }
   p.k_new = static_cast<const __nv_bfloat16*>(k_new);
   p.v_new = static_cast<const __nv_bfloat16*>(v_new);
   p.pool = static_cast<__nv_bfloat16*>(c.kv_pool);
-  p.slot = reinterpret_cast<const int32_t*>(ctx->ws + ctx->lim.off_meta);
+  p.slot = inline_slots ? nullptr : reinterpret_cast<const int32_t*>(slot->device);
   p.n_tokens = static_cast<int32_t>(total);
   p.Hkv = c.n_kv_heads;
   const int64_t warps = total * c.n_kv_heads;
@@ -432,7 +520,8 @@ vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_ne
   else
     kv_append_kernel<64><<<grid, 128, 0, stream>>>(p);
   ++ctx->launches;
-  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return VOSTI_ERR_CUDA;
+  return inline_slots ? VOSTI_OK : release_slot(slot, stream);
 }
 
 vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, const int32_t* q_lens,
@@ -443,9 +532,10 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
   if (batch > 0 && !block_tables) return VOSTI_ERR_INVALID_ARG;
   const vosti_config& c = ctx->cfg;
-  Plan plan;
-  std::vector<int64_t> part_base;
-  vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, &plan, &part_base);
+  Plan& plan = ctx->plan;
+  std::vector<int64_t>& part_base = ctx->part_base;
+  part_base.resize(static_cast<size_t>(std::max(batch, 0)));
+  vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, &plan, part_base.data());
   if (st != VOSTI_OK) return st;
   if (plan.items.empty()) return VOSTI_OK;
   if (!q || !out) return VOSTI_ERR_INVALID_ARG;
@@ -457,16 +547,20 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   HostSlot* slot = nullptr;
   st = claim_slot(ctx, &slot);
   if (st != VOSTI_OK) return st;
-  // Blob: [ReqMeta x batch][items][flat page ids][split tokens]
+  // Blob: [ReqMeta x batch][SplitItem x n_split][sequential items][flat page ids][split tokens]
   const int G = c.n_q_heads / c.n_kv_heads;
+  const int64_t n_seq = static_cast<int64_t>(plan.items.size()) - plan.n_split;
   uint8_t* blob = slot->pinned;
   size_t at = 0;
   ReqMeta* reqs = reinterpret_cast<ReqMeta*>(blob + at);
   const size_t off_reqs = at;
   at += align_up(sizeof(ReqMeta) * batch, 16);
+  const size_t off_split = at;
+  SplitItem* split_items = reinterpret_cast<SplitItem*>(blob + at);
+  at += align_up(sizeof(SplitItem) * plan.n_split, 16);
   const size_t off_items = at;
-  std::memcpy(blob + at, plan.items.data(), sizeof(vosti_work_item) * plan.items.size());
-  at += align_up(sizeof(vosti_work_item) * plan.items.size(), 16);
+  std::memcpy(blob + at, plan.items.data() + plan.n_split, sizeof(vosti_work_item) * n_seq);
+  at += align_up(sizeof(vosti_work_item) * n_seq, 16);
   const size_t off_bt = at;
   int32_t* bt_flat = reinterpret_cast<int32_t*>(blob + at);
   int64_t bt_used = 0, row0 = 0, n_split_tokens = 0;
@@ -498,6 +592,22 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
     if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
   }
   at += align_up(sizeof(int32_t) * bt_used, 16);
+  for (int64_t i = 0; i < plan.n_split; ++i) {
+    const vosti_work_item& it = plan.items[i];
+    const ReqMeta& m = reqs[it.req];
+    SplitItem& si = split_items[i];
+    si.q_row0 = m.q_row0;
+    si.q_len = m.q_len;
+    si.start = m.start;
+    si.n_pages = m.n_pages;
+    si.bt_index = m.bt_off + it.split_begin * nc::kPagesPerSplit;
+    si.split = it.split_begin;
+    si.row_group = it.row_group;
+    si.n_splits = m.n_splits;
+    si.part_base = m.part_base;
+    si.req = it.req;
+    si.pad = 0;
+  }
   const size_t off_tok = at;
   int2* toks = reinterpret_cast<int2*>(blob + at);
   {
@@ -512,12 +622,15 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   st = push_blob(ctx, slot, at, stream);
   if (st != VOSTI_OK) return st;
 
-  uint8_t* dmeta = ctx->ws + ctx->lim.off_meta;
+  uint8_t* dmeta = slot->device;
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.reqs = reinterpret_cast<const ReqMeta*>(dmeta + off_reqs);
   p.items = reinterpret_cast<const vosti_work_item*>(dmeta + off_items);
+  p.split_items = reinterpret_cast<const SplitItem*>(dmeta + off_split);
+  p.ticket = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 64);
+  p.done = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 128);
   p.bt_flat = reinterpret_cast<const int32_t*>(dmeta + off_bt);
   p.split_tokens = reinterpret_cast<const int2*>(dmeta + off_tok);
   p.ws_u = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_part_u);
@@ -529,9 +642,10 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   p.Hkv = c.n_kv_heads;
   p.G = G;
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
-  const int64_t n_seq = static_cast<int64_t>(plan.items.size()) - plan.n_split;
-  return c.head_dim == 128 ? launch_attention<128>(ctx, p, plan.n_split, n_seq, stream)
-                           : launch_attention<64>(ctx, p, plan.n_split, n_seq, stream);
+  st = c.head_dim == 128 ? launch_attention<128>(ctx, p, plan.n_split, n_seq, stream)
+                         : launch_attention<64>(ctx, p, plan.n_split, n_seq, stream);
+  if (st != VOSTI_OK) return st;
+  return release_slot(slot, stream);
 }
 
 vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
@@ -579,7 +693,7 @@ vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
   uint32_t word = 0;
   uint8_t* d = ctx->ws + ctx->lim.off_status;
   if (cudaMemcpyAsync(&word, d, sizeof word, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaMemsetAsync(d, 0, sizeof word, stream) != cudaSuccess ||
+      cudaMemsetAsync(d, 0, kAlign, stream) != cudaSuccess ||
       cudaStreamSynchronize(stream) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   return (word & kStatusTimeout) ? VOSTI_ERR_TIMEOUT : VOSTI_OK;
