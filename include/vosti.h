@@ -166,6 +166,41 @@ vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host,
                              const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
                              float softmax_scale, void* cuda_stream);
 
+/* Split-parallel paged attention for callers that must not allocate.  (The
+ * paper has no counterpart: this is a packaging variant of the operation
+ * above, not a different computation.)
+ *
+ * Some callers cannot call cudaMalloc or create a vosti_ctx (which pins host
+ * memory and creates events): code that runs while a stream is being captured,
+ * serving loops whose memory is budgeted up front and owned by an outside
+ * allocator, plug-ins that receive device pointers but may not create their
+ * own.  This entry point allocates nothing on host or device and needs no
+ * context.  Its scratch (scheduler words, the call's metadata, the partial
+ * (m, z, U) rows) is a 16 MiB file-scope device array that every GPU loading
+ * the library holds until the process exits.  It launches the same kernels
+ * as vosti_paged_attention, so the output bits are the same.
+ *
+ *   kv_pool, q, out   device, as for vosti_paged_attention (pool 1024-byte aligned)
+ *   q_lens, start_pos, seq_lens, block_tables   host, same meaning as above
+ * Limits (beyond them the call returns VOSTI_ERR_WORKSPACE and launches
+ * nothing): batch <= 64, sum of q_lens <= 256, at most 16384 page-table
+ * entries in use, at most 1024 (row group, split) items, at most 28000
+ * partial rows (n_kv_heads * splits * q_len * G summed over requests).  Every
+ * request must satisfy q_len * G <= 32 (decode / speculative queries);
+ * longer queries return VOSTI_ERR_UNSUPPORTED_CONFIG.
+ * The first call on a device resolves the scratch array's device address and
+ * sets kernel attributes; make that first call before any stream capture.
+ * All calls share the one array: it is cleared where it must start at zero,
+ * and two calls that overlap on the GPU (different streams, or the same
+ * library used from two threads without ordering) race on it.  Host metadata
+ * is staged synchronously; the kernels run asynchronously on the stream. */
+vosti_status vosti_paged_attention_noalloc(int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
+                                           int32_t page_size, const void* kv_pool, int64_t num_pages,
+                                           const void* q, void* out, const int32_t* q_lens,
+                                           const int32_t* start_pos, const int32_t* seq_lens,
+                                           const int32_t* block_tables, int32_t block_table_stride,
+                                           int32_t batch, float softmax_scale, void* cuda_stream);
+
 /* Waits for the stream and reads the device status word: VOSTI_OK, or
  * VOSTI_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is
  * then undefined).  The word is cleared by the read. */

@@ -28,7 +28,7 @@ VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
 
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_create", "vosti_destroy", "vosti_kv_append",
-    "vosti_paged_attention", "vosti_step_host", "vosti_poll_device_status",
+    "vosti_paged_attention", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
     "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
 )
@@ -71,6 +71,10 @@ _lib.vosti_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, ctypes.c_in
 _lib.vosti_paged_attention.restype = ctypes.c_int
 _lib.vosti_paged_attention.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32,
                                        ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_paged_attention_noalloc.restype = ctypes.c_int
+_lib.vosti_paged_attention_noalloc.argtypes = [
+    ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp, ctypes.c_int64, _vp, _vp,
+    _i32p, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
 _lib.vosti_step_host.restype = ctypes.c_int
 _lib.vosti_step_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p,
                                  ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
@@ -229,6 +233,22 @@ def vosti_paged_attention(ctx: Context, q, out, q_lens, start_pos, seq_lens, blo
     _check(_lib.vosti_paged_attention(ctx.handle, _dev(q), _dev(out), _ip(ql), _ip(s), _ip(n),
                                       _ip(bt), bt.shape[1], len(ql), float(softmax_scale),
                                       _stream(stream)), "vosti_paged_attention")
+
+
+def vosti_paged_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_size, kv_pool, q, out,
+                                  q_lens, start_pos, seq_lens, block_tables,
+                                  softmax_scale: float, stream=None) -> None:
+    """Context-free variant that allocates nothing (see include/vosti.h for its
+    limits).  kv_pool is the torch tensor holding the whole pool."""
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    assert bt.ndim == 2 and bt.shape[0] == len(ql)
+    page_bytes = n_kv_heads * 2 * page_size * head_dim * 2
+    num_pages = kv_pool.numel() * kv_pool.element_size() // page_bytes
+    _check(_lib.vosti_paged_attention_noalloc(
+        n_q_heads, n_kv_heads, head_dim, page_size, _dev(kv_pool), num_pages, _dev(q), _dev(out),
+        _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1], len(ql), float(softmax_scale),
+        _stream(stream)), "vosti_paged_attention_noalloc")
 
 
 def vosti_step_host(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_lens, start_pos,
