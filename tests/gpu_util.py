@@ -71,3 +71,42 @@ def assert_same_bits(a: torch.Tensor, b: torch.Tensor, what=""):
         bad = (a != b).reshape(a.shape[0], -1).any(dim=1).nonzero().flatten()
         raise AssertionError(f"{what}: {bad.numel()} of {a.shape[0]} rows differ bitwise, "
                              f"first at positions {bad[:8].tolist()}")
+
+
+def compact_host_pool(w):
+    """The oracle's view of a workload: a host pool holding only the used pages
+    (page ids renumbered in order of first use; shared pages stay shared) filled
+    from the requests' logical content, and the renumbered block tables."""
+    from oracle import oracle
+    geo = w.geo
+    seen, tables = {}, []
+    for tb in w.tables:
+        tables.append([seen.setdefault(p, len(seen)) for p in tb])
+    pool = np.zeros((len(seen), geo.n_kv_heads, 2, geo.page_size, geo.head_dim), dtype=np.uint16)
+    for r, tb in zip(w.requests, tables):
+        oracle.kv_append(pool, inputs.bits(r.k), inputs.bits(r.v), [r.n], [0],
+                         inputs.block_table_array([tb]))
+    return pool, inputs.block_table_array(tables)
+
+
+def sampled_parity(w, out_bits, n_samples, seed=0):
+    """Compare `n_samples` random (request, token, head) outputs of a workload's
+    call against the oracle's paged front-end.  out_bits: int16 [T, Hq, d]."""
+    from oracle import oracle
+    geo = w.geo
+    rng = np.random.default_rng(seed)
+    pool, bt = compact_host_pool(w)
+    sel = []
+    for _ in range(n_samples):
+        r = int(rng.integers(0, w.batch))
+        sel.append((r, int(rng.integers(0, w.q_lens[r])), int(rng.integers(0, geo.n_q_heads))))
+    sel = np.array(sel, dtype=np.int32)
+    ref = oracle.paged_attention(inputs.bits(w.packed_q()), pool, w.q_lens, w.start_pos, w.seq_lens,
+                                 bt, n_kv_heads=geo.n_kv_heads, page_size=geo.page_size,
+                                 scale=geo.head_dim ** -0.5, sel=sel)
+    row0 = np.concatenate([[0], np.cumsum(w.q_lens)])
+    got = np.stack([widen_bits(out_bits[row0[r] + i, h]) for r, i, h in sel])
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all()
+    assert err.max() <= 1e-2 and err.mean() <= 1e-3, (err.max(), err.mean())
+    return float(err.max()), float(err.mean())
