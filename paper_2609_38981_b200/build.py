@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvosti.so")
 SOURCES = ["vosti.cu", "vosti_noalloc.cu"]
-HEADERS = ["attn_split.cuh", "attn_seq.cuh", "aux_kernels.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", os.path.join("..", "..", "include", "vosti.h")]
+HEADERS = ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", os.path.join("..", "..", "include", "vosti.h")]
 
 
 def _stale() -> bool:

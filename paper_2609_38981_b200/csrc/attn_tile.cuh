@@ -1,0 +1,440 @@
+// Tile attention for long queries (prefill chunks): one CTA per (128-row tile,
+// KV head), QK^T and PV on the 5th-generation tensor cores (tcgen05.mma, M = 128)
+// with the accumulators in tensor memory, K/V tiles gathered from the page pool
+// by TMA.
+//
+// It executes the same numerical contract as the split-parallel kernel: key
+// tiles of 64 in ascending order; S from head-dim chunks of 16 ascending with a
+// fresh accumulator; the scalar softmax rules of nc_math.cuh applied by one
+// thread per row (all 64 lanes of the row in its registers, so the pinned
+// row-sum order is a matter of adding in that order); U rescaled by alpha and
+// then accumulated over key chunks of 16 ascending; at every 512-key split
+// boundary the finished split is folded into the running result with
+// fold_scalars / fold_u.  tcgen05.mma and mma.sync.m16n8k16 give bit-identical
+// sums for the same chunk order (measured on B200), which is what lets this
+// kernel and the warp-MMA kernels agree bit for bit.
+//
+// Roles (192 threads): warps 0-3 = softmax / correction, one thread per row;
+// warp 4 = TMA producer; warp 5 = MMA issuer (one elected thread).
+// Tensor memory (512 columns): S x2 (64 each), P x2 (32 each, bf16 pairs),
+// U (D), running fold U_c (D).
+#pragma once
+#include "meta.cuh"
+#include "tile_math.cuh"
+
+namespace vosti {
+
+template <int D>
+struct TileKernelCfg {
+  static constexpr int kRows = 128;
+  static constexpr int kThreads = 192;
+  static constexpr int kStages = 3;                          // K+V tile pairs in flight
+  static constexpr int kQBytes = kRows * D * 2;              // [half][row][128 B]
+  static constexpr int kKBytes = nc::kKeyTile * D * 2;       // [half][key][128 B]
+  static constexpr int kStageBytes = 2 * kKBytes;            // K then V
+  static constexpr int kBarBytes = 256;
+  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;
+  // tensor-memory columns
+  static constexpr uint32_t kColS = 0, kColP = 128, kColU = 192, kColUc = 192 + D;
+};
+
+// ---- tcgen05 wrappers ---------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// 32 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,"
+      "%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31,%32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((saddr >> 4) & 0x3FFF);
+  d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFF) << 16;
+  d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFF) << 32;
+  d |= static_cast<uint64_t>(1) << 46;  // descriptor version
+  d |= static_cast<uint64_t>(2) << 61;  // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, A K-major, B K-major or MN-major.
+__host__ __device__ constexpr uint32_t umma_idesc(int m, int n, bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn_major ? (1u << 16) : 0u) |
+         (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+template <int D>
+__global__ void __launch_bounds__(TileKernelCfg<D>::kThreads, 1)
+attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {
+  using Cfg = TileKernelCfg<D>;
+  constexpr int NS = Cfg::kStages;
+  constexpr int TPS = nc::kTilesPerSplit;
+  constexpr int KT = nc::kKeyTile;
+  constexpr uint32_t kAbortAfterNs = 1000000000u;
+
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_smem = base;
+  const uint32_t kv_smem = base + Cfg::kQBytes;
+  const uint32_t bars = kv_smem + NS * Cfg::kStageBytes;
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 192);
+  // barrier map (8 bytes each)
+  const uint32_t k_full = bars, v_full = bars + 8 * NS, k_empty = bars + 16 * NS, v_empty = bars + 24 * NS;
+  const uint32_t s_full = bars + 32 * NS, s_empty = s_full + 16, p_full = s_full + 32, pv_done = s_full + 48;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  const vosti_work_item item = P.items[blockIdx.x / P.Hkv];
+  const int kvh = blockIdx.x % P.Hkv;
+  const ReqMeta rq = P.reqs[item.req];
+  const int G = P.G;
+  const int row0 = item.row_group * nc::kRowsPerGroup;  // first row of the 128-row tile
+  const int rows = rq.q_len * G;
+  const int last_tok = min(rq.q_len - 1, (row0 + Cfg::kRows - 1) / G);
+  const int p_max = rq.start + last_tok;
+  const int n_eff = rq.start + rq.q_len;
+  const int n_tiles = p_max / KT + 1;
+
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(k_full + 8 * i, 1);
+      mbar_init(v_full + 8 * i, 1);
+      mbar_init(k_empty + 8 * i, 1);
+      mbar_init(v_empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(s_full + 8 * i, 1);
+      mbar_init(s_empty + 8 * i, 128);
+      mbar_init(p_full + 8 * i, 128);
+      mbar_init(pv_done + 8 * i, 1);
+    }
+    flags[0] = 0u;  // abort flag
+    mbar_fence_init();
+    tma_prefetch_desc(&kv_map);
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 200), "r"(512));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  // Q tile -> shared memory, [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
+  if (warp < 4) {
+    griddep_wait();
+    const int row = row0 + tid;
+    const bool valid = row < rows;
+    const int tok = row / G;
+    const uint4* src = reinterpret_cast<const uint4*>(
+        P.q + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D);
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+      const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
+      const uint32_t addr = q_smem + (c >> 3) * (Cfg::kRows * 128) + tid * 128 + (((c & 7) ^ (tid & 7)) << 4);
+      asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                   : "memory");
+    }
+    fence_proxy_async();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 200);
+
+  // Bounded wait shared by all roles: gives up after ~1 s or as soon as another
+  // thread of the CTA has given up, records the failure, and lets the caller
+  // fall through to the common exit (tensor memory is still released).
+  auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 0;; ++it) {
+      if (mbar_try_wait(bar, parity)) return true;
+      if ((it & 63u) == 63u) {
+        if (flags[0] != 0u) return false;
+        if (global_timer_ns() - t0 > kAbortAfterNs) {
+          flags[0] = 1u;
+          atomicOr(P.status, kStatusTimeout);
+          return false;
+        }
+      }
+    }
+  };
+
+  if (warp == 4) {
+    // ================= TMA producer =================================================
+    griddep_wait();
+    const int32_t* bt = P.bt_flat + rq.bt_off;
+    auto fetch_pages = [&](int split) -> int {
+      const int pg = split * nc::kPagesPerSplit + lane;
+      return pg < rq.n_pages ? __ldg(bt + pg) : -1;
+    };
+    int pages_even = fetch_pages(0), pages_odd = -1;
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int s = t % NS, use = t / NS;
+      const int split = t / TPS, tl = t - split * TPS;
+      if (tl == TPS / 2 && (split + 1) * TPS < n_tiles) {
+        const int ids = fetch_pages(split + 1);
+        if ((split + 1) & 1) pages_odd = ids; else pages_even = ids;
+      }
+      const int ids = (split & 1) ? pages_odd : pages_even;
+      const int n_valid = min(nc::kPagesPerTile, rq.n_pages - t * nc::kPagesPerTile);
+      const uint32_t kdst = kv_smem + s * Cfg::kStageBytes;
+      if (use > 0) ok = __all_sync(kFullMask, wait(k_empty + 8 * s, (use - 1) & 1));
+      if (!ok) break;
+      issue_stage_load<D, KT>(&kv_map, kdst, k_full + 8 * s, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, 0, lane);
+      if (use > 0) ok = __all_sync(kFullMask, wait(v_empty + 8 * s, (use - 1) & 1));
+      if (!ok) break;
+      issue_stage_load<D, KT>(&kv_map, kdst + Cfg::kKBytes, v_full + 8 * s, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv,
+                              kvh, 1, lane);
+    }
+  } else if (warp == 5) {
+    // ================= MMA issuer ====================================================
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = umma_idesc(128, KT, false);
+      constexpr uint32_t idesc_pv = umma_idesc(128, D, true);
+      bool ok = true;
+      auto issue_s = [&](int t) {
+        const int s = t % NS, b = t & 1;
+        ok = ok && wait(k_full + 8 * s, (t / NS) & 1);
+        if (ok && t >= 2) ok = wait(s_empty + 8 * b, ((t >> 1) - 1) & 1);
+        if (!ok) return;
+        tc_fence_after();
+        const uint32_t kst = kv_smem + s * Cfg::kStageBytes;
+#pragma unroll
+        for (int kc = 0; kc < D / 16; ++kc) {
+          const uint64_t da = smem_desc_sw128(q_smem + (kc >> 2) * (Cfg::kRows * 128) + (kc & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
+          tc_mma_ss(tmem + Cfg::kColS + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
+        }
+        tc_commit(s_full + 8 * b);
+        tc_commit(k_empty + 8 * s);
+      };
+      issue_s(0);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        if (t + 1 < n_tiles) issue_s(t + 1);
+        if (!ok) break;
+        const int s = t % NS, b = t & 1;
+        ok = wait(p_full + 8 * b, (t >> 1) & 1);
+        if (ok) ok = wait(v_full + 8 * s, (t / NS) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+#pragma unroll
+        for (int kc = 0; kc < KT / 16; ++kc) {
+          // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
+          const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
+          const uint32_t acc = (kc > 0 || (t % TPS) != 0) ? 1u : 0u;  // a split starts from a fresh accumulator
+          tc_mma_ts(tmem + Cfg::kColU, tmem + Cfg::kColP + b * 32 + kc * 8, db, idesc_pv, acc);
+        }
+        tc_commit(pv_done + 8 * b);
+        tc_commit(v_empty + 8 * s);
+      }
+    }
+  } else {
+    // ================= softmax / correction: one thread per row ======================
+    const int row = row0 + tid;
+    const bool valid = row < rows;
+    const int tok = row / G;
+    const int p = valid ? rq.start + tok : -1;  // padding rows see nothing
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    const float c = P.c;
+    float m = -INFINITY, z = 0.f, mc = 0.f, zc = 0.f;
+    bool ok = true;
+    for (int t = 0; t < n_tiles && ok; ++t) {
+      const int b = t & 1, s = t % NS;
+      const int key0 = t * KT;
+      ok = __all_sync(kFullMask, wait(s_full + 8 * b, (t >> 1) & 1));
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t sr[64];
+      {
+        uint32_t lo[32], hi[32];
+        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT, lo);
+        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT + 32, hi);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) { sr[i] = lo[i]; sr[32 + i] = hi[i]; }
+      }
+      tc_fence_before();
+      mbar_arrive(s_empty + 8 * b);
+
+      // ---- the scalar rules, lanes b = 0..63 of this row --------------------------
+      const bool h = key0 <= p;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < KT; ++i) mx = fmaxf(mx, key0 + i <= p ? __uint_as_float(sr[i]) : -INFINITY);
+      const float mn = h ? nc::new_max(m, mx, c) : m;
+      const float alpha = h ? nc::rescale(m, mn) : 1.0f;
+      const float ng = -mn;
+      float w[KT];
+#pragma unroll
+      for (int i = 0; i < KT; ++i) w[i] = key0 + i <= p ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
+      {
+        // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3)
+        float part[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float a16[16];
+#pragma unroll
+          for (int n = 0; n < 8; ++n) { a16[2 * n] = w[8 * n + 2 * q]; a16[2 * n + 1] = w[8 * n + 2 * q + 1]; }
+          part[q] = nc::quad_partial(a16);
+        }
+        const float total = nc::quad_total(part[0], part[1], part[2], part[3]);
+        z = h ? nc::z_update(z, alpha, total) : z;
+        m = mn;
+      }
+      uint32_t pk[32];
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(w[2 * i], w[2 * i + 1]);
+        pk[i] = *reinterpret_cast<uint32_t*>(&t2);
+      }
+
+      // ---- U must be at rest before it is rescaled: PV of the previous tile done -----
+      if (t > 0) {
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * ((t - 1) & 1), ((t - 1) >> 1) & 1));
+        if (!ok) break;
+        tc_fence_after();
+      }
+      if ((t % TPS) != 0 && !__all_sync(kFullMask, alpha == 1.0f)) {
+#pragma unroll 1
+        for (int cb = 0; cb < D; cb += 32) {
+          uint32_t ur[32];
+          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) ur[i] = __float_as_uint(nc::u_rescale(__uint_as_float(ur[i]), alpha));
+          tmem_st32(tmem + lane_sel + Cfg::kColU + cb, ur);
+        }
+      }
+      tmem_st32(tmem + lane_sel + Cfg::kColP + b * 32, pk);
+      tmem_wait_st();
+      if (key0 + KT > n_eff) {
+        // Tail tile: zero the value rows at or beyond n_eff (not loaded, or pool garbage).
+        ok = __all_sync(kFullMask, wait(v_full + 8 * s, (t / NS) & 1));
+        if (!ok) break;
+        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+        const int first = n_eff - key0;
+        const int per_half = (KT - first) * 8;
+        for (int x = tid; x < per_half * (D / 64); x += 128) {
+          const int half = x / per_half, y = x - half * per_half;
+          const uint32_t addr = vst + half * (KT * 128) + (first + (y >> 3)) * 128 + ((y & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+        fence_proxy_async();
+      }
+      tc_fence_before();
+      mbar_arrive(p_full + 8 * b);
+
+      // ---- end of a split: fold it into the running result ---------------------------
+      if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * b, (t >> 1) & 1));
+        if (!ok) break;
+        tc_fence_after();
+        const int split = t / TPS;
+        const bool sees = p >= split * nc::kSplitLen;
+        nc::FoldFactors f;
+        f.a = 1.f;
+        f.b = 0.f;
+        if (split == 0) {
+          mc = m;
+          zc = z;
+        } else if (sees) {
+          f = nc::fold_scalars(mc, zc, m, z);
+        }
+#pragma unroll 1
+        for (int cb = 0; cb < D; cb += 32) {
+          uint32_t ur[32];
+          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
+          if (split == 0) {
+            tmem_wait_ld();
+            tmem_st32(tmem + lane_sel + Cfg::kColUc + cb, ur);
+          } else {
+            uint32_t uc[32];
+            tmem_ld32(tmem + lane_sel + Cfg::kColUc + cb, uc);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              uc[i] = sees ? __float_as_uint(nc::fold_u(__uint_as_float(uc[i]), __uint_as_float(ur[i]), f)) : uc[i];
+            tmem_st32(tmem + lane_sel + Cfg::kColUc + cb, uc);
+          }
+        }
+        tmem_wait_st();
+        m = -INFINITY;
+        z = 0.f;
+      }
+    }
+    // ---- normalise and store --------------------------------------------------------------
+    if (ok) {
+      const float inv = nc::out_scale(zc);
+      __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
+#pragma unroll 1
+      for (int cb = 0; cb < D; cb += 32) {
+        uint32_t uc[32];
+        tmem_ld32(tmem + lane_sel + Cfg::kColUc + cb, uc);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint32_t o[4];
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              __nv_bfloat162 t2 =
+                  __floats2bfloat162_rn(nc::out_value(__uint_as_float(uc[i + 2 * x]), inv),
+                                        nc::out_value(__uint_as_float(uc[i + 2 * x + 1]), inv));
+              o[x] = *reinterpret_cast<uint32_t*>(&t2);
+            }
+            *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+      }
+    }
+  }
+
+  // Common exit: every role ends here, also after a timeout, so tensor memory is always released.
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
+}
+
+}  // namespace vosti

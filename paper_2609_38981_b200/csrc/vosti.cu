@@ -8,7 +8,8 @@
 #include <utility>
 #include <vector>
 
-#include "attn_seq.cuh"
+#include "attn_split.cuh"
+#include "attn_tile.cuh"
 #include "aux_kernels.cuh"
 
 namespace vosti {
@@ -16,6 +17,7 @@ namespace {
 
 constexpr int kHostSlots = 8;        // ring of pinned staging buffers
 constexpr size_t kAlign = 1024;
+constexpr int kTileRows = 128;       // rows of one tile-kernel work item (8 row groups)
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -51,7 +53,7 @@ Limits limits_of(const vosti_config& c) {
   L.pages_max = int64_t{c.max_batch} * ((c.max_seq_len + nc::kPageSize - 1) / nc::kPageSize);
   const int64_t groups_split = (nc::kSplitRowsMax + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
   const int64_t items_split = int64_t{c.max_batch} * groups_split * L.k_max;
-  const int64_t items_seq = (c.max_total_q * G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup + c.max_batch;
+  const int64_t items_seq = (c.max_total_q * G + kTileRows - 1) / kTileRows + c.max_batch;
   L.items_max = items_split + items_seq;
   const int64_t rows_by_batch = int64_t{c.max_batch} * nc::kSplitRowsMax;
   const int64_t rows_by_total = c.max_total_q * G;
@@ -118,7 +120,7 @@ vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const i
       }
     } else {
       if (part_base) part_base[r] = 0;
-      n_seq += groups;
+      n_seq += (rows + kTileRows - 1) / kTileRows;
     }
   }
   if (total_q > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
@@ -138,17 +140,20 @@ vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const i
     const int64_t q = q_lens[r], st = start_pos[r];
     if (q == 0) continue;
     const int64_t rows = q * G;
-    const int groups = static_cast<int>((rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup);
     const bool split_parallel = rows <= nc::kSplitRowsMax;
-    for (int g = 0; g < groups; ++g) {
-      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{g} * nc::kRowsPerGroup + 15) / G);
+    // split-parallel requests: one item per (16-row group, split); others: one per 128-row tile
+    const int64_t rows_per_item = split_parallel ? nc::kRowsPerGroup : kTileRows;
+    const int n_row_items = static_cast<int>((rows + rows_per_item - 1) / rows_per_item);
+    for (int x = 0; x < n_row_items; ++x) {
+      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
       const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
       const int k_g = static_cast<int>((tiles + TPS - 1) / TPS);
       if (split_parallel) {
-        for (int k = 0; k + 1 < k_g; ++k) out[at[TPS]++] = {r, g, k, k + 1};
-        out[at[tiles - int64_t{k_g - 1} * TPS]++] = {r, g, k_g - 1, k_g};
+        for (int k = 0; k + 1 < k_g; ++k) out[at[TPS]++] = {r, x, k, k + 1};
+        out[at[tiles - int64_t{k_g - 1} * TPS]++] = {r, x, k_g - 1, k_g};
       } else {
-        plan->seq_scratch.push_back({tiles, vosti_work_item{r, g, 0, k_g}});
+        const int first_group = x * (kTileRows / nc::kRowsPerGroup);
+        plan->seq_scratch.push_back({tiles, vosti_work_item{r, first_group, 0, k_g}});
       }
     }
   }
@@ -316,10 +321,10 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
   if (n_seq > 0) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_seq * Hkv);
-    using SeqCfg = SeqKernelCfg<D>;
-    const int grid = (p.n_workers + SeqCfg::kWarps - 1) / SeqCfg::kWarps;
+    using TileCfg_ = TileKernelCfg<D>;
     timed(2, [&] {
-      attn_seq_kernel<D><<<grid, SeqCfg::kWarps * 32, SeqCfg::kSmemBytes, stream>>>(ctx->kv_map, p);
+      launch_dependent(attn_tile_kernel<D>, p.n_workers, TileCfg_::kThreads, TileCfg_::kSmemBytes, stream,
+                       ctx->kv_map, p);
     });
   }
   if (base.n_split_tokens > 0) {
@@ -335,8 +340,8 @@ vosti_status set_kernel_attributes() {
   if (cudaFuncSetAttribute(attn_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            Cfg::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
-  if (cudaFuncSetAttribute(attn_seq_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           SeqKernelCfg<D>::kSmemBytes) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           TileKernelCfg<D>::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   return VOSTI_OK;
 }
