@@ -187,7 +187,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (uint32_t it = 0;; ++it) {
-      if (mbar_try_wait(bar, parity)) return true;
+      if (mbar_try_wait_hint(bar, parity, 4000u)) return true;  // sleeps in hardware, no issue slots burnt
       if ((it & 63u) == 63u) {
         if (flags[0] != 0u) return false;
         if (global_timer_ns() - t0 > kAbortAfterNs) {
@@ -299,16 +299,34 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       mbar_arrive(s_empty + 8 * b);
 
       // ---- the scalar rules, lanes b = 0..63 of this row --------------------------
-      const bool h = key0 <= p;
-      float mx = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < KT; ++i) mx = fmaxf(mx, key0 + i <= p ? __uint_as_float(sr[i]) : -INFINITY);
-      const float mn = h ? nc::new_max(m, mx, c) : m;
-      const float alpha = h ? nc::rescale(m, mn) : 1.0f;
-      const float ng = -mn;
+      // Schedule-only shortcut: when every key of the tile is visible to every real
+      // row of the warp the selects all take the visible arm and are skipped.
+      const bool all_visible = __all_sync(kFullMask, !valid || key0 + KT - 1 <= p);
+      const bool h = all_visible || key0 <= p;
+      float mn, alpha;
       float w[KT];
+      if (all_visible) {
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // the maximum is order-free
 #pragma unroll
-      for (int i = 0; i < KT; ++i) w[i] = key0 + i <= p ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
+        for (int i = 0; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        mn = nc::new_max(m, mx, c);
+        alpha = nc::rescale(m, mn);
+        const float ng = -mn;
+#pragma unroll
+        for (int i = 0; i < KT; ++i) w[i] = nc::weight(__uint_as_float(sr[i]), c, ng);
+      } else {
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < KT; ++i)
+          mx4[i & 3] = fmaxf(mx4[i & 3], key0 + i <= p ? __uint_as_float(sr[i]) : -INFINITY);
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        mn = h ? nc::new_max(m, mx, c) : m;
+        alpha = h ? nc::rescale(m, mn) : 1.0f;
+        const float ng = -mn;
+#pragma unroll
+        for (int i = 0; i < KT; ++i) w[i] = key0 + i <= p ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
+      }
       {
         // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3)
         float part[4];
