@@ -47,17 +47,20 @@ def parse_args():
                              "mixed_chunked_prefill"])
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (experiments only)")
     ap.add_argument("--pool-pages", type=int, default=0,
                     help="override the pool size (small pools keep profiler captures short)")
     return ap.parse_args()
 
 
-def make_workload(name: str, rank: int, pool_pages: int = 0):
+def make_workload(name: str, rank: int, pool_pages: int = 0, batch: int = 0):
     from paper_2609_38981_b200 import inputs
     fn = getattr(inputs, name)
     base = {"decode_heavy": 2, "mixed_chunked_prefill": 3, "prefix_sharing": 4,
             "long_context_speculative": 5}[name]
     kw = {"num_pages": pool_pages} if pool_pages else {}
+    if batch:
+        kw["batch"] = batch
     return fn(seed=inputs.BASE_SEED * 10 + base + 1000 * rank, **kw)
 
 
@@ -211,7 +214,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = make_workload(args.workload, rank, args.pool_pages)
+    w = make_workload(args.workload, rank, args.pool_pages, args.batch)
     geo = w.geo
     scale = geo.head_dim ** -0.5
     max_seq = max(w.seq_lens)

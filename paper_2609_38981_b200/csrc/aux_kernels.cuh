@@ -11,11 +11,13 @@ namespace vosti {
 // normalises.  Order depends on the split index only.
 template <int D>
 __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
-  constexpr int V = D / 32;  // floats per lane
+  constexpr int V = D / 32;   // floats per lane
+  constexpr int BATCH = 8;    // partial rows whose loads are in flight together
   const int lane = threadIdx.x & 31;
   const int widx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (widx >= P.n_split_tokens * P.Hq) return;
-  griddep_wait();  // partials come from the kernel before this one in the stream
+  // Metadata does not depend on the kernel before this one: read it first, so that
+  // only the partial rows themselves wait for the attention kernel to finish.
   const int2 rt = P.split_tokens[widx / P.Hq];
   const int head = widx % P.Hq;
   const ReqMeta rq = P.reqs[rt.x];
@@ -25,38 +27,44 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
   const int p = rq.start + rt.y;
   const int n_splits = p / nc::kSplitLen + 1;
   const int64_t slab0 = rq.part_base + static_cast<int64_t>(kvh) * rq.n_splits * rows + row;
+  griddep_wait();  // partials come from the kernel before this one in the stream
 
-  float uc[V];
-  float mc, zc;
-  {
-    const float2 mz = P.ws_mz[slab0];
-    mc = mz.x;
-    zc = mz.y;
-    const float* src = P.ws_u + slab0 * D + lane * V;
-    if constexpr (V == 4) {
-      const float4 x = *reinterpret_cast<const float4*>(src);
-      uc[0] = x.x; uc[1] = x.y; uc[2] = x.z; uc[3] = x.w;
-    } else {
-      const float2 x = *reinterpret_cast<const float2*>(src);
-      uc[0] = x.x; uc[1] = x.y;
-    }
-  }
-#pragma unroll 4
-  for (int k = 1; k < n_splits; ++k) {
-    const int64_t slab = slab0 + static_cast<int64_t>(k) * rows;
-    const float2 mz = P.ws_mz[slab];
-    float uk[V];
+  auto load_u = [&](int64_t slab, float (&u)[V]) {
     const float* src = P.ws_u + slab * D + lane * V;
     if constexpr (V == 4) {
       const float4 x = *reinterpret_cast<const float4*>(src);
-      uk[0] = x.x; uk[1] = x.y; uk[2] = x.z; uk[3] = x.w;
+      u[0] = x.x; u[1] = x.y; u[2] = x.z; u[3] = x.w;
     } else {
       const float2 x = *reinterpret_cast<const float2*>(src);
-      uk[0] = x.x; uk[1] = x.y;
+      u[0] = x.x; u[1] = x.y;
     }
-    const nc::FoldFactors f = nc::fold_scalars(mc, zc, mz.x, mz.y);
+  };
+  float uc[V];
+  float mc = 0.f, zc = 0.f;
+  for (int k0 = 0; k0 < n_splits; k0 += BATCH) {
+    float uk[BATCH][V];
+    float2 mz[BATCH];
 #pragma unroll
-    for (int i = 0; i < V; ++i) uc[i] = nc::fold_u(uc[i], uk[i], f);
+    for (int j = 0; j < BATCH; ++j)
+      if (k0 + j < n_splits) {
+        const int64_t slab = slab0 + static_cast<int64_t>(k0 + j) * rows;
+        mz[j] = P.ws_mz[slab];
+        load_u(slab, uk[j]);
+      }
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)
+      if (k0 + j < n_splits) {
+        if (k0 + j == 0) {  // folding starts from the first partial as it is
+          mc = mz[0].x;
+          zc = mz[0].y;
+#pragma unroll
+          for (int i = 0; i < V; ++i) uc[i] = uk[0][i];
+        } else {
+          const nc::FoldFactors f = nc::fold_scalars(mc, zc, mz[j].x, mz[j].y);
+#pragma unroll
+          for (int i = 0; i < V; ++i) uc[i] = nc::fold_u(uc[i], uk[j][i], f);
+        }
+      }
   }
   const float inv = nc::out_scale(zc);
   __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + rt.y) * P.Hq + head) * D + lane * V;
@@ -75,6 +83,7 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams P) {
   if (widx >= P.n_tokens * P.Hkv) return;
   const int tok = widx / P.Hkv, kvh = widx % P.Hkv;
   const int slot = P.slot ? P.slot[tok] : P.inline_slot[tok];
+  griddep_wait();  // earlier kernels in the stream may still be reading the pool
   const int page = slot / nc::kPageSize, within = slot % nc::kPageSize;
   const int is_v = lane >> 4, part = lane & 15;
   const __nv_bfloat16* src = (is_v ? P.v_new : P.k_new) + (static_cast<size_t>(tok) * P.Hkv + kvh) * D;

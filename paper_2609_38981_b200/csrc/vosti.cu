@@ -257,6 +257,11 @@ vosti_status push_blob(vosti_ctx* ctx, HostSlot* s, size_t bytes, cudaStream_t s
     return VOSTI_ERR_CUDA;
   if (cudaEventRecord(s->copied, cs) != cudaSuccess) return VOSTI_ERR_CUDA;
   s->in_flight = true;
+  // The copy usually lands within microseconds.  If it is seen complete, the stream
+  // needs no wait node, which keeps the kernels of consecutive calls adjacent in
+  // the stream (a wait node between two kernels defeats dependent launch).
+  for (int spin = 0; spin < 400; ++spin)
+    if (cudaEventQuery(s->copied) == cudaSuccess) return VOSTI_OK;
   if (cudaStreamWaitEvent(stream, s->copied, 0) != cudaSuccess) return VOSTI_ERR_CUDA;
   return VOSTI_OK;
 }
@@ -521,9 +526,9 @@ vosti_status vosti_kv_append(vosti_ctx* ctx, const void* k_new, const void* v_ne
   const int64_t warps = total * c.n_kv_heads;
   const int grid = static_cast<int>((warps + 3) / 4);
   if (c.head_dim == 128)
-    kv_append_kernel<128><<<grid, 128, 0, stream>>>(p);
+    launch_dependent(kv_append_kernel<128>, grid, 128, 0, stream, p);
   else
-    kv_append_kernel<64><<<grid, 128, 0, stream>>>(p);
+    launch_dependent(kv_append_kernel<64>, grid, 128, 0, stream, p);
   ++ctx->launches;
   if (cudaGetLastError() != cudaSuccess) return VOSTI_ERR_CUDA;
   return inline_slots ? VOSTI_OK : release_slot(slot, stream);
