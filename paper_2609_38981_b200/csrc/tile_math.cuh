@@ -62,21 +62,27 @@ template <int D, int SK>
 __device__ __forceinline__ void tile_scores(uint32_t ks, const uint32_t (&qa)[D / 16][4],
                                             float (&s)[8][4], int n0, int lane) {
   using C = TileCfg<D, SK>;
+  constexpr int NN = SK / 8;
   const int lm_mat = lane >> 3, lm_row = lane & 7;
 #pragma unroll
-  for (int nn = 0; nn < SK / 8; ++nn) {
-    float(&acc)[4] = s[n0 + nn];
-    acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
-    const int key = nn * 8 + lm_row;
+  for (int nn = 0; nn < NN; ++nn) s[n0 + nn][0] = s[n0 + nn][1] = s[n0 + nn][2] = s[n0 + nn][3] = 0.f;
+  // Chunk pair outermost, column tile innermost: consecutive MMAs feed different
+  // accumulators, so their latencies overlap.  Each accumulator still receives
+  // its head-dim chunks in ascending order.
 #pragma unroll
-    for (int cp = 0; cp < C::KC / 2; ++cp) {
+  for (int cp = 0; cp < C::KC / 2; ++cp) {
+    uint32_t b[NN][4];
+#pragma unroll
+    for (int nn = 0; nn < NN; ++nn) {
+      const int key = nn * 8 + lm_row;
       const int x = 4 * cp + lm_mat;
       const uint32_t addr = ks + (x >> 3) * C::kHalfBytes + key * 128 + (((x & 7) ^ (key & 7)) << 4);
-      uint32_t b0, b1, b2, b3;
-      ldsm_x4(addr, b0, b1, b2, b3);
-      mma_bf16_16816(acc, qa[2 * cp], b0, b1);
-      mma_bf16_16816(acc, qa[2 * cp + 1], b2, b3);
+      ldsm_x4(addr, b[nn][0], b[nn][1], b[nn][2], b[nn][3]);
     }
+#pragma unroll
+    for (int nn = 0; nn < NN; ++nn) mma_bf16_16816(s[n0 + nn], qa[2 * cp], b[nn][0], b[nn][1]);
+#pragma unroll
+    for (int nn = 0; nn < NN; ++nn) mma_bf16_16816(s[n0 + nn], qa[2 * cp + 1], b[nn][2], b[nn][3]);
   }
 }
 
@@ -211,10 +217,12 @@ __device__ __forceinline__ void tile_pv(uint32_t vs, const uint32_t (&pa)[4][4],
                                         int kc0, int lane) {
   using C = TileCfg<D, SK>;
   const int lm_mat = lane >> 3, lm_row = lane & 7;
+  // Key chunk outermost, output column tile innermost: consecutive MMAs feed
+  // different accumulators; each accumulator gets its key chunks in ascending order.
 #pragma unroll
-  for (int e = 0; e < C::NE; e += 2) {
+  for (int kk = 0; kk < SK / 16; ++kk) {
 #pragma unroll
-    for (int kk = 0; kk < SK / 16; ++kk) {
+    for (int e = 0; e < C::NE; e += 2) {
       const int key = kk * 16 + (lm_mat & 1) * 8 + lm_row;
       const int x = e + (lm_mat >> 1);
       const uint32_t addr = vs + (x >> 3) * C::kHalfBytes + key * 128 + (((x & 7) ^ (key & 7)) << 4);
