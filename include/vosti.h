@@ -208,6 +208,14 @@ vosti_status vosti_paged_attention_noalloc(int32_t n_q_heads, int32_t n_kv_heads
  * then undefined).  The word is cleared by the read. */
 vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream);
 
+/* Failure-detection self-test (no GPU fault involved): launches one warp that
+ * waits, with the bounded wait every kernel of the library uses, on a barrier
+ * that nothing completes.  After limit_us microseconds (1..100000) the warp
+ * gives up, sets the device status word and returns normally; the next
+ * vosti_poll_device_status then reports VOSTI_ERR_TIMEOUT and clears it, and
+ * the context stays usable. */
+vosti_status vosti_selftest_bounded_wait(vosti_ctx* ctx, uint32_t limit_us, void* cuda_stream);
+
 /* Timing of one kernel of the path with CUDA events recorded on the caller's
  * stream around each of its launches.  mode: 0 stops recording; 1 times the
  * split-parallel attention kernel (the decode hot loop, a3-a7), 2 the

@@ -29,7 +29,7 @@ VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_create", "vosti_destroy", "vosti_kv_append",
     "vosti_paged_attention", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
-    "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
+    "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
 )
 
@@ -80,6 +80,8 @@ _lib.vosti_step_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _
                                  ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
 _lib.vosti_poll_device_status.restype = ctypes.c_int
 _lib.vosti_poll_device_status.argtypes = [_vp, _vp]
+_lib.vosti_selftest_bounded_wait.restype = ctypes.c_int
+_lib.vosti_selftest_bounded_wait.argtypes = [_vp, ctypes.c_uint32, _vp]
 _lib.vosti_profile_enable.restype = ctypes.c_int
 _lib.vosti_profile_enable.argtypes = [_vp, ctypes.c_int32]
 _lib.vosti_profile_read.restype = ctypes.c_int
@@ -262,6 +264,11 @@ def vosti_step_host(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_le
 
 def vosti_poll_device_status(ctx: Context, stream=None) -> int:
     return int(_lib.vosti_poll_device_status(ctx.handle, _stream(stream)))
+
+
+def vosti_selftest_bounded_wait(ctx: Context, limit_us: int, stream=None) -> None:
+    _check(_lib.vosti_selftest_bounded_wait(ctx.handle, int(limit_us), _stream(stream)),
+           "vosti_selftest_bounded_wait")
 
 
 def vosti_profile_enable(ctx: Context, mode: int) -> None:

@@ -97,4 +97,19 @@ __global__ void __launch_bounds__(128) kv_append_kernel(const AppendParams P) {
   }
 }
 
+// Failure-detection self-test: one warp waits on a barrier that nothing will ever
+// complete, with the same bounded wait the attention kernels use, gives up after
+// `limit_ns`, records the failure in the status word and returns normally.
+static __global__ void bounded_wait_selftest_kernel(uint32_t* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    mbar_fence_init();
+  }
+  __syncwarp();
+  const bool ok = __all_sync(0xffffffffu, mbar_wait_bounded(b, 0, limit_ns));
+  if (!ok && threadIdx.x == 0) atomicOr(status, 1u);
+}
+
 }  // namespace vosti

@@ -709,6 +709,15 @@ vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
   return (word & kStatusTimeout) ? VOSTI_ERR_TIMEOUT : VOSTI_OK;
 }
 
+vosti_status vosti_selftest_bounded_wait(vosti_ctx* ctx, uint32_t limit_us, void* cuda_stream) {
+  if (!ctx || limit_us == 0 || limit_us > 100000) return VOSTI_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status),
+                                                   static_cast<uint64_t>(limit_us) * 1000ull);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
 vosti_status vosti_profile_enable(vosti_ctx* ctx, int32_t mode) {
   if (!ctx || mode < 0 || mode > 3) return VOSTI_ERR_INVALID_ARG;
   ctx->profile_mode = mode;

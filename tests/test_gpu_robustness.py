@@ -1,0 +1,97 @@
+"""Failure detection without a GPU fault, randomized execution schedules, and
+contexts on every boundary of the tiling (page 16, key tile 64, split 512)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_38981_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def test_a_wait_that_runs_out_sets_the_status_and_leaves_the_context_usable():
+    from paper_2609_38981_b200 import binding as vb
+    from paper_2609_38981_b200.harness import DeviceCache, bf16_bits
+    import gpu_util as gu
+    geo = inputs.TINY
+    cache = DeviceCache(geo, 64, max_batch=4, max_total_q=256, max_seq_len=512)
+    assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_OK
+    vb.vosti_selftest_bounded_wait(cache.ctx, 500)                 # gives up after 0.5 ms
+    assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_ERR_TIMEOUT
+    assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_OK   # cleared by the read
+    # the context still computes correctly afterwards
+    r = inputs.make_request(geo, 3, 0, 90)
+    out = gu.run_schedule(cache, [r], [list(range(6))], [[(0, 0, 90)]], geo.head_dim ** -0.5)[0]
+    ref = gu.oracle_rows([r], geo.head_dim ** -0.5)[0]
+    gu.assert_parity(out, ref, "after a timed-out wait")
+    with pytest.raises(vb.VostiError):
+        vb.vosti_selftest_bounded_wait(cache.ctx, 0)
+    cache.close()
+
+
+@pytest.mark.parametrize("geo_name", ["d64_g2", "d128_g4"])
+def test_contexts_on_every_tiling_boundary(geo_name):
+    """Prefill in one call vs token-by-token decode of the last positions, for
+    contexts at k*16, k*64 and k*512 plus/minus one."""
+    import gpu_util as gu
+    from paper_2609_38981_b200.harness import DeviceCache
+    geo = {"d64_g2": inputs.TINY, "d128_g4": inputs.Geometry(8, 2, 128, 16)}[geo_name]
+    scale = geo.head_dim ** -0.5
+    contexts = [15, 16, 17, 63, 64, 65, 127, 128, 129, 191, 192, 193, 575, 576, 577]
+    reqs = [inputs.make_request(geo, 777, i, n) for i, n in enumerate(contexts)]
+    tables = inputs._assign_private_pages(inputs.generator(777), geo, 400, contexts)
+    cache = DeviceCache(geo, 400, max_batch=16, max_total_q=4096, max_seq_len=1024, pool_fill="nan")
+    full = gu.run_schedule(cache, reqs, tables, [[(i, 0, r.n) for i, r in enumerate(reqs)]], scale)
+    ref = gu.oracle_rows(reqs, scale)
+    for i in full:
+        gu.assert_parity(full[i], ref[i], f"context {contexts[i]}")
+    tail = 3
+    sched = [[(i, r.n - tail + s, 1) for i, r in enumerate(reqs)] for s in range(tail)]
+    dec = gu.run_schedule(cache, reqs, tables, sched, scale, append=False,
+                          seq_lens_override={i: r.n for i, r in enumerate(reqs)})
+    for i, r in enumerate(reqs):
+        gu.assert_same_bits(dec[i][r.n - tail:], full[i][r.n - tail:], f"context {r.n}")
+    cache.close()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_schedules_give_the_canonical_bits(seed):
+    """Random chunk sizes, random co-batching, random batch order, random page
+    placement, random table width: every row must equal the canonical run."""
+    import gpu_util as gu
+    from paper_2609_38981_b200.harness import DeviceCache
+    rng = np.random.default_rng(1000 + seed)
+    geo = [inputs.TINY, inputs.Geometry(8, 2, 128, 16), inputs.Geometry(8, 1, 128, 16)][seed % 3]
+    scale = geo.head_dim ** -0.5
+    n_req = 5
+    contexts = [int(x) for x in rng.integers(1, 1400, n_req)]
+    reqs = [inputs.make_request(geo, 2000 + seed, i, n) for i, n in enumerate(contexts)]
+    ident = inputs._assign_private_pages(inputs.generator(seed), geo, 600, contexts)
+
+    def cache(fill):
+        return DeviceCache(geo, 600, max_batch=8, max_total_q=4096, max_seq_len=2048, pool_fill=fill)
+
+    c = cache("zeros")
+    canon = {}
+    for i, r in enumerate(reqs):
+        canon[i] = gu.run_schedule(c, reqs, ident, [[(i, 0, r.n)]], scale)[i]
+    c.close()
+    # a random schedule on a randomly placed, garbage-filled pool
+    tables = inputs._assign_private_pages(inputs.generator(50 + seed), geo, 600, contexts)
+    done = [0] * n_req
+    sched = []
+    while any(d < n for d, n in zip(done, contexts)):
+        call = []
+        for i in rng.permutation(n_req):
+            if done[i] < contexts[i] and rng.random() < 0.7:
+                q = int(min(contexts[i] - done[i], rng.choice([1, 1, 2, 3, 5, 8, 9, 33, 64, 130, 300])))
+                call.append((int(i), done[i], q))
+                done[i] += q
+        if call:
+            sched.append(call)
+    c = cache("random")
+    outs = gu.run_schedule(c, reqs, tables, sched, scale, stride=int(rng.integers(90, 200)),
+                           fill=int(rng.integers(0, 600)))
+    for i in outs:
+        gu.assert_same_bits(outs[i], canon[i], f"seed {seed} request {i} (context {contexts[i]})")
+    c.close()
