@@ -144,14 +144,28 @@ vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const i
     // split-parallel requests: one item per (16-row group, split); others: one per 128-row tile
     const int64_t rows_per_item = split_parallel ? nc::kRowsPerGroup : kTileRows;
     const int n_row_items = static_cast<int>((rows + rows_per_item - 1) / rows_per_item);
-    for (int x = 0; x < n_row_items; ++x) {
-      const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
-      const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
-      const int k_g = static_cast<int>((tiles + TPS - 1) / TPS);
-      if (split_parallel) {
-        for (int k = 0; k + 1 < k_g; ++k) out[at[TPS]++] = {r, x, k, k + 1};
-        out[at[tiles - int64_t{k_g - 1} * TPS]++] = {r, x, k_g - 1, k_g};
-      } else {
+    if (split_parallel) {
+      // Split outermost, row group innermost: the (at most two) row groups that read the
+      // same split get neighbouring tickets, run at about the same time on different SMs,
+      // and the second read of the split's K/V is served by L2 instead of HBM.
+      int64_t tiles_g[nc::kSplitRowsMax / nc::kRowsPerGroup];
+      int k_max = 0;
+      for (int x = 0; x < n_row_items; ++x) {
+        const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
+        tiles_g[x] = (st + last_tok) / nc::kKeyTile + 1;
+        k_max = std::max(k_max, static_cast<int>((tiles_g[x] + TPS - 1) / TPS));
+      }
+      for (int k = 0; k < k_max; ++k)
+        for (int x = 0; x < n_row_items; ++x) {
+          const int k_g = static_cast<int>((tiles_g[x] + TPS - 1) / TPS);
+          if (k + 1 < k_g) out[at[TPS]++] = {r, x, k, k + 1};
+          else if (k + 1 == k_g) out[at[tiles_g[x] - int64_t{k_g - 1} * TPS]++] = {r, x, k, k + 1};
+        }
+    } else {
+      for (int x = 0; x < n_row_items; ++x) {
+        const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
+        const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
+        const int k_g = static_cast<int>((tiles + TPS - 1) / TPS);
         const int first_group = x * (kTileRows / nc::kRowsPerGroup);
         plan->seq_scratch.push_back({tiles, vosti_work_item{r, first_group, 0, k_g}});
       }
