@@ -207,6 +207,8 @@ __device__ __forceinline__ void zero_value_tail(uint32_t vs, int first_bad_row, 
     const uint32_t addr = vs + half * C::kHalfBytes + (first_bad_row + (y >> 3)) * 128 + ((y & 7) << 4);
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
   }
+  // These generic-proxy writes precede a later TMA (async-proxy) refill of the same stage.
+  fence_proxy_async();
   __syncwarp();
 }
 
@@ -236,25 +238,25 @@ __device__ __forceinline__ void tile_pv(uint32_t vs, const uint32_t (&pa)[4][4],
 
 // One TMA page gather: the K or V rows of `n_valid` pages (at most SK / 16) for
 // one KV head into a stage; `ids` holds one page id per lane, `first_lane` the
-// lane of the stage's first page.  Called by all lanes; lane 0 issues.
+// lane of the stage's first page.  Called by all lanes.  Lane 0 arms the
+// barrier; then every box of the stage is issued by its own lane in ONE warp
+// instruction (a thread needs on the order of a hundred cycles per TMA
+// instruction, so issuing the boxes one after another from a single lane makes
+// the issuing warp the bottleneck).
 template <int D, int SK>
 __device__ __forceinline__ void issue_stage_load(const CUtensorMap* map, uint32_t dst, uint32_t bar,
                                                  int ids, int first_lane, int n_valid, int Hkv, int kvh,
                                                  int is_v, int lane) {
   using C = TileCfg<D, SK>;
-  if (lane == 0) {
-    fence_proxy_async();
-    mbar_expect_tx(bar, n_valid * nc::kPageSize * D * 2);
-  }
-#pragma unroll
-  for (int j = 0; j < C::kPagesPerStage; ++j) {
-    const int page = __shfl_sync(kFullMask, ids, first_lane + j);
-    if (lane == 0 && j < n_valid) {
-      const int32_t y = ((page * Hkv + kvh) * 2 + is_v) * nc::kPageSize;
-#pragma unroll
-      for (int h = 0; h < D / 64; ++h)
-        tma_load_2d(dst + h * C::kHalfBytes + j * C::kPageBytes, map, h * 64, y, bar);
-    }
+  constexpr int HALVES = D / 64;
+  constexpr int BOXES = C::kPagesPerStage * HALVES;
+  if (lane == 0) mbar_expect_tx(bar, n_valid * nc::kPageSize * D * 2);
+  const int j = lane / HALVES, h = lane % HALVES;  // page of the stage, 64-element half
+  const int page = __shfl_sync(kFullMask, ids, first_lane + (lane < BOXES ? j : 0));
+  __syncwarp();
+  if (lane < BOXES && j < n_valid) {
+    const int32_t y = ((page * Hkv + kvh) * 2 + is_v) * nc::kPageSize;
+    tma_load_2d(dst + h * C::kHalfBytes + j * C::kPageBytes, map, h * 64, y, bar);
   }
 }
 
