@@ -83,8 +83,8 @@ typedef struct {
  * tiles and heads; the KV split is this library's addition).  Rows of a
  * request are numbered token*G + head_in_group; row group g holds rows
  * 16g..16g+15.  A split-parallel item is one row group and one KV split
- * (split_end = split_begin + 1); a sequential item is a tile of eight row
- * groups starting at row_group (128 rows) that walks splits 0..split_end-1 of
+ * (split_end = split_begin + 1); a sequential item is a tile of sixteen row
+ * groups starting at row_group (256 rows) that walks splits 0..split_end-1 of
  * 512 keys each in order.  Every item is run once per KV head. */
 typedef struct {
   int32_t req, row_group, split_begin, split_end;

@@ -1,7 +1,7 @@
-// Tile attention for long queries (prefill chunks): one CTA per (128-row tile,
-// KV head), QK^T and PV on the 5th-generation tensor cores (tcgen05.mma, M = 128)
-// with the accumulators in tensor memory, K/V tiles gathered from the page pool
-// by TMA.
+// Tile attention for long queries (prefill chunks): one CTA per (256-row super
+// tile, KV head), QK^T and PV on the 5th-generation tensor cores (tcgen05.mma,
+// M = 128) with the accumulators in tensor memory, K/V tiles gathered from the
+// page pool by TMA.
 //
 // It executes the same numerical contract as the split-parallel kernel: key
 // tiles of 64 in ascending order; S from head-dim chunks of 16 ascending with a
@@ -14,10 +14,18 @@
 // sums for the same chunk order (measured on B200), which is what lets this
 // kernel and the warp-MMA kernels agree bit for bit.
 //
-// Roles (192 threads): warps 0-3 = softmax / correction, one thread per row;
-// warp 4 = TMA producer; warp 5 = MMA issuer (one elected thread).
-// Tensor memory (512 columns): S x2 (64 each), P x2 (32 each, bf16 pairs),
-// U (D), running fold U_c (D).
+// A CTA holds TWO 128-row tiles (X = 0, 1) that share every staged K/V tile:
+// the softmax work of one overlaps the waits of the other on every scheduler,
+// and K/V is fetched through L2 once per 256 rows.
+// Roles (352 threads): warps 0-3 = softmax / correction of tile 0, warps 4-7 of
+// tile 1, one thread per row; warp 9 = MMA issuer (one elected thread); warps 8
+// and 10 = TMA producers for K and for V (a TMA instruction occupies its issuing
+// warp for about a hundred cycles per 2 KB box).
+// Tensor memory (512 columns): per tile S x2 (64 each; the bf16 weights P are
+// written over the first 32 columns of the S buffer they were computed from)
+// and U (D).  The running fold U_c lives in global memory (per CTA and tile a
+// [D/4][128 rows] array of float4, so that a warp's rows are contiguous; touched
+// once per split): there is no room for it on chip.
 #pragma once
 #include "meta.cuh"
 #include "tile_math.cuh"
@@ -26,16 +34,18 @@ namespace vosti {
 
 template <int D>
 struct TileKernelCfg {
-  static constexpr int kRows = 128;
-  static constexpr int kThreads = 192;
+  static constexpr int kRows = 256;                          // rows of a work item: two tiles
+  static constexpr int kTileRows = 128;
+  static constexpr int kThreads = 352;
   static constexpr int kStages = 3;                          // K+V tile pairs in flight
   static constexpr int kQBytes = kRows * D * 2;              // [half][row][128 B]
   static constexpr int kKBytes = nc::kKeyTile * D * 2;       // [half][key][128 B]
   static constexpr int kStageBytes = 2 * kKBytes;            // K then V
-  static constexpr int kBarBytes = 256;
+  static constexpr int kBarBytes = 512;
   static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;
   // tensor-memory columns
-  static constexpr uint32_t kColS = 0, kColP = 128, kColU = 192, kColUc = 192 + D;
+  static constexpr uint32_t kColS = 0;    // tile X, buffer b: S / P at 128 X + 64 b
+  static constexpr uint32_t kColU = 256;  // tile X: U at 256 + D X
 };
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------
@@ -111,18 +121,19 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   constexpr int NS = Cfg::kStages;
   constexpr int TPS = nc::kTilesPerSplit;
   constexpr int KT = nc::kKeyTile;
+  constexpr int TR = Cfg::kTileRows;
   constexpr uint32_t kAbortAfterNs = 1000000000u;
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base;
+  const uint32_t q_smem = base;  // tile X at X * TR * D * 2
   const uint32_t kv_smem = base + Cfg::kQBytes;
   const uint32_t bars = kv_smem + NS * Cfg::kStageBytes;
-  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 192);
-  // barrier map (8 bytes each)
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 448);
+  // barrier map (8 bytes each); per tile X and S buffer b: index 2 X + b
   const uint32_t k_full = bars, v_full = bars + 8 * NS, k_empty = bars + 16 * NS, v_empty = bars + 24 * NS;
-  const uint32_t s_full = bars + 32 * NS, s_empty = s_full + 16, p_full = s_full + 32, pv_done = s_full + 48;
+  const uint32_t s_full = bars + 32 * NS, p_full = s_full + 32, pv_done = s_full + 64;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -130,12 +141,18 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   const int kvh = blockIdx.x % P.Hkv;
   const ReqMeta rq = P.reqs[item.req];
   const int G = P.G;
-  const int row0 = item.row_group * nc::kRowsPerGroup;  // first row of the 128-row tile
+  const int row0 = item.row_group * nc::kRowsPerGroup;  // first row of the 256-row super tile
   const int rows = rq.q_len * G;
-  const int last_tok = min(rq.q_len - 1, (row0 + Cfg::kRows - 1) / G);
-  const int p_max = rq.start + last_tok;
   const int n_eff = rq.start + rq.q_len;
-  const int n_tiles = p_max / KT + 1;
+  // key tiles each 128-row tile walks (0: the tile does not exist)
+  int n_tiles_x[2];
+#pragma unroll
+  for (int X = 0; X < 2; ++X) {
+    const int first = row0 + X * TR;
+    const int last_tok = min(rq.q_len - 1, (first + TR - 1) / G);
+    n_tiles_x[X] = first < rows ? (rq.start + last_tok) / KT + 1 : 0;
+  }
+  const int n_tiles = max(n_tiles_x[0], n_tiles_x[1]);  // tile 1 holds later positions: it is the longer one
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -144,10 +161,9 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       mbar_init(k_empty + 8 * i, 1);
       mbar_init(v_empty + 8 * i, 1);
     }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
       mbar_init(s_full + 8 * i, 1);
-      mbar_init(s_empty + 8 * i, 128);
-      mbar_init(p_full + 8 * i, 128);
+      mbar_init(p_full + 8 * i, TR);
       mbar_init(pv_done + 8 * i, 1);
     }
     flags[0] = 0u;  // abort flag
@@ -155,13 +171,14 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     tma_prefetch_desc(&kv_map);
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 200), "r"(512));
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 456), "r"(512));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
-  // Q tile -> shared memory, [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
-  if (warp < 4) {
+  // Q tiles -> shared memory, per tile [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
+  if (warp < 8) {
     griddep_wait();
-    const int row = row0 + tid;
+    const int X = warp >> 2, r = tid & (TR - 1);
+    const int row = row0 + X * TR + r;
     const bool valid = row < rows;
     const int tok = row / G;
     const uint4* src = reinterpret_cast<const uint4*>(
@@ -169,7 +186,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
 #pragma unroll
     for (int c = 0; c < D / 8; ++c) {
       const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-      const uint32_t addr = q_smem + (c >> 3) * (Cfg::kRows * 128) + tid * 128 + (((c & 7) ^ (tid & 7)) << 4);
+      const uint32_t addr = q_smem + X * (TR * D * 2) + (c >> 3) * (TR * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
       asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                    : "memory");
     }
@@ -178,7 +195,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 200);
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 456);
 
   // Bounded wait shared by all roles: gives up after ~1 s or as soon as another
   // thread of the CTA has given up, records the failure, and lets the caller
@@ -199,9 +216,10 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     }
   };
 
-  if (warp == 4) {
-    // ================= TMA producer =================================================
+  if (warp == 8 || warp == 10) {
+    // ================= TMA producers: warp 8 loads the K tiles, warp 10 the V tiles =======
     griddep_wait();
+    const int is_v = warp == 10;
     const int32_t* bt = P.bt_flat + rq.bt_off;
     auto fetch_pages = [&](int split) -> int {
       const int pg = split * nc::kPagesPerSplit + lane;
@@ -218,35 +236,39 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       }
       const int ids = (split & 1) ? pages_odd : pages_even;
       const int n_valid = min(nc::kPagesPerTile, rq.n_pages - t * nc::kPagesPerTile);
-      const uint32_t kdst = kv_smem + s * Cfg::kStageBytes;
-      if (use > 0) ok = __all_sync(kFullMask, wait(k_empty + 8 * s, (use - 1) & 1));
+      const uint32_t dst = kv_smem + s * Cfg::kStageBytes + is_v * Cfg::kKBytes;
+      const uint32_t full = (is_v ? v_full : k_full) + 8 * s;
+      const uint32_t empty = (is_v ? v_empty : k_empty) + 8 * s;
+      if (use > 0) ok = __all_sync(kFullMask, wait(empty, (use - 1) & 1));
       if (!ok) break;
-      issue_stage_load<D, KT>(&kv_map, kdst, k_full + 8 * s, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, 0, lane);
-      if (use > 0) ok = __all_sync(kFullMask, wait(v_empty + 8 * s, (use - 1) & 1));
-      if (!ok) break;
-      issue_stage_load<D, KT>(&kv_map, kdst + Cfg::kKBytes, v_full + 8 * s, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv,
-                              kvh, 1, lane);
+      issue_stage_load<D, KT>(&kv_map, dst, full, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, is_v, lane);
     }
-  } else if (warp == 5) {
+  } else if (warp == 9) {
     // ================= MMA issuer ====================================================
+    // One thread's MMAs run in issue order.  S of key tile t+2 overwrites the buffer whose
+    // first columns PV of key tile t reads its weights from, so it is issued after that PV.
     if (lane == 0) {
       constexpr uint32_t idesc_s = umma_idesc(128, KT, false);
       constexpr uint32_t idesc_pv = umma_idesc(128, D, true);
       bool ok = true;
-      auto issue_s = [&](int t) {
+      auto issue_s = [&](int t) {  // S of both tiles for key tile t
         const int s = t % NS, b = t & 1;
         ok = ok && wait(k_full + 8 * s, (t / NS) & 1);
-        if (ok && t >= 2) ok = wait(s_empty + 8 * b, ((t >> 1) - 1) & 1);
         if (!ok) return;
         tc_fence_after();
         const uint32_t kst = kv_smem + s * Cfg::kStageBytes;
 #pragma unroll
-        for (int kc = 0; kc < D / 16; ++kc) {
-          const uint64_t da = smem_desc_sw128(q_smem + (kc >> 2) * (Cfg::kRows * 128) + (kc & 3) * 32, 16, 1024);
-          const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
-          tc_mma_ss(tmem + Cfg::kColS + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
+        for (int X = 0; X < 2; ++X) {
+          if (t >= n_tiles_x[X]) continue;
+          const uint32_t qx = q_smem + X * (TR * D * 2);
+#pragma unroll
+          for (int kc = 0; kc < D / 16; ++kc) {
+            const uint64_t da = smem_desc_sw128(qx + (kc >> 2) * (TR * 128) + (kc & 3) * 32, 16, 1024);
+            const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
+            tc_mma_ss(tmem + Cfg::kColS + X * 128 + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
+          }
+          tc_commit(s_full + 8 * (2 * X + b));
         }
-        tc_commit(s_full + 8 * b);
         tc_commit(k_empty + 8 * s);
       };
       issue_s(0);
@@ -254,49 +276,60 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         if (t + 1 < n_tiles) issue_s(t + 1);
         if (!ok) break;
         const int s = t % NS, b = t & 1;
-        ok = wait(p_full + 8 * b, (t >> 1) & 1);
-        if (ok) ok = wait(v_full + 8 * s, (t / NS) & 1);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+        ok = wait(v_full + 8 * s, (t / NS) & 1);
 #pragma unroll
-        for (int kc = 0; kc < KT / 16; ++kc) {
-          // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
-          const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
-          const uint32_t acc = (kc > 0 || (t % TPS) != 0) ? 1u : 0u;  // a split starts from a fresh accumulator
-          tc_mma_ts(tmem + Cfg::kColU, tmem + Cfg::kColP + b * 32 + kc * 8, db, idesc_pv, acc);
+        for (int X = 0; X < 2; ++X) {
+          if (!ok || t >= n_tiles_x[X]) continue;
+          ok = wait(p_full + 8 * (2 * X + b), (t >> 1) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+#pragma unroll
+          for (int kc = 0; kc < KT / 16; ++kc) {
+            // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
+            const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
+            const uint32_t acc = (kc > 0 || (t % TPS) != 0) ? 1u : 0u;  // a split starts from a fresh accumulator
+            tc_mma_ts(tmem + Cfg::kColU + X * D, tmem + Cfg::kColS + X * 128 + b * KT + kc * 8, db, idesc_pv, acc);
+          }
+          tc_commit(pv_done + 8 * (2 * X + b));
         }
-        tc_commit(pv_done + 8 * b);
+        if (!ok) break;
         tc_commit(v_empty + 8 * s);
       }
     }
-  } else {
+  } else if (warp < 8) {
     // ================= softmax / correction: one thread per row ======================
-    const int row = row0 + tid;
+    const int X = warp >> 2;                    // which 128-row tile
+    const int r = tid & (TR - 1);               // row of the tile = tensor-memory lane
+    const int row = row0 + X * TR + r;
     const bool valid = row < rows;
     const int tok = row / G;
     const int p = valid ? rq.start + tok : -1;  // padding rows see nothing
-    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t col_s = Cfg::kColS + X * 128, col_u = Cfg::kColU + X * D;
+    const int my_tiles = n_tiles_x[X];
     const float c = P.c;
+    // running fold of this tile in global memory ([D/4][128] float4: this thread owns column r),
+    // and the row's place in the output
+    float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + (static_cast<size_t>(blockIdx.x) * 2 + X) * (D / 4) * TR + r;
+    __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
     float m = -INFINITY, z = 0.f, mc = 0.f, zc = 0.f;
     bool ok = true;
-    for (int t = 0; t < n_tiles && ok; ++t) {
+    for (int t = 0; t < my_tiles && ok; ++t) {
       const int b = t & 1, s = t % NS;
       const int key0 = t * KT;
-      ok = __all_sync(kFullMask, wait(s_full + 8 * b, (t >> 1) & 1));
+      ok = __all_sync(kFullMask, wait(s_full + 8 * (2 * X + b), (t >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
       {
         uint32_t lo[32], hi[32];
-        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT, lo);
-        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT + 32, hi);
+        tmem_ld32(tmem + lane_sel + col_s + b * KT, lo);
+        tmem_ld32(tmem + lane_sel + col_s + b * KT + 32, hi);
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 32; ++i) { sr[i] = lo[i]; sr[32 + i] = hi[i]; }
       }
-      tc_fence_before();
-      mbar_arrive(s_empty + 8 * b);
 
       // ---- the scalar rules, lanes b = 0..63 of this row --------------------------
       // Schedule-only shortcut: when every key of the tile is visible to every real
@@ -350,7 +383,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
 
       // ---- U must be at rest before it is rescaled: PV of the previous tile done -----
       if (t > 0) {
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * ((t - 1) & 1), ((t - 1) >> 1) & 1));
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + ((t - 1) & 1)), ((t - 1) >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
       }
@@ -358,38 +391,46 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
 #pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t ur[32];
-          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
+          tmem_ld32(tmem + lane_sel + col_u + cb, ur);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) ur[i] = __float_as_uint(nc::u_rescale(__uint_as_float(ur[i]), alpha));
-          tmem_st32(tmem + lane_sel + Cfg::kColU + cb, ur);
+          tmem_st32(tmem + lane_sel + col_u + cb, ur);
         }
       }
-      tmem_st32(tmem + lane_sel + Cfg::kColP + b * 32, pk);
+      tmem_st32(tmem + lane_sel + col_s + b * KT, pk);  // the weights take the place of the scores read above
       tmem_wait_st();
       if (key0 + KT > n_eff) {
-        // Tail tile: zero the value rows at or beyond n_eff (not loaded, or pool garbage).
+        // Tail tile: zero the value rows at or beyond n_eff (not loaded, or pool garbage).  Only the
+        // last 128-row tile of a request reaches it; its 128 threads do the work.
         ok = __all_sync(kFullMask, wait(v_full + 8 * s, (t / NS) & 1));
         if (!ok) break;
         const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
         const int first = n_eff - key0;
         const int per_half = (KT - first) * 8;
-        for (int x = tid; x < per_half * (D / 64); x += 128) {
-          const int half = x / per_half, y = x - half * per_half;
+        for (int xx = r; xx < per_half * (D / 64); xx += TR) {
+          const int half = xx / per_half, y = xx - half * per_half;
           const uint32_t addr = vst + half * (KT * 128) + (first + (y >> 3)) * 128 + ((y & 7) << 4);
           asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
         }
         fence_proxy_async();
       }
       tc_fence_before();
-      mbar_arrive(p_full + 8 * b);
+      mbar_arrive(p_full + 8 * (2 * X + b));
 
-      // ---- end of a split: fold it into the running result ---------------------------
-      if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * b, (t >> 1) & 1));
+      // ---- end of a split: fold it into the running result (kept in global memory) -------
+      if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
+        const int split = t / TPS;
+        // the running-fold values do not depend on the PV in flight: request the first chunk now
+        float4 nxt4[8];
+        if (split > 0) {
+#pragma unroll
+          for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
+        }
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + b), (t >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
-        const int split = t / TPS;
+        const bool last = t + 1 == my_tiles;
         const bool sees = p >= split * nc::kSplitLen;
         nc::FoldFactors f;
         f.a = 1.f;
@@ -400,51 +441,51 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         } else if (sees) {
           f = nc::fold_scalars(mc, zc, m, z);
         }
+        const float inv = nc::out_scale(zc);  // used on the last split only
+        // chunks of 32 columns; the running-fold values of chunk c+1 are requested before chunk c is processed
 #pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t ur[32];
-          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
-          if (split == 0) {
-            tmem_wait_ld();
-            tmem_st32(tmem + lane_sel + Cfg::kColUc + cb, ur);
-          } else {
-            uint32_t uc[32];
-            tmem_ld32(tmem + lane_sel + Cfg::kColUc + cb, uc);
-            tmem_wait_ld();
+          tmem_ld32(tmem + lane_sel + col_u + cb, ur);
+          float un[32];
+          if (split > 0) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              uc[i] = sees ? __float_as_uint(nc::fold_u(__uint_as_float(uc[i]), __uint_as_float(ur[i]), f)) : uc[i];
-            tmem_st32(tmem + lane_sel + Cfg::kColUc + cb, uc);
+            for (int i = 0; i < 8; ++i) {
+              un[4 * i] = nxt4[i].x; un[4 * i + 1] = nxt4[i].y; un[4 * i + 2] = nxt4[i].z; un[4 * i + 3] = nxt4[i].w;
+            }
+            if (cb + 32 < D) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>((cb + 32) / 4 + i) * TR];
+            }
+          }
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float u = __uint_as_float(ur[i]);
+            un[i] = split == 0 ? u : (sees ? nc::fold_u(un[i], u, f) : un[i]);
+          }
+          if (last) {
+            if (valid) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 8) {
+                uint32_t o[4];
+#pragma unroll
+                for (int xx = 0; xx < 4; ++xx) {
+                  __nv_bfloat162 t2 = __floats2bfloat162_rn(nc::out_value(un[i + 2 * xx], inv),
+                                                            nc::out_value(un[i + 2 * xx + 1], inv));
+                  o[xx] = *reinterpret_cast<uint32_t*>(&t2);
+                }
+                *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(o[0], o[1], o[2], o[3]);
+              }
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              ucg[static_cast<size_t>(cb / 4 + i) * TR] = make_float4(un[4 * i], un[4 * i + 1], un[4 * i + 2], un[4 * i + 3]);
           }
         }
-        tmem_wait_st();
         m = -INFINITY;
         z = 0.f;
-      }
-    }
-    // ---- normalise and store --------------------------------------------------------------
-    if (ok) {
-      const float inv = nc::out_scale(zc);
-      __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
-#pragma unroll 1
-      for (int cb = 0; cb < D; cb += 32) {
-        uint32_t uc[32];
-        tmem_ld32(tmem + lane_sel + Cfg::kColUc + cb, uc);
-        tmem_wait_ld();
-        if (valid) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint32_t o[4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              __nv_bfloat162 t2 =
-                  __floats2bfloat162_rn(nc::out_value(__uint_as_float(uc[i + 2 * x]), inv),
-                                        nc::out_value(__uint_as_float(uc[i + 2 * x + 1]), inv));
-              o[x] = *reinterpret_cast<uint32_t*>(&t2);
-            }
-            *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(o[0], o[1], o[2], o[3]);
-          }
-        }
       }
     }
   }

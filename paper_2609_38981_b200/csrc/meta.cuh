@@ -41,6 +41,7 @@ struct AttnParams {
   const int2* split_tokens;  // (request, token) of every row the combine kernel finishes
   float* ws_u;               // partial U rows [rows][D]
   float2* ws_mz;             // partial (m, z) per row
+  float* ws_uc;              // running fold of the tile kernel: per CTA 2 x [D/4][128] float4
   uint32_t* status;
   int32_t n_workers;         // items of this launch times n_kv_heads
   int32_t n_split_tokens;

@@ -17,7 +17,7 @@ namespace {
 
 constexpr int kHostSlots = 8;        // ring of pinned staging buffers
 constexpr size_t kAlign = 1024;
-constexpr int kTileRows = 128;       // rows of one tile-kernel work item (8 row groups)
+constexpr int kTileRows = 256;       // rows of one tile-kernel work item (16 row groups)
 
 size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
 
@@ -42,7 +42,7 @@ struct Limits {
   int64_t part_rows_max;
   size_t meta_bytes;     // one metadata blob (attention or append)
   // workspace offsets
-  size_t off_status, off_meta, off_part_u, off_part_mz, off_stage_q, off_stage_o, off_stage_k,
+  size_t off_status, off_meta, off_part_u, off_part_mz, off_uc, off_stage_q, off_stage_o, off_stage_k,
       off_stage_v, total;
 };
 
@@ -70,6 +70,8 @@ Limits limits_of(const vosti_config& c) {
   L.off_meta = at; at += L.meta_bytes * kHostSlots;  // one region per staging slot
   L.off_part_u = at; at += align_up(sizeof(float) * L.part_rows_max * c.head_dim);
   L.off_part_mz = at; at += align_up(sizeof(float2) * L.part_rows_max);
+  L.off_uc = at;  // running fold of the tile kernel: one 256-row fp32 tile per (item, KV head)
+  at += align_up(sizeof(float) * items_seq * c.n_kv_heads * kTileRows * c.head_dim);
   const size_t qbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_q_heads * c.head_dim;
   const size_t kbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_kv_heads * c.head_dim;
   L.off_stage_q = at; at += align_up(qbytes);
@@ -659,6 +661,7 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   p.split_tokens = reinterpret_cast<const int2*>(dmeta + off_tok);
   p.ws_u = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_part_u);
   p.ws_mz = reinterpret_cast<float2*>(ctx->ws + ctx->lim.off_part_mz);
+  p.ws_uc = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_uc);
   p.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status);
   p.n_workers = 0;
   p.n_split_tokens = static_cast<int32_t>(n_split_tokens);

@@ -223,6 +223,7 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
                                                  sizeof(int32_t) * kMaxPageIds);
   p.ws_u = reinterpret_cast<float*>(scratch + kOffPartU);
   p.ws_mz = reinterpret_cast<float2*>(scratch + kOffPartMz);
+  p.ws_uc = nullptr;
   p.status = reinterpret_cast<uint32_t*>(scratch + kOffWords);
   p.n_workers = static_cast<int32_t>(n_items * n_kv_heads);
   p.n_split_tokens = static_cast<int32_t>(n_tok);

@@ -101,13 +101,13 @@ def test_plan_shapes(vb):
     # 8 tokens x G=4 = 32 rows: two row groups, still split-parallel
     items, n_split, _ = plan_of_request(vb, c, 8, 508)   # positions 508..515
     assert items == [(0, 0, 1), (1, 0, 1), (1, 1, 2)] and n_split == 3
-    # 9 tokens: 36 rows > 32 -> one 128-row tile item that walks all its splits in order
+    # 9 tokens: 36 rows > 32 -> one tile item that walks all its splits in order
     items, n_split, n_part = plan_of_request(vb, c, 9, 1020)
     assert n_split == 0 and n_part == 0
     assert items == [(0, 0, 3)]
-    # 100 tokens x G=4 = 400 rows: four tiles starting at row groups 0, 8, 16, 24
+    # 100 tokens x G=4 = 400 rows: two 256-row tiles starting at row groups 0 and 16
     items, n_split, _ = plan_of_request(vb, c, 100, 500)
-    assert n_split == 0 and items == [(0, 0, 2), (8, 0, 2), (16, 0, 2), (24, 0, 2)]
+    assert n_split == 0 and items == [(0, 0, 2), (16, 0, 2)]
     # boundaries: position exactly at a split edge
     assert plan_of_request(vb, c, 1, 511)[0] == [(0, 0, 1)]
     assert plan_of_request(vb, c, 1, 512)[0] == [(0, 0, 1), (0, 1, 2)]
