@@ -30,7 +30,8 @@ struct SplitKernelCfg {
 
 template <int D>
 __global__ void __launch_bounds__(SplitKernelCfg<D>::kWarps * 32, 1)
-attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {
+attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {  // kv_map: the 3-D page map
+  constexpr bool PM = true;  // stages are page-major: one TMA box per (page, K|V)
   constexpr int SK = SplitKernelCfg<D>::kStageKeys;
   using C = TileCfg<D, SK>;
   constexpr int kWarpsPerCta = SplitKernelCfg<D>::kWarps;
@@ -135,7 +136,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     const int part = sub - is_v * C::kParts;
     const int first_page = tl * nc::kPagesPerTile + part * C::kPagesPerStage;  // within the split
     const int stage = g_issue % R;
-    issue_stage_load<D, SK>(&kv_map, stage0 + stage * C::kStageBytes, bar0 + stage * 8, ids, first_page,
+    issue_stage_load<D, SK, PM>(&kv_map, stage0 + stage * C::kStageBytes, bar0 + stage * 8, ids, first_page,
                             max(0, min(C::kPagesPerStage, n_pages - (t_begin * nc::kPagesPerTile + first_page))),
                             P.Hkv, kvh, is_v, lane);
     ++g_issue;
@@ -192,7 +193,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
           timed_out = true;  // warp-uniform: every lane leaves together
           break;
         }
-        tile_scores<D, SK>(stage0 + stage * C::kStageBytes, qa, s, part * (SK / 8), lane);
+        tile_scores<D, SK, PM>(stage0 + stage * C::kStageBytes, qa, s, part * (SK / 8), lane);
         __syncwarp();
         ++g_cons;
         issue_one();
@@ -209,8 +210,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
         }
         const uint32_t vs = stage0 + stage * C::kStageBytes;
         const int part_key0 = key0 + part * SK;
-        if (part_key0 + SK > n_eff) zero_value_tail<D, SK>(vs, max(0, n_eff - part_key0), lane);
-        tile_pv<D, SK>(vs, pa, u, part * (SK / 16), lane);
+        if (part_key0 + SK > n_eff) zero_value_tail<D, SK, PM>(vs, max(0, n_eff - part_key0), lane);
+        tile_pv<D, SK, PM>(vs, pa, u, part * (SK / 16), lane);
         __syncwarp();
         ++g_cons;
         issue_one();

@@ -31,6 +31,20 @@ struct TileCfg {
   static constexpr int NT = nc::kKeyTile / 8;               // key column tiles of 8
 };
 
+// Address of the 16-byte chunk x (0 .. D/8-1) of key row `key` inside a stage.
+//   PM = false ("half-major", written by 2 KB boxes of 64 elements x 16 rows):
+//        [half][key 0..SK-1][128 B]            -- the canonical layout tcgen05 descriptors need
+//   PM = true ("page-major", written by ONE 4 KB box per page covering both halves):
+//        [page][half][16 rows][128 B]           -- half as many TMA instructions per stage
+// Either way a 128-byte row is swizzled by its row index mod 8.
+template <int D, int SK, bool PM>
+__device__ __forceinline__ uint32_t stage_addr(uint32_t base, int key, int x) {
+  if constexpr (PM)
+    return base + (key >> 4) * (D * 32) + (x >> 3) * 2048 + (key & 15) * 128 + (((x & 7) ^ (key & 7)) << 4);
+  else
+    return base + (x >> 3) * (SK * 128) + key * 128 + (((x & 7) ^ (key & 7)) << 4);
+}
+
 // Per-thread view of its two rows.
 struct RowPair {
   int p_a, p_b;       // logical positions (-1 for padding rows: they see nothing)
@@ -58,7 +72,7 @@ __device__ __forceinline__ void load_q_frags(uint32_t (&qa)[D / 16][4], const __
 
 // S = Q K^T for the keys of one K stage: column tiles n0 .. n0 + SK/8 - 1 of the
 // tile.  Head-dim chunks of 16 in ascending order.
-template <int D, int SK>
+template <int D, int SK, bool PM = false>
 __device__ __forceinline__ void tile_scores(uint32_t ks, const uint32_t (&qa)[D / 16][4],
                                             float (&s)[8][4], int n0, int lane) {
   using C = TileCfg<D, SK>;
@@ -76,8 +90,7 @@ __device__ __forceinline__ void tile_scores(uint32_t ks, const uint32_t (&qa)[D 
     for (int nn = 0; nn < NN; ++nn) {
       const int key = nn * 8 + lm_row;
       const int x = 4 * cp + lm_mat;
-      const uint32_t addr = ks + (x >> 3) * C::kHalfBytes + key * 128 + (((x & 7) ^ (key & 7)) << 4);
-      ldsm_x4(addr, b[nn][0], b[nn][1], b[nn][2], b[nn][3]);
+      ldsm_x4(stage_addr<D, SK, PM>(ks, key, x), b[nn][0], b[nn][1], b[nn][2], b[nn][3]);
     }
 #pragma unroll
     for (int nn = 0; nn < NN; ++nn) mma_bf16_16816(s[n0 + nn], qa[2 * cp], b[nn][0], b[nn][1]);
@@ -196,15 +209,15 @@ __device__ __forceinline__ void tile_softmax_dispatch(const float (&s)[8][4], in
 // whatever the pool had; zero them so that a zero weight times a non-finite
 // value cannot poison the row (the paper's zero-padded out-of-range loads).
 // first_bad_row: first row of the stage to clear (0 .. SK-1).
-template <int D, int SK>
+template <int D, int SK, bool PM = false>
 __device__ __forceinline__ void zero_value_tail(uint32_t vs, int first_bad_row, int lane) {
-  using C = TileCfg<D, SK>;
   const int per_half = (SK - first_bad_row) * 8;
   const int n_chunks = per_half * (D / 64);
   for (int x = lane; x < n_chunks; x += 32) {
     const int half = x / per_half;
     const int y = x - half * per_half;
-    const uint32_t addr = vs + half * C::kHalfBytes + (first_bad_row + (y >> 3)) * 128 + ((y & 7) << 4);
+    // every 16-byte chunk of the row is cleared, so the swizzle inside the row does not matter
+    const uint32_t addr = stage_addr<D, SK, PM>(vs, first_bad_row + (y >> 3), half * 8 + (y & 7));
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
   }
   // These generic-proxy writes precede a later TMA (async-proxy) refill of the same stage.
@@ -214,7 +227,7 @@ __device__ __forceinline__ void zero_value_tail(uint32_t vs, int first_bad_row, 
 
 // U += P V for the keys of one V stage: key chunks kc0 .. kc0 + SK/16 - 1 of the
 // tile.  Per accumulator the chunks are applied in ascending order.
-template <int D, int SK>
+template <int D, int SK, bool PM = false>
 __device__ __forceinline__ void tile_pv(uint32_t vs, const uint32_t (&pa)[4][4], float (&u)[D / 8][4],
                                         int kc0, int lane) {
   using C = TileCfg<D, SK>;
@@ -227,9 +240,8 @@ __device__ __forceinline__ void tile_pv(uint32_t vs, const uint32_t (&pa)[4][4],
     for (int e = 0; e < C::NE; e += 2) {
       const int key = kk * 16 + (lm_mat & 1) * 8 + lm_row;
       const int x = e + (lm_mat >> 1);
-      const uint32_t addr = vs + (x >> 3) * C::kHalfBytes + key * 128 + (((x & 7) ^ (key & 7)) << 4);
       uint32_t b0, b1, b2, b3;
-      ldsm_x4_trans(addr, b0, b1, b2, b3);
+      ldsm_x4_trans(stage_addr<D, SK, PM>(vs, key, x), b0, b1, b2, b3);
       mma_bf16_16816(u[e], pa[kc0 + kk], b0, b1);
       mma_bf16_16816(u[e + 1], pa[kc0 + kk], b2, b3);
     }
@@ -243,12 +255,13 @@ __device__ __forceinline__ void tile_pv(uint32_t vs, const uint32_t (&pa)[4][4],
 // instruction (a thread needs on the order of a hundred cycles per TMA
 // instruction, so issuing the boxes one after another from a single lane makes
 // the issuing warp the bottleneck).
-template <int D, int SK>
+// PM = true: `map` is the 3-D map (64 elements, rows, halves) and one box brings a whole page chunk.
+template <int D, int SK, bool PM = false>
 __device__ __forceinline__ void issue_stage_load(const CUtensorMap* map, uint32_t dst, uint32_t bar,
                                                  int ids, int first_lane, int n_valid, int Hkv, int kvh,
                                                  int is_v, int lane) {
   using C = TileCfg<D, SK>;
-  constexpr int HALVES = D / 64;
+  constexpr int HALVES = PM ? 1 : D / 64;
   constexpr int BOXES = C::kPagesPerStage * HALVES;
   if (lane == 0) mbar_expect_tx(bar, n_valid * nc::kPageSize * D * 2);
   const int j = lane / HALVES, h = lane % HALVES;  // page of the stage, 64-element half
@@ -256,7 +269,10 @@ __device__ __forceinline__ void issue_stage_load(const CUtensorMap* map, uint32_
   __syncwarp();
   if (lane < BOXES && j < n_valid) {
     const int32_t y = ((page * Hkv + kvh) * 2 + is_v) * nc::kPageSize;
-    tma_load_2d(dst + h * C::kHalfBytes + j * C::kPageBytes, map, h * 64, y, bar);
+    if constexpr (PM)
+      tma_load_3d(dst + j * (D * 32), map, 0, y, 0, bar);
+    else
+      tma_load_2d(dst + h * C::kHalfBytes + j * C::kPageBytes, map, h * 64, y, bar);
   }
 }
 

@@ -210,7 +210,8 @@ struct vosti_ctx {
   Limits lim;
   int device = 0;
   int sm_count = 1;
-  alignas(64) CUtensorMap kv_map;
+  alignas(64) CUtensorMap kv_map;    // 2-D: (d, rows), box 64 x 16: half-major stages (tile kernel)
+  alignas(64) CUtensorMap kv_map3;   // 3-D: (64, rows, d/64), box 64 x 16 x d/64: page-major stages (split kernel)
   HostSlot slots[kHostSlots];
   int next_slot = 0;
   cudaStream_t copy_stream = nullptr;  // metadata uploads overlap the previous call's kernels
@@ -248,7 +249,19 @@ vosti_status build_kv_map(vosti_ctx* ctx) {
       &ctx->kv_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, c.kv_pool, dims, strides, box, estr,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? VOSTI_OK : VOSTI_ERR_CUDA;
+  if (r != CUDA_SUCCESS) return VOSTI_ERR_CUDA;
+  // The same pool with the two 64-element halves of a row as a third dimension (its stride,
+  // 128 bytes, is smaller than the row stride: the encoder accepts that), so that one box
+  // of 64 x 16 x d/64 brings a whole 4 KB (page, head, K|V) chunk as [half][16 rows][128 B].
+  const cuuint64_t dims3[3] = {64, dims[1], static_cast<cuuint64_t>(c.head_dim / 64)};
+  const cuuint64_t strides3[2] = {static_cast<cuuint64_t>(c.head_dim) * 2, 128};
+  const cuuint32_t box3[3] = {64, static_cast<cuuint32_t>(c.page_size), static_cast<cuuint32_t>(c.head_dim / 64)};
+  const cuuint32_t estr3[3] = {1, 1, 1};
+  const CUresult r3 = reinterpret_cast<EncodeTiledFn>(fn)(
+      &ctx->kv_map3, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, c.kv_pool, dims3, strides3, box3, estr3,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r3 == CUDA_SUCCESS ? VOSTI_OK : VOSTI_ERR_CUDA;
 }
 
 // Claim the next pinned staging buffer, waiting for its previous copy if needed.
@@ -336,7 +349,7 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
     // persistent: one CTA per SM, warps draw (item, KV head) tickets
     const int grid = std::min((p.n_workers + Cfg::kWarps - 1) / Cfg::kWarps, ctx->sm_count);
     timed(1, [&] {
-      launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map, p);
+      launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3, p);
     });
   }
   if (n_seq > 0) {

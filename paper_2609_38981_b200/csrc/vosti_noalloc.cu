@@ -188,14 +188,14 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || !fn)
     return VOSTI_ERR_CUDA;
-  alignas(64) CUtensorMap map;
+  alignas(64) CUtensorMap map;  // the 3-D page map the split kernel gathers with: (64, rows, d/64)
   {
-    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(head_dim),
-                                static_cast<cuuint64_t>(num_pages) * n_kv_heads * 2 * page_size};
-    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(head_dim) * 2};
-    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(page_size)};
-    const cuuint32_t estr[2] = {1, 1};
-    if (reinterpret_cast<EncodeTiledFn>(fn)(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(kv_pool),
+    const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(num_pages) * n_kv_heads * 2 * page_size,
+                                static_cast<cuuint64_t>(head_dim / 64)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(head_dim) * 2, 128};
+    const cuuint32_t box[3] = {64, static_cast<cuuint32_t>(page_size), static_cast<cuuint32_t>(head_dim / 64)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    if (reinterpret_cast<EncodeTiledFn>(fn)(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(kv_pool),
                                             dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
