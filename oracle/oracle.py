@@ -47,12 +47,12 @@ def _load():
             lib.vosti_oracle_attention_dense.restype = ctypes.c_int
             lib.vosti_oracle_attention_dense.argtypes = [
                 u16p, u16p, u16p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
-                ctypes.c_int, ctypes.c_int, ctypes.c_double, f64p]
+                ctypes.c_int, ctypes.c_int, ctypes.c_double, ctypes.c_int64, f64p, f64p]
             lib.vosti_oracle_paged_attention.restype = ctypes.c_int
             lib.vosti_oracle_paged_attention.argtypes = [
                 u16p, u16p, i32p, i32p, i32p, i32p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                 ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_double,
-                i32p, ctypes.c_int64, f64p]
+                ctypes.c_int64, i32p, ctypes.c_int64, f64p, f64p]
             lib.vosti_oracle_kv_append.restype = ctypes.c_int
             lib.vosti_oracle_kv_append.argtypes = [
                 u16p, u16p, u16p, i32p, i32p, i32p, ctypes.c_int, ctypes.c_int, ctypes.c_int,
@@ -79,26 +79,30 @@ def num_threads() -> int:
     return int(_load().vosti_oracle_num_threads())
 
 
-def attention_dense(q, k, v, start: int, scale: float) -> np.ndarray:
+def attention_dense(q, k, v, start: int, scale: float, window: int = 0, return_lse: bool = False):
     """q [s,Hq,d], k/v [n,Hkv,d] (uint16 bf16 bits) -> float64 [s,Hq,d].
 
-    Row i is at logical position ``start + i`` and sees keys ``0..start+i``.
+    Row i is at logical position ``start + i`` and sees keys ``0..start+i``, or
+    only the last ``window`` of them when ``window > 0``.  With ``return_lse``
+    also returns the natural-log log-sum-exp of the scaled scores, [s,Hq].
     """
     q, k, v = _u16(q), _u16(k), _u16(v)
     s, Hq, d = q.shape
     n, Hkv, d2 = k.shape
     assert d == d2 and v.shape == k.shape
     out = np.empty((s, Hq, d), dtype=np.float64)
+    lse = np.empty((s, Hq), dtype=np.float64) if return_lse else None
     rc = _load().vosti_oracle_attention_dense(
         _ptr(q, ctypes.c_uint16), _ptr(k, ctypes.c_uint16), _ptr(v, ctypes.c_uint16),
-        s, n, int(start), Hq, Hkv, d, float(scale), _ptr(out, ctypes.c_double))
+        s, n, int(start), Hq, Hkv, d, float(scale), int(window), _ptr(out, ctypes.c_double),
+        _ptr(lse, ctypes.c_double) if return_lse else None)
     if rc:
         raise ValueError(f"oracle attention_dense failed: {rc}")
-    return out
+    return (out, lse) if return_lse else out
 
 
 def paged_attention(q, pool, q_lens, start_pos, seq_lens, block_tables, *, n_kv_heads: int,
-                    page_size: int, scale: float, sel=None) -> np.ndarray:
+                    page_size: int, scale: float, sel=None, window: int = 0, return_lse: bool = False):
     """Paged front-end.  q [T,Hq,d] uint16; pool uint16 of shape
     [num_pages,Hkv,2,P,d]; block_tables int32 [B,stride].
 
@@ -116,19 +120,22 @@ def paged_attention(q, pool, q_lens, start_pos, seq_lens, block_tables, *, n_kv_
     assert int(q_lens.sum()) == T
     if sel is None:
         out = np.empty((T, Hq, d), dtype=np.float64)
+        lse = np.empty((T, Hq), dtype=np.float64) if return_lse else None
         selp, nsel = None, 0
     else:
         sel = _i32(sel).reshape(-1, 3)
         out = np.empty((sel.shape[0], d), dtype=np.float64)
+        lse = np.empty((sel.shape[0],), dtype=np.float64) if return_lse else None
         selp, nsel = _ptr(sel, ctypes.c_int32), sel.shape[0]
     rc = _load().vosti_oracle_paged_attention(
         _ptr(q, ctypes.c_uint16), _ptr(pool, ctypes.c_uint16), _ptr(q_lens, ctypes.c_int32),
         _ptr(start_pos, ctypes.c_int32), _ptr(seq_lens, ctypes.c_int32),
         _ptr(bt, ctypes.c_int32), bt.shape[1], B, Hq, n_kv_heads, d, page_size, num_pages,
-        float(scale), selp, nsel, _ptr(out, ctypes.c_double))
+        float(scale), int(window), selp, nsel, _ptr(out, ctypes.c_double),
+        _ptr(lse, ctypes.c_double) if return_lse else None)
     if rc:
         raise ValueError(f"oracle paged_attention failed: {rc}")
-    return out
+    return (out, lse) if return_lse else out
 
 
 def kv_append(pool, k_new, v_new, q_lens, start_pos, block_tables) -> None:

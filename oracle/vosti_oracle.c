@@ -25,6 +25,12 @@
  *     No tiling, no online softmax, no splitting: those are properties of
  *     the kernel, not of the result.
  *   - Query head h reads KV head floor(h / G), G = n_q_heads / n_kv_heads.
+ *   - Sliding window (App. A, last paragraph: "adds j > p - w for shared window
+ *     size w > 0"): with window w > 0 key j is visible iff  p - w < j <= p;
+ *     w = 0 means no window.
+ *   - The auxiliary log-sum-exp the paper's kernel emits (App. A, after the
+ *     output equation): lse = log sum_j exp(scale * q.K_j) over visible keys,
+ *     natural logarithm, computed as  max + log(sum exp(s - max)).
  *
  * Inputs are bf16 bit patterns (uint16) widened exactly to double; every
  * sum is a plain left-to-right double sum.
@@ -78,9 +84,10 @@ static const uint16_t* kv_row(const kv_view* w, int64_t j, int kappa, int which)
  * over keys 0..p of KV head kappa.  out receives d doubles.
  * Returns 0, or -1 if memory ran out. */
 static int attend_row(const uint16_t* q, const kv_view* w, int64_t p, int kappa, double scale,
-                      double* out) {
+                      int64_t window, double* out, double* lse) {
   const int d = w->d;
-  const int64_t nvis = p + 1; /* keys j = 0..p are visible */
+  const int64_t j0 = (window > 0 && p - window + 1 > 0) ? p - window + 1 : 0; /* first visible key */
+  const int64_t nvis = p + 1 - j0;                                             /* keys j0..p are visible */
   double* s = (double*)malloc(sizeof(double) * (size_t)(nvis > 0 ? nvis : 1));
   if (!s) return -1;
   double qd[1024];
@@ -89,7 +96,7 @@ static int attend_row(const uint16_t* q, const kv_view* w, int64_t p, int kappa,
   /* scores and their maximum */
   double mx = -INFINITY;
   for (int64_t j = 0; j < nvis; ++j) {
-    const uint16_t* kr = kv_row(w, j, kappa, 0);
+    const uint16_t* kr = kv_row(w, j0 + j, kappa, 0);
     double acc = 0.0;
     for (int e = 0; e < d; ++e) acc += qd[e] * bf16_to_f64(kr[e]);
     s[j] = scale * acc;
@@ -104,11 +111,12 @@ static int attend_row(const uint16_t* q, const kv_view* w, int64_t p, int kappa,
   /* weighted values */
   for (int e = 0; e < d; ++e) out[e] = 0.0;
   for (int64_t j = 0; j < nvis; ++j) {
-    const uint16_t* vr = kv_row(w, j, kappa, 1);
+    const uint16_t* vr = kv_row(w, j0 + j, kappa, 1);
     for (int e = 0; e < d; ++e) out[e] += s[j] * bf16_to_f64(vr[e]);
   }
   const double inv = (z > 0.0) ? 1.0 / z : 0.0;
   for (int e = 0; e < d; ++e) out[e] *= inv;
+  if (lse) *lse = mx + log(z);
   free(s);
   return 0;
 }
@@ -124,11 +132,11 @@ int vosti_oracle_num_threads(void) {
 /* Dense front-end, one request.
  *   q   [s][Hq][d] bf16     rows at positions start .. start+s-1
  *   k,v [n][Hkv][d] bf16    the logical sequence, n >= start + s
- *   out [s][Hq][d] double
+ *   out [s][Hq][d] double;  lse [s][Hq] double or NULL;  window: 0 = none
  * Returns 0 on success, 1 on bad arguments, 2 if memory ran out. */
 int vosti_oracle_attention_dense(const uint16_t* q, const uint16_t* k, const uint16_t* v, int s,
                                  int n, int start, int Hq, int Hkv, int d, double scale,
-                                 double* out) {
+                                 int64_t window, double* out, double* lse /* [s][Hq] or NULL */) {
   if (s < 0 || n < 0 || start < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || d > 1024) return 1;
   if (Hq % Hkv != 0 || (int64_t)start + s > n) return 1;
   const int G = Hq / Hkv;
@@ -138,7 +146,9 @@ int vosti_oracle_attention_dense(const uint16_t* q, const uint16_t* k, const uin
   for (int i = 0; i < s; ++i)
     for (int h = 0; h < Hq; ++h) {
       const size_t row = (size_t)i * Hq + h;
-      if (attend_row(q + row * d, &w, (int64_t)start + i, h / G, scale, out + row * d)) fail = 1;
+      if (attend_row(q + row * d, &w, (int64_t)start + i, h / G, scale, window, out + row * d,
+                     lse ? lse + row : NULL))
+        fail = 1;
     }
   return fail ? 2 : 0;
 }
@@ -150,12 +160,13 @@ int vosti_oracle_attention_dense(const uint16_t* q, const uint16_t* k, const uin
  *   block_tables [B][bt_stride]   only entries < ceil(seq_len/P) are read
  *   sel          NULL: compute every row, out is [T][Hq][d];
  *                else n_sel triples (request, token i, head h): out is [n_sel][d]
+ *   lse          NULL, or [T][Hq] (resp. [n_sel]) doubles;  window: 0 = none
  * Returns 0 on success, 1 on bad arguments, 2 if memory ran out. */
 int vosti_oracle_paged_attention(const uint16_t* q, const uint16_t* pool, const int32_t* q_lens,
                                  const int32_t* start_pos, const int32_t* seq_lens,
                                  const int32_t* block_tables, int bt_stride, int B, int Hq, int Hkv,
-                                 int d, int P, int64_t num_pages, double scale,
-                                 const int32_t* sel, int64_t n_sel, double* out) {
+                                 int d, int P, int64_t num_pages, double scale, int64_t window,
+                                 const int32_t* sel, int64_t n_sel, double* out, double* lse) {
   if (B < 0 || Hq <= 0 || Hkv <= 0 || d <= 0 || d > 1024 || P <= 0 || Hq % Hkv != 0) return 1;
   const int G = Hq / Hkv;
   int64_t* row0 = (int64_t*)malloc(sizeof(int64_t) * (size_t)(B + 1));
@@ -190,7 +201,8 @@ int vosti_oracle_paged_attention(const uint16_t* q, const uint16_t* pool, const 
       const int64_t i = t - row0[r];
       kv_view w = {1, NULL, NULL, pool, block_tables + (size_t)r * bt_stride, P, Hkv, d};
       const size_t row = (size_t)t * Hq + h;
-      if (attend_row(q + row * d, &w, (int64_t)start_pos[r] + i, h / G, scale, out + row * d))
+      if (attend_row(q + row * d, &w, (int64_t)start_pos[r] + i, h / G, scale, window, out + row * d,
+                     lse ? lse + row : NULL))
         fail = 1;
     }
   } else {
@@ -206,8 +218,8 @@ int vosti_oracle_paged_attention(const uint16_t* q, const uint16_t* pool, const 
       const int r = sel[3 * x], i = sel[3 * x + 1], h = sel[3 * x + 2];
       kv_view w = {1, NULL, NULL, pool, block_tables + (size_t)r * bt_stride, P, Hkv, d};
       const size_t row = (size_t)(row0[r] + i) * Hq + h;
-      if (attend_row(q + row * d, &w, (int64_t)start_pos[r] + i, h / G, scale,
-                     out + (size_t)x * d))
+      if (attend_row(q + row * d, &w, (int64_t)start_pos[r] + i, h / G, scale, window,
+                     out + (size_t)x * d, lse ? lse + x : NULL))
         fail = 1;
     }
   }

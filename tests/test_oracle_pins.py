@@ -288,3 +288,84 @@ def test_kv_append_follows_the_logical_map_and_touches_nothing_else():
     assert np.array_equal(pool[~written], garbage[~written])
     with pytest.raises(ValueError):
         oracle.kv_append(pool, k, v, lens, [70, 1], bt)     # position beyond the table
+
+
+# ------------------------------------------------- sliding window and log-sum-exp
+
+def brute_force_window(q, k, v, start, scale, window):
+    """Dense attention with the window mask written out: p - w < j <= p."""
+    qf, kf, vf = widen(q), widen(k), widen(v)
+    s, Hq, d = qf.shape
+    n, Hkv, _ = kf.shape
+    G = Hq // Hkv
+    out = np.zeros((s, Hq, d))
+    lse = np.zeros((s, Hq))
+    pos = start + np.arange(s)[:, None]
+    j = np.arange(n)[None, :]
+    vis = (j <= pos) & ((j > pos - window) if window > 0 else True)
+    for h in range(Hq):
+        S = scale * (qf[:, h, :] @ kf[:, h // G, :].T)
+        S = np.where(vis, S, -np.inf)
+        mx = S.max(axis=1, keepdims=True)
+        W = np.exp(S - mx)
+        Z = W.sum(axis=1, keepdims=True)
+        out[:, h, :] = (W / Z) @ vf[:, h // G, :]
+        lse[:, h] = (mx + np.log(Z))[:, 0]
+    return out, lse
+
+
+@pytest.mark.parametrize("window", [1, 2, 5, 16, 17, 1000])
+def test_window_against_brute_force_and_lse(window):
+    gen = inputs.generator(300 + window)
+    s, n, start, Hq, Hkv, d = 11, 29, 18, 4, 2, 16
+    q, k, v = rand_bits(gen, s, Hq, d), rand_bits(gen, n, Hkv, d), rand_bits(gen, n, Hkv, d)
+    out, lse = oracle.attention_dense(q, k, v, start, 0.21, window=window, return_lse=True)
+    ref, ref_lse = brute_force_window(q, k, v, start, 0.21, window)
+    np.testing.assert_allclose(out, ref, rtol=1e-12, atol=1e-13)
+    np.testing.assert_allclose(lse, ref_lse, rtol=1e-12, atol=1e-13)
+
+
+def test_window_closed_forms():
+    gen = inputs.generator(31)
+    n, d = 21, 8
+    q, k, v = rand_bits(gen, n, 2, d), rand_bits(gen, n, 1, d), rand_bits(gen, n, 1, d)
+    vf = widen(v)
+    # a window of one sees only the key at the row's own position
+    out = oracle.attention_dense(q, k, v, 0, 0.4, window=1)
+    for p in range(n):
+        assert np.array_equal(out[p, 0], vf[p, 0]) and np.array_equal(out[p, 1], vf[p, 0])
+    # a window at least as long as the prefix changes nothing
+    assert np.array_equal(oracle.attention_dense(q, k, v, 0, 0.4, window=n),
+                          oracle.attention_dense(q, k, v, 0, 0.4))
+    # sigma = 0: the mean of the last w values, and lse = log(number of visible keys)
+    out, lse = oracle.attention_dense(q, k, v, 0, 0.0, window=4, return_lse=True)
+    for p in range(n):
+        lo = max(0, p - 3)
+        np.testing.assert_allclose(out[p, 0], vf[lo:p + 1, 0].mean(axis=0), rtol=1e-13, atol=1e-14)
+        np.testing.assert_allclose(lse[p], np.log(p + 1 - lo), rtol=1e-13, atol=1e-14)
+
+
+def test_lse_against_scipy_logsumexp():
+    from scipy.special import logsumexp
+    gen = inputs.generator(32)
+    n, d = 40, 32
+    q, k, v = rand_bits(gen, n, 2, d), rand_bits(gen, n, 2, d), rand_bits(gen, n, 2, d)
+    _, lse = oracle.attention_dense(q, k, v, 0, 0.3, return_lse=True)
+    qf, kf = widen(q), widen(k)
+    for p in (0, 7, 39):
+        for h in range(2):
+            np.testing.assert_allclose(lse[p, h], logsumexp(0.3 * (kf[:p + 1, h] @ qf[p, h])), rtol=1e-13)
+
+
+def test_paged_window_equals_dense_window():
+    geo = inputs.TINY
+    reqs = _paged_setup(41, geo, (90,), 16)
+    tables = inputs._assign_private_pages(inputs.generator(41), geo, 16, (90,))
+    pool = _fill_pool(geo, 16, reqs, tables, garbage_seed=5)
+    r = reqs[0]
+    dense, dlse = oracle.attention_dense(inputs.bits(r.q), inputs.bits(r.k), inputs.bits(r.v), 0, 0.125,
+                                         window=20, return_lse=True)
+    paged, plse = oracle.paged_attention(inputs.bits(r.q), pool, [90], [0], [90],
+                                         inputs.block_table_array(tables), n_kv_heads=2, page_size=16,
+                                         scale=0.125, window=20, return_lse=True)
+    assert np.array_equal(dense, paged) and np.array_equal(dlse, plse)
