@@ -109,6 +109,16 @@ vosti_status vosti_plan(const vosti_config* config, const int32_t* q_lens, const
                         const int32_t* seq_lens, int32_t batch, vosti_work_item* items, int64_t cap,
                         int64_t* n_items, int64_t* n_split, int64_t* n_partial_rows);
 
+/* The same plan under a sliding window of `window` keys (0: none; < 0 is
+ * INVALID_ARG): a row group only gets items for the splits that hold a key
+ * some row of the group sees (App. A, masks: the window adds j > p - w), and
+ * partial rows are counted from the first split the request's first row sees.
+ * A sequential item reports in split_begin / split_end the splits it walks. */
+vosti_status vosti_plan_ex(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
+                           const int32_t* seq_lens, int32_t batch, int32_t window,
+                           vosti_work_item* items, int64_t cap, int64_t* n_items, int64_t* n_split,
+                           int64_t* n_partial_rows);
+
 /* Create a context on the current CUDA device: checks the geometry, builds
  * the TMA tensor map of the pool, allocates host staging (the only memory
  * the library owns) and clears the device status word.  Synchronous. */
@@ -154,6 +164,29 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
                                    const int32_t* start_pos, const int32_t* seq_lens,
                                    const int32_t* block_tables, int32_t block_table_stride,
                                    int32_t batch, float softmax_scale, void* cuda_stream);
+
+/* vosti_paged_attention with the two options of App. A:
+ *   window   sliding window w >= 0 (App. A, masks: a window adds j > p - w to
+ *            the causal mask, so the row at p sees keys max(0, p-w+1) .. p);
+ *            0 means no window and gives exactly vosti_paged_attention.  Key
+ *            tiles and KV splits stay absolute (counted from key 0), so the
+ *            bits of a row still depend only on its own (p, head), the keys it
+ *            sees, sigma and w -- and with w > p they equal the unwindowed bits.
+ *            Block-table entries of pages that lie wholly before the window of
+ *            the request's first row, i.e. entries b < max(0, start_pos-w+1)/P,
+ *            are not read: the caller may have released those pages.
+ *   lse      device [T, n_q_heads] fp32, 4-byte aligned, or NULL: receives the
+ *            auxiliary log-sum-exp of the scaled scores over the visible keys
+ *            (App. A, after the output equation), natural logarithm:
+ *            (m + log2 z) ln 2 from the same folded (m, z) the output uses, so
+ *            it is batch-invariant bit for bit as well.
+ * All other arguments, premises and errors as for vosti_paged_attention;
+ * window < 0 is INVALID_ARG. */
+vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, float* lse,
+                                      const int32_t* q_lens, const int32_t* start_pos,
+                                      const int32_t* seq_lens, const int32_t* block_tables,
+                                      int32_t block_table_stride, int32_t batch, float softmax_scale,
+                                      int32_t window, void* cuda_stream);
 
 /* One serving step from HOST buffers: copies q, k_new, v_new to the device,
  * runs vosti_kv_append then vosti_paged_attention, copies the output back

@@ -27,8 +27,8 @@ VOSTI_OK, VOSTI_ERR_INVALID_ARG, VOSTI_ERR_UNSUPPORTED_CONFIG, VOSTI_ERR_OUT_OF_
 VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
 
 EXPORTS = (
-    "vosti_workspace_bytes", "vosti_plan", "vosti_create", "vosti_destroy", "vosti_kv_append",
-    "vosti_paged_attention", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
+    "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
+    "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
 )
@@ -61,6 +61,11 @@ _lib.vosti_plan.argtypes = [_cfgp, _i32p, _i32p, _i32p, ctypes.c_int32,
                             ctypes.POINTER(vosti_work_item), ctypes.c_int64,
                             ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
                             ctypes.POINTER(ctypes.c_int64)]
+_lib.vosti_plan_ex.restype = ctypes.c_int
+_lib.vosti_plan_ex.argtypes = [_cfgp, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32,
+                               ctypes.POINTER(vosti_work_item), ctypes.c_int64,
+                               ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                               ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_create.restype = ctypes.c_int
 _lib.vosti_create.argtypes = [ctypes.POINTER(_vp), _cfgp]
 _lib.vosti_destroy.restype = ctypes.c_int
@@ -71,6 +76,9 @@ _lib.vosti_kv_append.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, ctypes.c_in
 _lib.vosti_paged_attention.restype = ctypes.c_int
 _lib.vosti_paged_attention.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32,
                                        ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_paged_attention_ex.restype = ctypes.c_int
+_lib.vosti_paged_attention_ex.argtypes = [_vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32,
+                                          ctypes.c_int32, ctypes.c_float, ctypes.c_int32, _vp]
 _lib.vosti_paged_attention_noalloc.restype = ctypes.c_int
 _lib.vosti_paged_attention_noalloc.argtypes = [
     ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp, ctypes.c_int64, _vp, _vp,
@@ -167,6 +175,21 @@ def vosti_plan(cfg: vosti_config, q_lens, start_pos, seq_lens):
     return arr, nsp.value, npr.value
 
 
+def vosti_plan_ex(cfg: vosti_config, q_lens, start_pos, seq_lens, window: int):
+    """Host-only planning under a sliding window.  Returns like vosti_plan."""
+    q, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    cnt, nsp, npr = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.vosti_plan_ex(ctypes.byref(cfg), _ip(q), _ip(s), _ip(n), len(q), int(window), None, 0,
+                              ctypes.byref(cnt), ctypes.byref(nsp), ctypes.byref(npr)), "vosti_plan_ex")
+    items = (vosti_work_item * max(cnt.value, 1))()
+    _check(_lib.vosti_plan_ex(ctypes.byref(cfg), _ip(q), _ip(s), _ip(n), len(q), int(window), items,
+                              cnt.value, ctypes.byref(cnt), ctypes.byref(nsp), ctypes.byref(npr)),
+           "vosti_plan_ex")
+    arr = np.array([[it.req, it.row_group, it.split_begin, it.split_end]
+                    for it in items[:cnt.value]], dtype=np.int32).reshape(-1, 4)
+    return arr, nsp.value, npr.value
+
+
 def vosti_fingerprint(ctx=None) -> int:
     return int(_lib.vosti_fingerprint(ctx.handle if ctx is not None else None))
 
@@ -235,6 +258,18 @@ def vosti_paged_attention(ctx: Context, q, out, q_lens, start_pos, seq_lens, blo
     _check(_lib.vosti_paged_attention(ctx.handle, _dev(q), _dev(out), _ip(ql), _ip(s), _ip(n),
                                       _ip(bt), bt.shape[1], len(ql), float(softmax_scale),
                                       _stream(stream)), "vosti_paged_attention")
+
+
+def vosti_paged_attention_ex(ctx: Context, q, out, lse, q_lens, start_pos, seq_lens, block_tables,
+                             softmax_scale: float, window: int = 0, stream=None) -> None:
+    """With a sliding window and / or the log-sum-exp output (lse: fp32 [T, Hq] or None)."""
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    assert bt.ndim == 2 and bt.shape[0] == len(ql)
+    _check(_lib.vosti_paged_attention_ex(ctx.handle, _dev(q), _dev(out), _dev(lse) if lse is not None else None,
+                                         _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1], len(ql),
+                                         float(softmax_scale), int(window), _stream(stream)),
+           "vosti_paged_attention_ex")
 
 
 def vosti_paged_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_size, kv_pool, q, out,

@@ -64,6 +64,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
   struct Desc {
     uint32_t ticket;
     int kvh, t_begin, n_loads, n_pages, ids;
+    int split_tile0;  // first key tile of the item's split (t_begin may lie after it under a window)
   };
   auto read_item = [&](uint32_t ticket) -> SplitItem {
     const int4* src = reinterpret_cast<const int4*>(P.split_items + ticket / P.Hkv);
@@ -72,7 +73,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     si.q_row0 = a.x; si.q_len = a.y; si.start = a.z; si.n_pages = a.w;
     si.bt_index = b.x; si.split = b.y; si.row_group = b.z; si.n_splits = b.w;
     si.part_base = (static_cast<int64_t>(static_cast<uint32_t>(d.y)) << 32) | static_cast<uint32_t>(d.x);
-    si.req = d.z; si.pad = d.w;
+    si.req = d.z; si.first_split = d.w;
     return si;
   };
   // The first ticket of worker w is w itself; later ones come from the counter.
@@ -87,9 +88,13 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     const SplitItem si = read_item(t);
     const int last_tok = min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
     const int t_end = min((si.split + 1) * TPS, (si.start + last_tok) / nc::kKeyTile + 1);
+    // under a sliding window the group's first row needs nothing before this tile
+    const int first_tok = (si.row_group * nc::kRowsPerGroup) / G;
+    const int t_first = nc::first_key(si.start + first_tok, P.window) / nc::kKeyTile;
     d.ticket = t;
     d.kvh = static_cast<int>(t % P.Hkv);
-    d.t_begin = si.split * TPS;
+    d.split_tile0 = si.split * TPS;
+    d.t_begin = max(si.split * TPS, t_first);
     d.n_loads = LPT * (t_end - d.t_begin);
     d.n_pages = si.n_pages;
     d.ids = (si.split * nc::kPagesPerSplit + lane < si.n_pages) ? __ldg(P.bt_flat + si.bt_index + lane) : -1;
@@ -130,14 +135,16 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     const int n_loads = ahead ? nxt.n_loads : cur.n_loads;
     const int n_pages = ahead ? nxt.n_pages : cur.n_pages;
     const int ids = ahead ? nxt.ids : cur.ids;
-    const int tl = prod_li / LPT;          // tile within the split
-    const int sub = prod_li - tl * LPT;    // 0 .. kParts-1: K parts, then V parts
+    const int split_tile0 = ahead ? nxt.split_tile0 : cur.split_tile0;
+    const int tl = t_begin - split_tile0 + prod_li / LPT;  // tile within the split
+    const int tw = prod_li / LPT;                           // tile within the item
+    const int sub = prod_li - tw * LPT;    // 0 .. kParts-1: K parts, then V parts
     const int is_v = sub >= C::kParts;
     const int part = sub - is_v * C::kParts;
     const int first_page = tl * nc::kPagesPerTile + part * C::kPagesPerStage;  // within the split
     const int stage = g_issue % R;
     issue_stage_load<D, SK, PM>(&kv_map, stage0 + stage * C::kStageBytes, bar0 + stage * 8, ids, first_page,
-                            max(0, min(C::kPagesPerStage, n_pages - (t_begin * nc::kPagesPerTile + first_page))),
+                            max(0, min(C::kPagesPerStage, n_pages - (split_tile0 * nc::kPagesPerTile + first_page))),
                             P.Hkv, kvh, is_v, lane);
     ++g_issue;
     if (++prod_li == n_loads) {
@@ -162,10 +169,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     RowPair r;
     r.p_a = valid_a ? si.start + tok_a : -1;
     r.p_b = valid_b ? si.start + tok_b : -1;
+    r.lo_a = nc::window_lo(r.p_a, P.window);
+    r.lo_b = nc::window_lo(r.p_b, P.window);
     r.reset();
     const int n_eff = si.start + si.q_len;
-    // schedule-only facts about the group: lowest real position, whether rows 8..15 hold real rows
+    // schedule-only facts about the group: lowest and highest real position (a tile between the
+    // highest row's window start and the lowest row's position is visible to every real row),
+    // and whether rows 8..15 hold real rows
     const int p_min = si.start + (si.row_group * nc::kRowsPerGroup) / G;
+    const int p_top = si.start + min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
+    const int lo_top = nc::window_lo(p_top, P.window);
+    const int lo_first = nc::window_lo(p_min, P.window);  // keys up to here are invisible to the whole group
     const bool upper_rows = (si.row_group * nc::kRowsPerGroup + 8) / G < si.q_len;
     uint32_t qa[C::KC][4];
     load_q_frags<D>(qa,
@@ -200,7 +214,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
       }
       if (timed_out) break;
       uint32_t pa[4][4];
-      tile_softmax_dispatch<D>(s, key0, c, r, u, pa, quad, key0 + nc::kKeyTile - 1 <= p_min, upper_rows);
+      tile_softmax_dispatch<D>(s, key0, c, r, u, pa, quad, key0 + nc::kKeyTile - 1 <= p_min && key0 > lo_top,
+                               upper_rows);
 #pragma unroll
       for (int part = 0; part < C::kParts; ++part) {
         const int stage = g_cons % R;
@@ -211,6 +226,7 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
         const uint32_t vs = stage0 + stage * C::kStageBytes;
         const int part_key0 = key0 + part * SK;
         if (part_key0 + SK > n_eff) zero_value_tail<D, SK, PM>(vs, max(0, n_eff - part_key0), lane);
+        if (part_key0 <= lo_first) zero_value_rows<D, SK, PM>(vs, 0, min(SK, lo_first - part_key0 + 1), lane);
         tile_pv<D, SK, PM>(vs, pa, u, part * (SK / 16), lane);
         __syncwarp();
         ++g_cons;
@@ -223,16 +239,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     // ---- partial (m, z, U) of this split for the rows that see it -----------------
     {
       const int rows = si.q_len * G;
-      const int64_t slab = si.part_base + (static_cast<int64_t>(kvh) * si.n_splits + si.split) * rows;
-      const int first_key = si.split * nc::kSplitLen;
-      if (valid_a && r.p_a >= first_key) {
+      const int64_t slab =
+          si.part_base + (static_cast<int64_t>(kvh) * si.n_splits + (si.split - si.first_split)) * rows;
+      const int first_key = si.split * nc::kSplitLen, last_key = first_key + nc::kSplitLen - 1;
+      if (valid_a && r.p_a >= first_key && r.lo_a < last_key) {
         float* dst = P.ws_u + (slab + row_a) * D + 2 * quad;
 #pragma unroll
         for (int e = 0; e < C::NE; ++e)
           *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][0], u[e][1]);
         if (quad == 0) P.ws_mz[slab + row_a] = make_float2(r.m_a, r.z_a);
       }
-      if (valid_b && r.p_b >= first_key) {
+      if (valid_b && r.p_b >= first_key && r.lo_b < last_key) {
         float* dst = P.ws_u + (slab + row_b) * D + 2 * quad;
 #pragma unroll
         for (int e = 0; e < C::NE; ++e)

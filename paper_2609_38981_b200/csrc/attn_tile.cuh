@@ -153,6 +153,12 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     n_tiles_x[X] = first < rows ? (rq.start + last_tok) / KT + 1 : 0;
   }
   const int n_tiles = max(n_tiles_x[0], n_tiles_x[1]);  // tile 1 holds later positions: it is the longer one
+  // Under a sliding window nothing before the first visible key of the item's first row is
+  // needed: both tiles start at key tile T0 (rows whose own window starts later take identity
+  // steps until it does).  Stages, S buffers and barrier phases are indexed by t - T0.
+  const int p_first = rq.start + row0 / G;
+  const int T0 = nc::first_key(p_first, P.window) / KT;
+  const int lo_first = nc::window_lo(p_first, P.window);  // keys up to here are invisible to every row
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -225,12 +231,13 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       const int pg = split * nc::kPagesPerSplit + lane;
       return pg < rq.n_pages ? __ldg(bt + pg) : -1;
     };
-    int pages_even = fetch_pages(0), pages_odd = -1;
+    int pages_even = -1, pages_odd = -1;
+    if ((T0 / TPS) & 1) pages_odd = fetch_pages(T0 / TPS); else pages_even = fetch_pages(T0 / TPS);
     bool ok = true;
-    for (int t = 0; t < n_tiles && ok; ++t) {
-      const int s = t % NS, use = t / NS;
+    for (int t = T0; t < n_tiles && ok; ++t) {
+      const int s = (t - T0) % NS, use = (t - T0) / NS;
       const int split = t / TPS, tl = t - split * TPS;
-      if (tl == TPS / 2 && (split + 1) * TPS < n_tiles) {
+      if ((tl == TPS / 2 || (t == T0 && tl > TPS / 2)) && (split + 1) * TPS < n_tiles) {
         const int ids = fetch_pages(split + 1);
         if ((split + 1) & 1) pages_odd = ids; else pages_even = ids;
       }
@@ -252,8 +259,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       constexpr uint32_t idesc_pv = umma_idesc(128, D, true);
       bool ok = true;
       auto issue_s = [&](int t) {  // S of both tiles for key tile t
-        const int s = t % NS, b = t & 1;
-        ok = ok && wait(k_full + 8 * s, (t / NS) & 1);
+        const int i = t - T0, s = i % NS, b = i & 1;
+        ok = ok && wait(k_full + 8 * s, (i / NS) & 1);
         if (!ok) return;
         tc_fence_after();
         const uint32_t kst = kv_smem + s * Cfg::kStageBytes;
@@ -271,16 +278,16 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         }
         tc_commit(k_empty + 8 * s);
       };
-      issue_s(0);
-      for (int t = 0; t < n_tiles && ok; ++t) {
+      issue_s(T0);
+      for (int t = T0; t < n_tiles && ok; ++t) {
         if (t + 1 < n_tiles) issue_s(t + 1);
         if (!ok) break;
-        const int s = t % NS, b = t & 1;
-        ok = wait(v_full + 8 * s, (t / NS) & 1);
+        const int i = t - T0, s = i % NS, b = i & 1;
+        ok = wait(v_full + 8 * s, (i / NS) & 1);
 #pragma unroll
         for (int X = 0; X < 2; ++X) {
           if (!ok || t >= n_tiles_x[X]) continue;
-          ok = wait(p_full + 8 * (2 * X + b), (t >> 1) & 1);
+          ok = wait(p_full + 8 * (2 * X + b), (i >> 1) & 1);
           if (!ok) break;
           tc_fence_after();
           const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
@@ -288,7 +295,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           for (int kc = 0; kc < KT / 16; ++kc) {
             // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
             const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
-            const uint32_t acc = (kc > 0 || (t % TPS) != 0) ? 1u : 0u;  // a split starts from a fresh accumulator
+            // a split (and the first tile walked) starts from a fresh accumulator
+            const uint32_t acc = (kc > 0 || ((t % TPS) != 0 && t != T0)) ? 1u : 0u;
             tc_mma_ts(tmem + Cfg::kColU + X * D, tmem + Cfg::kColS + X * 128 + b * KT + kc * 8, db, idesc_pv, acc);
           }
           tc_commit(pv_done + 8 * (2 * X + b));
@@ -305,6 +313,10 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     const bool valid = row < rows;
     const int tok = row / G;
     const int p = valid ? rq.start + tok : -1;  // padding rows see nothing
+    const int lo = nc::window_lo(p, P.window);  // key j is visible iff lo < j <= p
+    // first split the row sees; before it (and in the first split the CTA walks) the
+    // running result is simply taken from the split, as the fold of the split kernels does
+    const int k_first = max(nc::first_key(p, P.window) / nc::kSplitLen, T0 / TPS);
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const uint32_t col_s = Cfg::kColS + X * 128, col_u = Cfg::kColU + X * D;
     const int my_tiles = n_tiles_x[X];
@@ -315,10 +327,10 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
     float m = -INFINITY, z = 0.f, mc = 0.f, zc = 0.f;
     bool ok = true;
-    for (int t = 0; t < my_tiles && ok; ++t) {
-      const int b = t & 1, s = t % NS;
+    for (int t = T0; t < my_tiles && ok; ++t) {
+      const int ti = t - T0, b = ti & 1, s = ti % NS;
       const int key0 = t * KT;
-      ok = __all_sync(kFullMask, wait(s_full + 8 * (2 * X + b), (t >> 1) & 1));
+      ok = __all_sync(kFullMask, wait(s_full + 8 * (2 * X + b), (ti >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
@@ -334,8 +346,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       // ---- the scalar rules, lanes b = 0..63 of this row --------------------------
       // Schedule-only shortcut: when every key of the tile is visible to every real
       // row of the warp the selects all take the visible arm and are skipped.
-      const bool all_visible = __all_sync(kFullMask, !valid || key0 + KT - 1 <= p);
-      const bool h = all_visible || key0 <= p;
+      const bool all_visible = __all_sync(kFullMask, !valid || (key0 + KT - 1 <= p && key0 > lo));
+      const bool h = all_visible || (key0 <= p && key0 + KT - 1 > lo);
       float mn, alpha;
       float w[KT];
       if (all_visible) {
@@ -352,13 +364,14 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int i = 0; i < KT; ++i)
-          mx4[i & 3] = fmaxf(mx4[i & 3], key0 + i <= p ? __uint_as_float(sr[i]) : -INFINITY);
+          mx4[i & 3] = fmaxf(mx4[i & 3], (key0 + i <= p && key0 + i > lo) ? __uint_as_float(sr[i]) : -INFINITY);
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         mn = h ? nc::new_max(m, mx, c) : m;
         alpha = h ? nc::rescale(m, mn) : 1.0f;
         const float ng = -mn;
 #pragma unroll
-        for (int i = 0; i < KT; ++i) w[i] = key0 + i <= p ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
+        for (int i = 0; i < KT; ++i)
+          w[i] = (key0 + i <= p && key0 + i > lo) ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
       }
       {
         // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3)
@@ -382,12 +395,12 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       }
 
       // ---- U must be at rest before it is rescaled: PV of the previous tile done -----
-      if (t > 0) {
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + ((t - 1) & 1)), ((t - 1) >> 1) & 1));
+      if (ti > 0) {
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + ((ti - 1) & 1)), ((ti - 1) >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
       }
-      if ((t % TPS) != 0 && !__all_sync(kFullMask, alpha == 1.0f)) {
+      if ((t % TPS) != 0 && t != T0 && !__all_sync(kFullMask, alpha == 1.0f)) {
 #pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t ur[32];
@@ -403,7 +416,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       if (key0 + KT > n_eff) {
         // Tail tile: zero the value rows at or beyond n_eff (not loaded, or pool garbage).  Only the
         // last 128-row tile of a request reaches it; its 128 threads do the work.
-        ok = __all_sync(kFullMask, wait(v_full + 8 * s, (t / NS) & 1));
+        ok = __all_sync(kFullMask, wait(v_full + 8 * s, (ti / NS) & 1));
         if (!ok) break;
         const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
         const int first = n_eff - key0;
@@ -415,6 +428,20 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         }
         fence_proxy_async();
       }
+      if (key0 <= lo_first) {
+        // First tile under a sliding window: the value rows before the window of the item's first
+        // row are visible to no row, and their pages may have been given back: zero them as well.
+        ok = __all_sync(kFullMask, wait(v_full + 8 * s, (ti / NS) & 1));
+        if (!ok) break;
+        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+        const int per_half = min(KT, lo_first - key0 + 1) * 8;
+        for (int xx = r; xx < per_half * (D / 64); xx += TR) {
+          const int half = xx / per_half, y = xx - half * per_half;
+          const uint32_t addr = vst + half * (KT * 128) + (y >> 3) * 128 + ((y & 7) << 4);
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        }
+        fence_proxy_async();
+      }
       tc_fence_before();
       mbar_arrive(p_full + 8 * (2 * X + b));
 
@@ -422,20 +449,22 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
         const int split = t / TPS;
         // the running-fold values do not depend on the PV in flight: request the first chunk now
+        const bool resume = split > T0 / TPS;  // the CTA has stored a running result before
         float4 nxt4[8];
-        if (split > 0) {
+        if (resume) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
         }
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + b), (t >> 1) & 1));
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + b), (ti >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
         const bool last = t + 1 == my_tiles;
+        const bool take = split <= k_first;  // the row's first split: the running result starts from it
         const bool sees = p >= split * nc::kSplitLen;
         nc::FoldFactors f;
         f.a = 1.f;
         f.b = 0.f;
-        if (split == 0) {
+        if (take) {
           mc = m;
           zc = z;
         } else if (sees) {
@@ -448,7 +477,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           uint32_t ur[32];
           tmem_ld32(tmem + lane_sel + col_u + cb, ur);
           float un[32];
-          if (split > 0) {
+          if (resume) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
               un[4 * i] = nxt4[i].x; un[4 * i + 1] = nxt4[i].y; un[4 * i + 2] = nxt4[i].z; un[4 * i + 3] = nxt4[i].w;
@@ -462,10 +491,12 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
 #pragma unroll
           for (int i = 0; i < 32; ++i) {
             const float u = __uint_as_float(ur[i]);
-            un[i] = split == 0 ? u : (sees ? nc::fold_u(un[i], u, f) : un[i]);
+            un[i] = take ? u : (sees ? nc::fold_u(un[i], u, f) : un[i]);
           }
           if (last) {
             if (valid) {
+              if (cb == 0 && P.lse != nullptr)
+                P.lse[static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G] = nc::lse_value(mc, zc);
 #pragma unroll
               for (int i = 0; i < 32; i += 8) {
                 uint32_t o[4];

@@ -25,8 +25,12 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
   const int row = rt.y * P.G + head % P.G;
   const int rows = rq.q_len * P.G;
   const int p = rq.start + rt.y;
-  const int n_splits = p / nc::kSplitLen + 1;
-  const int64_t slab0 = rq.part_base + static_cast<int64_t>(kvh) * rq.n_splits * rows + row;
+  // the row's splits: from the one holding its first visible key to the one holding p;
+  // partial slabs of the request are indexed from the request's first split
+  const int k_lo = nc::first_key(p, P.window) / nc::kSplitLen;
+  const int n_splits = p / nc::kSplitLen - k_lo + 1;
+  const int64_t slab0 =
+      rq.part_base + (static_cast<int64_t>(kvh) * rq.n_splits + (k_lo - rq.first_split)) * rows + row;
   griddep_wait();  // partials come from the kernel before this one in the stream
 
   auto load_u = [&](int64_t slab, float (&u)[V]) {
@@ -67,6 +71,7 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
       }
   }
   const float inv = nc::out_scale(zc);
+  if (P.lse != nullptr && lane == 0) P.lse[static_cast<size_t>(rq.q_row0 + rt.y) * P.Hq + head] = nc::lse_value(mc, zc);
   __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + rt.y) * P.Hq + head) * D + lane * V;
 #pragma unroll
   for (int i = 0; i < V; i += 2)

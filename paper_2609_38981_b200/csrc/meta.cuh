@@ -14,7 +14,9 @@ struct ReqMeta {
   int32_t start;      // logical position of row 0
   int32_t n_pages;    // used pages = ceil((start + q_len) / P)
   int32_t bt_off;     // offset of the request's page ids in the flat table
-  int32_t n_splits;   // splits touched by the last row: (start + q_len - 1) / L_S + 1
+  int32_t n_splits;   // splits the request's rows touch: last split - first_split + 1
+  int32_t first_split;  // first split any row of the request sees (0 without a sliding window)
+  int32_t pad;
   int64_t part_base;  // first partial row of the request (split-parallel requests only)
 };
 
@@ -25,7 +27,8 @@ struct SplitItem {
   int32_t bt_index;  // index in the flat table of the first page of this split
   int32_t split, row_group, n_splits;
   int64_t part_base;
-  int32_t req, pad;
+  int32_t req;
+  int32_t first_split;  // of the request: partial slabs are indexed by split - first_split
 };
 static_assert(sizeof(SplitItem) == 48, "SplitItem is read as three 16-byte words");
 
@@ -47,6 +50,8 @@ struct AttnParams {
   int32_t n_split_tokens;
   int32_t Hq, Hkv, G;
   float c;                   // sigma * log2(e), rounded once on the host
+  int32_t window;            // sliding window w: key j visible iff p - w < j <= p; 0 = no window
+  float* lse;                // optional [T][Hq] natural-log log-sum-exp output, or nullptr
 };
 
 struct AppendParams {

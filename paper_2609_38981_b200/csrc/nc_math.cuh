@@ -92,5 +92,23 @@ __device__ __forceinline__ float out_value(float u, float inv) {
   return __fadd_rn(__fmul_rn(u, inv), 0.0f);
 }
 
+// Auxiliary log-sum-exp of the scaled scores, natural logarithm: (m + log2 z) ln 2.
+__device__ __forceinline__ float lse_value(float m, float z) {
+  float l;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(l) : "f"(z));
+  return __fmul_rn(__fadd_rn(m, l), 0.693147180559945309f);
+}
+
+// Sliding window (App. A: "adds j > p - w"): the row at p sees keys lo < j <= p with
+// lo = p - w; without a window lo lies below every key.  Padding rows (p = -1) see nothing.
+constexpr int kNoLowerBound = -0x40000000;
+__device__ __forceinline__ int window_lo(int p, int window) {
+  return (window > 0 && p >= 0) ? p - window : kNoLowerBound;
+}
+// First key tile / split a row (or a group whose first row is at p) needs.
+__device__ __forceinline__ int first_key(int p, int window) {
+  return (window > 0 && p - window + 1 > 0) ? p - window + 1 : 0;
+}
+
 }  // namespace nc
 }  // namespace vosti

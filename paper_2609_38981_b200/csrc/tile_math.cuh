@@ -48,6 +48,7 @@ __device__ __forceinline__ uint32_t stage_addr(uint32_t base, int key, int x) {
 // Per-thread view of its two rows.
 struct RowPair {
   int p_a, p_b;       // logical positions (-1 for padding rows: they see nothing)
+  int lo_a, lo_b;     // window lower bounds: key j is visible iff lo < j <= p
   float m_a, m_b;     // running maxima, scaled (base-two) domain
   float z_a, z_b;     // running normalisers
   __device__ __forceinline__ void reset() {
@@ -113,16 +114,17 @@ template <int D, bool MASKED, bool UPPER>
 __device__ __forceinline__ void tile_softmax(const float (&s)[8][4], int key0, float c, RowPair& r,
                                              float (&u)[D / 8][4], uint32_t (&pa)[4][4], int quad) {
   using C = TileCfg<D, nc::kKeyTile>;
-  const bool h_a = !MASKED || key0 <= r.p_a, h_b = !MASKED || key0 <= r.p_b;
+  const bool h_a = !MASKED || (key0 <= r.p_a && key0 + nc::kKeyTile - 1 > r.lo_a);
+  const bool h_b = !MASKED || (key0 <= r.p_b && key0 + nc::kKeyTile - 1 > r.lo_b);
   float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
   for (int n = 0; n < C::NT; ++n) {
     const int j = key0 + n * 8 + 2 * quad;
-    mx_a = fmaxf(mx_a, (!MASKED || j <= r.p_a) ? s[n][0] : -INFINITY);
-    mx_a = fmaxf(mx_a, (!MASKED || j + 1 <= r.p_a) ? s[n][1] : -INFINITY);
+    mx_a = fmaxf(mx_a, (!MASKED || (j <= r.p_a && j > r.lo_a)) ? s[n][0] : -INFINITY);
+    mx_a = fmaxf(mx_a, (!MASKED || (j + 1 <= r.p_a && j + 1 > r.lo_a)) ? s[n][1] : -INFINITY);
     if (UPPER) {
-      mx_b = fmaxf(mx_b, (!MASKED || j <= r.p_b) ? s[n][2] : -INFINITY);
-      mx_b = fmaxf(mx_b, (!MASKED || j + 1 <= r.p_b) ? s[n][3] : -INFINITY);
+      mx_b = fmaxf(mx_b, (!MASKED || (j <= r.p_b && j > r.lo_b)) ? s[n][2] : -INFINITY);
+      mx_b = fmaxf(mx_b, (!MASKED || (j + 1 <= r.p_b && j + 1 > r.lo_b)) ? s[n][3] : -INFINITY);
     }
   }
   mx_a = fmaxf(mx_a, __shfl_xor_sync(kFullMask, mx_a, 1));
@@ -140,11 +142,11 @@ __device__ __forceinline__ void tile_softmax(const float (&s)[8][4], int key0, f
 #pragma unroll
   for (int n = 0; n < C::NT; ++n) {
     const int j = key0 + n * 8 + 2 * quad;
-    w_a[2 * n] = (!MASKED || j <= r.p_a) ? nc::weight(s[n][0], c, ng_a) : 0.f;
-    w_a[2 * n + 1] = (!MASKED || j + 1 <= r.p_a) ? nc::weight(s[n][1], c, ng_a) : 0.f;
+    w_a[2 * n] = (!MASKED || (j <= r.p_a && j > r.lo_a)) ? nc::weight(s[n][0], c, ng_a) : 0.f;
+    w_a[2 * n + 1] = (!MASKED || (j + 1 <= r.p_a && j + 1 > r.lo_a)) ? nc::weight(s[n][1], c, ng_a) : 0.f;
     if (UPPER) {
-      w_b[2 * n] = (!MASKED || j <= r.p_b) ? nc::weight(s[n][2], c, ng_b) : 0.f;
-      w_b[2 * n + 1] = (!MASKED || j + 1 <= r.p_b) ? nc::weight(s[n][3], c, ng_b) : 0.f;
+      w_b[2 * n] = (!MASKED || (j <= r.p_b && j > r.lo_b)) ? nc::weight(s[n][2], c, ng_b) : 0.f;
+      w_b[2 * n + 1] = (!MASKED || (j + 1 <= r.p_b && j + 1 > r.lo_b)) ? nc::weight(s[n][3], c, ng_b) : 0.f;
     } else {
       w_b[2 * n] = w_b[2 * n + 1] = 0.f;
     }
@@ -205,24 +207,31 @@ __device__ __forceinline__ void tile_softmax_dispatch(const float (&s)[8][4], in
   }
 }
 
-// Tail of a request: value rows at or beyond n_eff were not loaded or hold
-// whatever the pool had; zero them so that a zero weight times a non-finite
-// value cannot poison the row (the paper's zero-padded out-of-range loads).
-// first_bad_row: first row of the stage to clear (0 .. SK-1).
+// Value rows no real row of the group can see must not reach the PV product as
+// they are: a zero weight times a non-finite value would poison the row (the
+// paper's zero-padded out-of-range loads).  Two cases: the tail of a request
+// (rows at or beyond n_eff were not loaded, or hold whatever the pool had) and,
+// under a sliding window, the rows of the first tile that lie before the window
+// of the group's first row (their pages may have been given back by the caller).
+// Clears rows [row_begin, row_end) of the stage.
 template <int D, int SK, bool PM = false>
-__device__ __forceinline__ void zero_value_tail(uint32_t vs, int first_bad_row, int lane) {
-  const int per_half = (SK - first_bad_row) * 8;
+__device__ __forceinline__ void zero_value_rows(uint32_t vs, int row_begin, int row_end, int lane) {
+  const int per_half = (row_end - row_begin) * 8;
   const int n_chunks = per_half * (D / 64);
   for (int x = lane; x < n_chunks; x += 32) {
     const int half = x / per_half;
     const int y = x - half * per_half;
     // every 16-byte chunk of the row is cleared, so the swizzle inside the row does not matter
-    const uint32_t addr = stage_addr<D, SK, PM>(vs, first_bad_row + (y >> 3), half * 8 + (y & 7));
+    const uint32_t addr = stage_addr<D, SK, PM>(vs, row_begin + (y >> 3), half * 8 + (y & 7));
     asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
   }
   // These generic-proxy writes precede a later TMA (async-proxy) refill of the same stage.
   fence_proxy_async();
   __syncwarp();
+}
+template <int D, int SK, bool PM = false>
+__device__ __forceinline__ void zero_value_tail(uint32_t vs, int first_bad_row, int lane) {
+  zero_value_rows<D, SK, PM>(vs, first_bad_row, SK, lane);
 }
 
 // U += P V for the keys of one V stage: key chunks kc0 .. kc0 + SK/16 - 1 of the

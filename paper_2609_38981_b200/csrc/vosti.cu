@@ -89,16 +89,36 @@ struct Plan {
   int64_t n_partial_rows = 0;
 };
 
-// The plan of one request depends on its own (q_len, start) and the geometry.
-// Items are ordered longest first (by key tiles walked): split-parallel items
-// by an 8-bucket counting sort, sequential ones by a stable sort on the
-// precomputed tile count, so the order is reproducible.
+// First key a row at position p sees under a sliding window w (0: no window).
+inline int64_t first_visible_key(int64_t p, int64_t w) { return (w > 0 && p - w + 1 > 0) ? p - w + 1 : 0; }
+
+// The plan of one request depends on its own (q_len, start), the window and the
+// geometry.  A split-parallel item is one (16-row group, split) pair whose keys
+// some row of the group sees: splits from the one holding the first visible key
+// of the group's first row to the one holding the last row's position.  Items
+// are ordered longest first (by key tiles walked): split-parallel items by an
+// 8-bucket counting sort, sequential ones by a stable sort on the precomputed
+// tile count, so the order is reproducible.
 vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const int32_t* start_pos,
-                           const int32_t* seq_lens, int32_t batch, Plan* plan, int64_t* part_base) {
-  if (batch < 0 || (batch > 0 && (!q_lens || !start_pos || !seq_lens))) return VOSTI_ERR_INVALID_ARG;
+                           const int32_t* seq_lens, int32_t batch, int32_t window, Plan* plan,
+                           int64_t* part_base) {
+  if (batch < 0 || window < 0 || (batch > 0 && (!q_lens || !start_pos || !seq_lens))) return VOSTI_ERR_INVALID_ARG;
   if (batch > c.max_batch) return VOSTI_ERR_OUT_OF_RANGE;
   const int G = c.n_q_heads / c.n_kv_heads;
   constexpr int TPS = nc::kTilesPerSplit;
+  constexpr int kGroupsMax = nc::kSplitRowsMax / nc::kRowsPerGroup;
+  // key tiles [t0, t1) a row group walks, and how many of them fall into split k
+  struct Span {
+    int64_t t0, t1;
+    int64_t k0() const { return t0 / TPS; }
+    int64_t k1() const { return (t1 + TPS - 1) / TPS; }
+    int64_t tiles_in(int64_t k) const { return std::min(t1, (k + 1) * TPS) - std::max(t0, k * TPS); }
+  };
+  auto span_of = [&](int64_t st, int64_t q, int64_t first_row, int64_t n_rows) -> Span {
+    const int64_t first_tok = first_row / G;
+    const int64_t last_tok = std::min<int64_t>(q - 1, (first_row + n_rows - 1) / G);
+    return Span{first_visible_key(st + first_tok, window) / nc::kKeyTile, (st + last_tok) / nc::kKeyTile + 1};
+  };
   int64_t total_q = 0, n_split = 0, n_seq = 0, part_rows = 0;
   int64_t bucket[TPS + 1] = {0};  // bucket[t] = split items that walk t tiles
   // pass 1: premises, counts
@@ -111,14 +131,17 @@ vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const i
     const int64_t groups = (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
     if (rows <= nc::kSplitRowsMax) {
       if (part_base) part_base[r] = part_rows;
-      part_rows += int64_t{c.n_kv_heads} * ((st + q - 1) / nc::kSplitLen + 1) * rows;
+      const int64_t first_split = first_visible_key(st, window) / nc::kSplitLen;
+      part_rows += int64_t{c.n_kv_heads} * ((st + q - 1) / nc::kSplitLen + 1 - first_split) * rows;
       for (int64_t g = 0; g < groups; ++g) {
-        const int64_t last_tok = std::min<int64_t>(q - 1, (g * nc::kRowsPerGroup + 15) / G);
-        const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
-        const int64_t k_g = (tiles + TPS - 1) / TPS;
-        bucket[TPS] += k_g - 1;
-        bucket[tiles - (k_g - 1) * TPS] += 1;
-        n_split += k_g;
+        const Span sp = span_of(st, q, g * nc::kRowsPerGroup, nc::kRowsPerGroup);
+        const int64_t k0 = sp.k0(), k1 = sp.k1();
+        bucket[sp.tiles_in(k0)] += 1;
+        if (k1 - k0 >= 2) {
+          bucket[sp.tiles_in(k1 - 1)] += 1;
+          bucket[TPS] += k1 - k0 - 2;
+        }
+        n_split += k1 - k0;
       }
     } else {
       if (part_base) part_base[r] = 0;
@@ -143,33 +166,30 @@ vosti_status plan_requests(const vosti_config& c, const int32_t* q_lens, const i
     if (q == 0) continue;
     const int64_t rows = q * G;
     const bool split_parallel = rows <= nc::kSplitRowsMax;
-    // split-parallel requests: one item per (16-row group, split); others: one per 128-row tile
+    // split-parallel requests: one item per (16-row group, split); others: one per 256-row tile
     const int64_t rows_per_item = split_parallel ? nc::kRowsPerGroup : kTileRows;
     const int n_row_items = static_cast<int>((rows + rows_per_item - 1) / rows_per_item);
     if (split_parallel) {
       // Split outermost, row group innermost: the (at most two) row groups that read the
       // same split get neighbouring tickets, run at about the same time on different SMs,
       // and the second read of the split's K/V is served by L2 instead of HBM.
-      int64_t tiles_g[nc::kSplitRowsMax / nc::kRowsPerGroup];
-      int k_max = 0;
+      Span sp[kGroupsMax];
+      int64_t k_lo = INT64_MAX, k_hi = 0;
       for (int x = 0; x < n_row_items; ++x) {
-        const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
-        tiles_g[x] = (st + last_tok) / nc::kKeyTile + 1;
-        k_max = std::max(k_max, static_cast<int>((tiles_g[x] + TPS - 1) / TPS));
+        sp[x] = span_of(st, q, int64_t{x} * rows_per_item, rows_per_item);
+        k_lo = std::min(k_lo, sp[x].k0());
+        k_hi = std::max(k_hi, sp[x].k1());
       }
-      for (int k = 0; k < k_max; ++k)
-        for (int x = 0; x < n_row_items; ++x) {
-          const int k_g = static_cast<int>((tiles_g[x] + TPS - 1) / TPS);
-          if (k + 1 < k_g) out[at[TPS]++] = {r, x, k, k + 1};
-          else if (k + 1 == k_g) out[at[tiles_g[x] - int64_t{k_g - 1} * TPS]++] = {r, x, k, k + 1};
-        }
+      for (int64_t k = k_lo; k < k_hi; ++k)
+        for (int x = 0; x < n_row_items; ++x)
+          if (k >= sp[x].k0() && k < sp[x].k1())
+            out[at[sp[x].tiles_in(k)]++] = {r, x, static_cast<int32_t>(k), static_cast<int32_t>(k + 1)};
     } else {
       for (int x = 0; x < n_row_items; ++x) {
-        const int64_t last_tok = std::min<int64_t>(q - 1, (int64_t{x} * rows_per_item + rows_per_item - 1) / G);
-        const int64_t tiles = (st + last_tok) / nc::kKeyTile + 1;
-        const int k_g = static_cast<int>((tiles + TPS - 1) / TPS);
+        const Span sp = span_of(st, q, int64_t{x} * rows_per_item, rows_per_item);
         const int first_group = x * (kTileRows / nc::kRowsPerGroup);
-        plan->seq_scratch.push_back({tiles, vosti_work_item{r, first_group, 0, k_g}});
+        plan->seq_scratch.push_back({sp.t1 - sp.t0, vosti_work_item{r, first_group, static_cast<int32_t>(sp.k0()),
+                                                                    static_cast<int32_t>(sp.k1())}});
       }
     }
   }
@@ -426,10 +446,17 @@ size_t vosti_workspace_bytes(const vosti_config* config) {
 vosti_status vosti_plan(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
                         const int32_t* seq_lens, int32_t batch, vosti_work_item* items, int64_t cap,
                         int64_t* n_items, int64_t* n_split, int64_t* n_partial_rows) {
+  return vosti_plan_ex(config, q_lens, start_pos, seq_lens, batch, 0, items, cap, n_items, n_split,
+                       n_partial_rows);
+}
+
+vosti_status vosti_plan_ex(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
+                           const int32_t* seq_lens, int32_t batch, int32_t window, vosti_work_item* items,
+                           int64_t cap, int64_t* n_items, int64_t* n_split, int64_t* n_partial_rows) {
   if (!config || cap < 0 || (cap > 0 && !items)) return VOSTI_ERR_INVALID_ARG;
   if (!geometry_ok(*config)) return VOSTI_ERR_UNSUPPORTED_CONFIG;
   Plan plan;
-  const vosti_status st = plan_requests(*config, q_lens, start_pos, seq_lens, batch, &plan, nullptr);
+  const vosti_status st = plan_requests(*config, q_lens, start_pos, seq_lens, batch, window, &plan, nullptr);
   if (st != VOSTI_OK) return st;
   const int64_t n = static_cast<int64_t>(plan.items.size());
   for (int64_t i = 0; i < std::min(n, cap); ++i) items[i] = plan.items[i];
@@ -567,18 +594,27 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
                                    const int32_t* start_pos, const int32_t* seq_lens,
                                    const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
                                    float softmax_scale, void* cuda_stream) {
-  if (!ctx || batch < 0 || block_table_stride < 0) return VOSTI_ERR_INVALID_ARG;
+  return vosti_paged_attention_ex(ctx, q, out, nullptr, q_lens, start_pos, seq_lens, block_tables,
+                                  block_table_stride, batch, softmax_scale, 0, cuda_stream);
+}
+
+vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, float* lse, const int32_t* q_lens,
+                                      const int32_t* start_pos, const int32_t* seq_lens,
+                                      const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
+                                      float softmax_scale, int32_t window, void* cuda_stream) {
+  if (!ctx || batch < 0 || block_table_stride < 0 || window < 0) return VOSTI_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
   if (batch > 0 && !block_tables) return VOSTI_ERR_INVALID_ARG;
   const vosti_config& c = ctx->cfg;
   Plan& plan = ctx->plan;
   std::vector<int64_t>& part_base = ctx->part_base;
   part_base.resize(static_cast<size_t>(std::max(batch, 0)));
-  vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, &plan, part_base.data());
+  vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, window, &plan, part_base.data());
   if (st != VOSTI_OK) return st;
   if (plan.items.empty()) return VOSTI_OK;
   if (!q || !out) return VOSTI_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16) return VOSTI_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(lse) % 4) return VOSTI_ERR_INVALID_ARG;
   if (static_cast<int64_t>(plan.items.size()) > ctx->lim.items_max ||
       plan.n_partial_rows > ctx->lim.part_rows_max)
     return VOSTI_ERR_WORKSPACE;
@@ -611,6 +647,8 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
     m.n_pages = 0;
     m.bt_off = static_cast<int32_t>(bt_used);
     m.n_splits = 0;
+    m.first_split = 0;
+    m.pad = 0;
     m.part_base = part_base[r];
     row0 += q_lens[r];
     if (q_lens[r] == 0) continue;
@@ -620,14 +658,21 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
         (int64_t{seq_lens[r]} + c.page_size - 1) / c.page_size > block_table_stride)
       return VOSTI_ERR_OUT_OF_RANGE;
     const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
-    for (int64_t b = 0; b < n_pages; ++b) {
+    // Pages that lie wholly before the window of the request's first row are never
+    // visible: their table entries are not read (the caller may have freed them);
+    // page 0 stands in where a tile load still covers them.
+    const int64_t first_key = first_visible_key(start_pos[r], window);
+    const int64_t first_page = first_key / c.page_size;
+    for (int64_t b = 0; b < first_page; ++b) bt_flat[bt_used + b] = 0;
+    for (int64_t b = first_page; b < n_pages; ++b) {
       const int32_t page = row[b];
       if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
       bt_flat[bt_used + b] = page;
     }
     bt_used += n_pages;
     m.n_pages = static_cast<int32_t>(n_pages);
-    m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1);
+    m.first_split = static_cast<int32_t>(first_key / nc::kSplitLen);
+    m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1) - m.first_split;
     if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
   }
   at += align_up(sizeof(int32_t) * bt_used, 16);
@@ -645,7 +690,7 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
     si.n_splits = m.n_splits;
     si.part_base = m.part_base;
     si.req = it.req;
-    si.pad = 0;
+    si.first_split = m.first_split;
   }
   const size_t off_tok = at;
   int2* toks = reinterpret_cast<int2*>(blob + at);
@@ -682,6 +727,8 @@ vosti_status vosti_paged_attention(vosti_ctx* ctx, const void* q, void* out, con
   p.Hkv = c.n_kv_heads;
   p.G = G;
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
+  p.window = window;
+  p.lse = lse;
   st = c.head_dim == 128 ? launch_attention<128>(ctx, p, plan.n_split, n_seq, stream)
                          : launch_attention<64>(ctx, p, plan.n_split, n_seq, stream);
   if (st != VOSTI_OK) return st;

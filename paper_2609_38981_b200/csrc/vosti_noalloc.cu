@@ -143,6 +143,8 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
     m.n_pages = 0;
     m.bt_off = static_cast<int32_t>(bt_used);
     m.n_splits = 0;
+    m.first_split = 0;
+    m.pad = 0;
     m.part_base = part_rows;
     row0 += ql;
     if (ql == 0) continue;
@@ -173,7 +175,7 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
         si.q_row0 = m.q_row0; si.q_len = m.q_len; si.start = m.start; si.n_pages = m.n_pages;
         si.bt_index = m.bt_off + k * nc::kPagesPerSplit;
         si.split = k; si.row_group = g; si.n_splits = m.n_splits;
-        si.part_base = m.part_base; si.req = r; si.pad = 0;
+        si.part_base = m.part_base; si.req = r; si.first_split = 0;
       }
     }
     for (int i = 0; i < ql; ++i) toks[n_tok++] = make_int2(r, i);
@@ -231,5 +233,7 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
   p.Hkv = n_kv_heads;
   p.G = G;
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
+  p.window = 0;
+  p.lse = nullptr;
   return head_dim == 128 ? launch<128>(map, p, sm_count, stream) : launch<64>(map, p, sm_count, stream);
 }

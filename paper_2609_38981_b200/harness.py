@@ -67,6 +67,20 @@ class DeviceCache:
                                  scale, stream=stream)
         return out
 
+    def attend_ex(self, q: torch.Tensor, q_lens, start_pos, seq_lens, block_tables, scale: float,
+                  window: int = 0, want_lse: bool = False, stream=None):
+        """Attention with a sliding window and / or the log-sum-exp output.
+        Returns (out, lse) with lse an fp32 [T, Hq] tensor or None."""
+        qd = q.to(self.device).contiguous()
+        out = torch.empty_like(qd)
+        _as_i16(out).fill_(0x7FC1)
+        lse = None
+        if want_lse:
+            lse = torch.full(qd.shape[:2], float("nan"), dtype=torch.float32, device=self.device)
+        vb.vosti_paged_attention_ex(self.ctx, qd, out, lse, q_lens, start_pos, seq_lens, block_tables,
+                                    scale, window=window, stream=stream)
+        return out, lse
+
     def upload(self, reqs: Sequence[RequestContent], tables: Sequence[Sequence[int]],
                upto: Optional[Sequence[int]] = None) -> None:
         """Write positions [0, upto_r) of every request into the pool through

@@ -15,13 +15,23 @@ Call = List[Tuple[int, int, int]]          # (request index, start position, q_l
 
 
 def run_schedule(cache: DeviceCache, reqs, tables, schedule: Sequence[Call], scale: float,
-                 stride=None, fill=-1, append=True, seq_lens_override=None) -> Dict[int, torch.Tensor]:
+                 stride=None, fill=-1, append=True, seq_lens_override=None, window=None,
+                 lse_out=None, drop_pages_before_window=False) -> Dict[int, torch.Tensor]:
     """Each call appends its tokens then attends.  Returns, per request, an int16
     tensor [n, Hq, d] with the bf16 bits of every computed row (rows never
-    computed stay at a sentinel)."""
+    computed stay at a sentinel).
+
+    window: None = the plain entry point; an int = the extended one with that
+    sliding window.  lse_out: a dict that receives, per request, an int32 tensor
+    [n, Hq] with the fp32 bits of the log-sum-exp.  drop_pages_before_window:
+    replace the block-table entries the extended entry point promises not to
+    read by -1."""
     geo = cache.geo
     outs = {i: torch.full((r.n, geo.n_q_heads, geo.head_dim), 0x7FC2, dtype=torch.int16)
             for i, r in enumerate(reqs)}
+    if lse_out is not None:
+        for i, r in enumerate(reqs):
+            lse_out.setdefault(i, torch.full((r.n, geo.n_q_heads), 0x7FC00002, dtype=torch.int32))
     for call in schedule:
         idx = [i for i, _, _ in call]
         starts = [s for _, s, _ in call]
@@ -34,10 +44,25 @@ def run_schedule(cache: DeviceCache, reqs, tables, schedule: Sequence[Call], sca
         seq = [s + q for s, q in zip(starts, qls)] if seq_lens_override is None else \
             [seq_lens_override[i] for i in idx]
         qt = torch.cat([reqs[i].q_rows(s, q) for i, s, q in call])
-        out = bf16_bits(cache.attend(qt, qls, starts, seq, bt, scale))
+        if window is None and lse_out is None:
+            out = bf16_bits(cache.attend(qt, qls, starts, seq, bt, scale))
+            lse = None
+        else:
+            bt_call = bt
+            if drop_pages_before_window and window:
+                bt_call = bt.copy()
+                for row, s in enumerate(starts):
+                    bt_call[row, :max(0, s - window + 1) // geo.page_size] = -1
+            o, lse = cache.attend_ex(qt, qls, starts, seq, bt_call, scale, window=window or 0,
+                                     want_lse=lse_out is not None)
+            out = bf16_bits(o)
+            if lse is not None:
+                lse = lse.cpu().view(torch.int32)
         at = 0
         for i, s, q in call:
             outs[i][s:s + q] = out[at:at + q]
+            if lse is not None:
+                lse_out[i][s:s + q] = lse[at:at + q]
             at += q
     return outs
 
@@ -89,7 +114,7 @@ def compact_host_pool(w):
     return pool, inputs.block_table_array(tables)
 
 
-def sampled_parity(w, out_bits, n_samples, seed=0):
+def sampled_parity(w, out_bits, n_samples, seed=0, window=0):
     """Compare `n_samples` random (request, token, head) outputs of a workload's
     call against the oracle's paged front-end.  out_bits: int16 [T, Hq, d]."""
     from oracle import oracle
@@ -103,7 +128,7 @@ def sampled_parity(w, out_bits, n_samples, seed=0):
     sel = np.array(sel, dtype=np.int32)
     ref = oracle.paged_attention(inputs.bits(w.packed_q()), pool, w.q_lens, w.start_pos, w.seq_lens,
                                  bt, n_kv_heads=geo.n_kv_heads, page_size=geo.page_size,
-                                 scale=geo.head_dim ** -0.5, sel=sel)
+                                 scale=geo.head_dim ** -0.5, sel=sel, window=window)
     row0 = np.concatenate([[0], np.cumsum(w.q_lens)])
     got = np.stack([widen_bits(out_bits[row0[r] + i, h]) for r, i, h in sel])
     err = np.abs(got - ref)

@@ -113,6 +113,44 @@ def test_plan_shapes(vb):
     assert plan_of_request(vb, c, 1, 512)[0] == [(0, 0, 1), (0, 1, 2)]
 
 
+def test_plan_under_a_sliding_window(vb):
+    """Items only for the splits that hold a key some row of the group sees; the first
+    visible key of a row at p is max(0, p - w + 1)."""
+    c = cfg(vb)          # G = 4, 8 kv heads
+
+    def plan_w(q, s, w):
+        items, n_split, n_part = vb.vosti_plan_ex(c, [q], [s], [s + q], w)
+        return list(map(tuple, items[:, 1:])), n_split, n_part
+
+    # window 0 and a window longer than the context: the unwindowed plan
+    for q, s in ((1, 1300), (8, 508), (9, 1020), (100, 500)):
+        base = vb.vosti_plan(c, [q], [s], [s + q])
+        for w in (0, s + q, 10 ** 6):
+            got = vb.vosti_plan_ex(c, [q], [s], [s + q], w)
+            assert (got[0] == base[0]).all() and got[1:] == base[1:]
+    # decode at p = 1300, w = 100: keys 1201..1300, all in split 2
+    assert plan_w(1, 1300, 100) == ([(0, 2, 3)], 1, 8 * 1 * 4)
+    # p = 1030, w = 100: keys 931..1030 -> tiles 14, 15 of split 1 and tile 16 of split 2 (longest first)
+    assert plan_w(1, 1030, 100) == ([(0, 1, 2), (0, 2, 3)], 2, 8 * 2 * 4)
+    # w = 1: only the key at p
+    assert plan_w(1, 1024, 1) == ([(0, 2, 3)], 1, 8 * 4)
+    assert plan_w(1, 1023, 1) == ([(0, 1, 2)], 1, 8 * 4)
+    # 8 tokens at 508..515, w = 4: group 0 (tokens 0..3, keys 505..511) split 0 only;
+    # group 1 (tokens 4..7, keys 509..515) splits 0 and 1; partial rows from split 0
+    items, n_split, n_part = plan_w(8, 508, 4)
+    assert sorted(items) == [(0, 0, 1), (1, 0, 1), (1, 1, 2)] and n_part == 8 * 2 * 32
+    # the same tokens at 1020..1027, w = 4: the request's first split is 1, so two splits of partial rows
+    items, n_split, n_part = plan_w(8, 1020, 4)
+    assert sorted(items) == [(0, 1, 2), (1, 1, 2), (1, 2, 3)] and n_part == 8 * 2 * 32
+    # a tile item reports the splits it walks: 100 tokens at 2000, w = 600 -> rows 0..255 are tokens
+    # 0..63 (keys 1401..2063: splits 2..4), rows 256..399 tokens 64..99 (keys 1465..2099: splits 2..4)
+    items, n_split, n_part = plan_w(100, 2000, 600)
+    assert n_split == 0 and n_part == 0 and items == [(0, 2, 5), (16, 2, 5)]
+    with pytest.raises(vb.VostiError) as e:
+        vb.vosti_plan_ex(c, [1], [0], [1], -1)
+    assert e.value.status == vb.VOSTI_ERR_INVALID_ARG
+
+
 def test_items_are_ordered_longest_first(vb):
     c = cfg(vb)
     items, n_split, _ = vb.vosti_plan(c, [1, 1, 1], [100, 4000, 700], [101, 4001, 701])
