@@ -14,13 +14,22 @@
 // sums for the same chunk order (measured on B200), which is what lets this
 // kernel and the warp-MMA kernels agree bit for bit.
 //
-// A CTA holds TWO 128-row tiles (X = 0, 1) that share every staged K/V tile:
-// the softmax work of one overlaps the waits of the other on every scheduler,
-// and K/V is fetched through L2 once per 256 rows.
-// Roles (352 threads): warps 0-3 = softmax / correction of tile 0, warps 4-7 of
-// tile 1, one thread per row; warp 9 = MMA issuer (one elected thread); warps 8
-// and 10 = TMA producers for K and for V (a TMA instruction occupies its issuing
-// warp for about a hundred cycles per 2 KB box).
+// A CTA holds TWO 128-row tiles (X = 0, 1) that share every staged K/V tile, so
+// K/V is fetched through L2 once per 256 rows.  Work on a row is divided between
+// two threads so that neither chain is long:
+//   * a softmax thread reads the row's 64 scores, applies the scalar rules
+//     (maximum, alpha, exponentials, pinned row sum), publishes alpha and writes
+//     the bf16 weights over the scores;
+//   * a correction thread takes alpha and rescales the row's U accumulator when
+//     some alpha of its warp is not 1, zero-fills value rows no query row may
+//     see, and at the end of every split folds the split into the running
+//     result (and, at the end of the row, normalises and stores it).
+// Roles by warpgroup (640 threads): 0 / 1 = softmax of tile 0 / 1, 2 / 3 =
+// correction of tile 0 / 1, 4 = { K producer, MMA issuer of tile 0, V producer,
+// MMA issuer of tile 1 }.  Registers are moved from warpgroup 4 to the others
+// with setmaxnreg.  Each tile has its own issuer thread: the MMAs of one thread
+// run in issue order, which the aliasing of weights over scores relies on, and
+// the two tiles never wait for each other.
 // Tensor memory (512 columns): per tile S x2 (64 each; the bf16 weights P are
 // written over the first 32 columns of the S buffer they were computed from)
 // and U (D).  The running fold U_c lives in global memory (per CTA and tile a
@@ -36,17 +45,32 @@ template <int D>
 struct TileKernelCfg {
   static constexpr int kRows = 256;                          // rows of a work item: two tiles
   static constexpr int kTileRows = 128;
-  static constexpr int kThreads = 352;
+  static constexpr int kThreads = 640;
   static constexpr int kStages = 3;                          // K+V tile pairs in flight
   static constexpr int kQBytes = kRows * D * 2;              // [half][row][128 B]
   static constexpr int kKBytes = nc::kKeyTile * D * 2;       // [half][key][128 B]
   static constexpr int kStageBytes = 2 * kKBytes;            // K then V
+  static constexpr int kAlphaBytes = 2 * 2 * kTileRows * 4;  // alpha[tile][buffer][row]
+  static constexpr int kMzBytes = 2 * 2 * kTileRows * 8;     // (m, z)[tile][split parity][row]
   static constexpr int kBarBytes = 512;
-  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kBarBytes + 1024;
+  static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kAlphaBytes + kMzBytes + kBarBytes + 1024;
+  // Registers per thread after the roles have split.  The total must not exceed what the CTA
+  // was given at launch (640 threads x 96 registers): a warpgroup asking for more than the
+  // others have released waits for ever.
+  static constexpr int kRegsSoftmax = 120;
+  static constexpr int kRegsCorrection = 104;
+  static constexpr int kRegsOther = 32;
+  static constexpr int kRegsAfterSplit = 32 * (8 * kRegsSoftmax + 8 * kRegsCorrection + 4 * kRegsOther);
+  static_assert(kRegsAfterSplit <= kThreads * 96, "register split exceeds the launch allocation");
   // tensor-memory columns
   static constexpr uint32_t kColS = 0;    // tile X, buffer b: S / P at 128 X + 64 b
   static constexpr uint32_t kColU = 256;  // tile X: U at 256 + D X
 };
+
+template <int N>
+__device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
 // ---- tcgen05 wrappers ---------------------------------------------------------------
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -129,13 +153,19 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t q_smem = base;  // tile X at X * TR * D * 2
   const uint32_t kv_smem = base + Cfg::kQBytes;
-  const uint32_t bars = kv_smem + NS * Cfg::kStageBytes;
-  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 448);
-  // barrier map (8 bytes each); per tile X and S buffer b: index 2 X + b
+  constexpr int kXchgOff = Cfg::kQBytes + NS * Cfg::kStageBytes;
+  float* alpha_s = reinterpret_cast<float*>(sbase + kXchgOff);                      // [X][b][row]
+  float2* mz_s = reinterpret_cast<float2*>(sbase + kXchgOff + Cfg::kAlphaBytes);     // [X][kb][row]
+  constexpr int kBarOff = kXchgOff + Cfg::kAlphaBytes + Cfg::kMzBytes;
+  const uint32_t bars = base + kBarOff;
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + kBarOff + 448);
+  // barrier map (8 bytes each); per tile X and buffer b: index 2 X + b
   const uint32_t k_full = bars, v_full = bars + 8 * NS, k_empty = bars + 16 * NS, v_empty = bars + 24 * NS;
   const uint32_t s_full = bars + 32 * NS, p_full = s_full + 32, pv_done = s_full + 64;
+  const uint32_t a_full = s_full + 96, mz_full = s_full + 128;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int wg = warp >> 2;
 
   const vosti_work_item item = P.items[blockIdx.x / P.Hkv];
   const int kvh = blockIdx.x % P.Hkv;
@@ -164,13 +194,15 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     for (int i = 0; i < NS; ++i) {
       mbar_init(k_full + 8 * i, 1);
       mbar_init(v_full + 8 * i, 1);
-      mbar_init(k_empty + 8 * i, 1);
-      mbar_init(v_empty + 8 * i, 1);
+      mbar_init(k_empty + 8 * i, 2);  // both issuers release a stage
+      mbar_init(v_empty + 8 * i, 2);
     }
     for (int i = 0; i < 4; ++i) {
       mbar_init(s_full + 8 * i, 1);
-      mbar_init(p_full + 8 * i, TR);
+      mbar_init(p_full + 8 * i, 2 * TR);  // softmax and correction thread of every row
       mbar_init(pv_done + 8 * i, 1);
+      mbar_init(a_full + 8 * i, TR);
+      mbar_init(mz_full + 8 * i, TR);
     }
     flags[0] = 0u;  // abort flag
     mbar_fence_init();
@@ -201,7 +233,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + Cfg::kQBytes + NS * Cfg::kStageBytes + 456);
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + kBarOff + 456);
 
   // Bounded wait shared by all roles: gives up after ~1 s or as soon as another
   // thread of the CTA has given up, records the failure, and lets the caller
@@ -222,125 +254,124 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     }
   };
 
-  if (warp == 8 || warp == 10) {
-    // ================= TMA producers: warp 8 loads the K tiles, warp 10 the V tiles =======
-    griddep_wait();
-    const int is_v = warp == 10;
-    const int32_t* bt = P.bt_flat + rq.bt_off;
-    auto fetch_pages = [&](int split) -> int {
-      const int pg = split * nc::kPagesPerSplit + lane;
-      return pg < rq.n_pages ? __ldg(bt + pg) : -1;
-    };
-    int pages_even = -1, pages_odd = -1;
-    if ((T0 / TPS) & 1) pages_odd = fetch_pages(T0 / TPS); else pages_even = fetch_pages(T0 / TPS);
-    bool ok = true;
-    for (int t = T0; t < n_tiles && ok; ++t) {
-      const int s = (t - T0) % NS, use = (t - T0) / NS;
-      const int split = t / TPS, tl = t - split * TPS;
-      if ((tl == TPS / 2 || (t == T0 && tl > TPS / 2)) && (split + 1) * TPS < n_tiles) {
-        const int ids = fetch_pages(split + 1);
-        if ((split + 1) & 1) pages_odd = ids; else pages_even = ids;
+  if (wg == 4) {
+    reg_dealloc<Cfg::kRegsOther>();
+    if (warp == 16 || warp == 18) {
+      // ================= TMA producers: warp 16 loads the K tiles, warp 18 the V tiles =======
+      griddep_wait();
+      const int is_v = warp == 18;
+      const int32_t* bt = P.bt_flat + rq.bt_off;
+      auto fetch_pages = [&](int split) -> int {
+        const int pg = split * nc::kPagesPerSplit + lane;
+        return pg < rq.n_pages ? __ldg(bt + pg) : -1;
+      };
+      int pages_even = -1, pages_odd = -1;
+      if ((T0 / TPS) & 1) pages_odd = fetch_pages(T0 / TPS); else pages_even = fetch_pages(T0 / TPS);
+      bool ok = true;
+      for (int t = T0; t < n_tiles && ok; ++t) {
+        const int s = (t - T0) % NS, use = (t - T0) / NS;
+        const int split = t / TPS, tl = t - split * TPS;
+        if ((tl == TPS / 2 || (t == T0 && tl > TPS / 2)) && (split + 1) * TPS < n_tiles) {
+          const int ids = fetch_pages(split + 1);
+          if ((split + 1) & 1) pages_odd = ids; else pages_even = ids;
+        }
+        const int ids = (split & 1) ? pages_odd : pages_even;
+        const int n_valid = min(nc::kPagesPerTile, rq.n_pages - t * nc::kPagesPerTile);
+        const uint32_t dst = kv_smem + s * Cfg::kStageBytes + is_v * Cfg::kKBytes;
+        const uint32_t full = (is_v ? v_full : k_full) + 8 * s;
+        const uint32_t empty = (is_v ? v_empty : k_empty) + 8 * s;
+        if (use > 0) ok = __all_sync(kFullMask, wait(empty, (use - 1) & 1));
+        if (!ok) break;
+        issue_stage_load<D, KT>(&kv_map, dst, full, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, is_v, lane);
       }
-      const int ids = (split & 1) ? pages_odd : pages_even;
-      const int n_valid = min(nc::kPagesPerTile, rq.n_pages - t * nc::kPagesPerTile);
-      const uint32_t dst = kv_smem + s * Cfg::kStageBytes + is_v * Cfg::kKBytes;
-      const uint32_t full = (is_v ? v_full : k_full) + 8 * s;
-      const uint32_t empty = (is_v ? v_empty : k_empty) + 8 * s;
-      if (use > 0) ok = __all_sync(kFullMask, wait(empty, (use - 1) & 1));
-      if (!ok) break;
-      issue_stage_load<D, KT>(&kv_map, dst, full, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, is_v, lane);
-    }
-  } else if (warp == 9) {
-    // ================= MMA issuer ====================================================
-    // One thread's MMAs run in issue order.  S of key tile t+2 overwrites the buffer whose
-    // first columns PV of key tile t reads its weights from, so it is issued after that PV.
-    if (lane == 0) {
+    } else if (lane == 0) {
+      // ================= MMA issuers: warp 17 for tile 0, warp 19 for tile 1 ==================
+      // One thread's MMAs run in issue order.  S of key tile t+2 overwrites the buffer whose
+      // first columns PV of key tile t reads its weights from, so it is issued after that PV.
+      const int X = (warp - 17) >> 1;
+      const int my_tiles = n_tiles_x[X];
       constexpr uint32_t idesc_s = umma_idesc(128, KT, false);
       constexpr uint32_t idesc_pv = umma_idesc(128, D, true);
+      const uint32_t qx = q_smem + X * (TR * D * 2);
       bool ok = true;
-      auto issue_s = [&](int t) {  // S of both tiles for key tile t
+      auto issue_s = [&](int t) {
         const int i = t - T0, s = i % NS, b = i & 1;
         ok = ok && wait(k_full + 8 * s, (i / NS) & 1);
         if (!ok) return;
         tc_fence_after();
         const uint32_t kst = kv_smem + s * Cfg::kStageBytes;
 #pragma unroll
-        for (int X = 0; X < 2; ++X) {
-          if (t >= n_tiles_x[X]) continue;
-          const uint32_t qx = q_smem + X * (TR * D * 2);
-#pragma unroll
-          for (int kc = 0; kc < D / 16; ++kc) {
-            const uint64_t da = smem_desc_sw128(qx + (kc >> 2) * (TR * 128) + (kc & 3) * 32, 16, 1024);
-            const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
-            tc_mma_ss(tmem + Cfg::kColS + X * 128 + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
-          }
-          tc_commit(s_full + 8 * (2 * X + b));
+        for (int kc = 0; kc < D / 16; ++kc) {
+          const uint64_t da = smem_desc_sw128(qx + (kc >> 2) * (TR * 128) + (kc & 3) * 32, 16, 1024);
+          const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
+          tc_mma_ss(tmem + Cfg::kColS + X * 128 + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
         }
+        tc_commit(s_full + 8 * (2 * X + b));
         tc_commit(k_empty + 8 * s);
       };
-      issue_s(T0);
-      for (int t = T0; t < n_tiles && ok; ++t) {
-        if (t + 1 < n_tiles) issue_s(t + 1);
+      if (T0 < my_tiles) issue_s(T0);
+      for (int t = T0; t < my_tiles && ok; ++t) {
+        if (t + 1 < my_tiles) issue_s(t + 1);
         if (!ok) break;
         const int i = t - T0, s = i % NS, b = i & 1;
         ok = wait(v_full + 8 * s, (i / NS) & 1);
-#pragma unroll
-        for (int X = 0; X < 2; ++X) {
-          if (!ok || t >= n_tiles_x[X]) continue;
-          ok = wait(p_full + 8 * (2 * X + b), (i >> 1) & 1);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
-#pragma unroll
-          for (int kc = 0; kc < KT / 16; ++kc) {
-            // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
-            const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
-            // a split (and the first tile walked) starts from a fresh accumulator
-            const uint32_t acc = (kc > 0 || ((t % TPS) != 0 && t != T0)) ? 1u : 0u;
-            tc_mma_ts(tmem + Cfg::kColU + X * D, tmem + Cfg::kColS + X * 128 + b * KT + kc * 8, db, idesc_pv, acc);
-          }
-          tc_commit(pv_done + 8 * (2 * X + b));
-        }
         if (!ok) break;
+        ok = wait(p_full + 8 * (2 * X + b), (i >> 1) & 1);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
+#pragma unroll
+        for (int kc = 0; kc < KT / 16; ++kc) {
+          // B = V: MN-major, 64-element halves of d KT*128 bytes apart, 8-key groups 1024 bytes apart
+          const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
+          // a split (and the first tile walked) starts from a fresh accumulator
+          const uint32_t acc = (kc > 0 || ((t % TPS) != 0 && t != T0)) ? 1u : 0u;
+          tc_mma_ts(tmem + Cfg::kColU + X * D, tmem + Cfg::kColS + X * 128 + b * KT + kc * 8, db, idesc_pv, acc);
+        }
+        tc_commit(pv_done + 8 * (2 * X + b));
         tc_commit(v_empty + 8 * s);
       }
+      // Key tiles only the other tile walks: hand the stages back unused, each after it has
+      // been filled (so that an arrival can never count towards an earlier use of the stage).
+      for (int t = max(my_tiles, T0); t < n_tiles && ok; ++t) {
+        const int i = t - T0, s = i % NS;
+        ok = wait(k_full + 8 * s, (i / NS) & 1);
+        if (!ok) break;
+        mbar_arrive(k_empty + 8 * s);
+        ok = wait(v_full + 8 * s, (i / NS) & 1);
+        if (!ok) break;
+        mbar_arrive(v_empty + 8 * s);
+      }
     }
-  } else if (warp < 8) {
-    // ================= softmax / correction: one thread per row ======================
-    const int X = warp >> 2;                    // which 128-row tile
+  } else if (wg < 2) {
+    // ================= softmax: one thread per row =======================================
+    reg_alloc<Cfg::kRegsSoftmax>();
+    const int X = wg;                           // which 128-row tile
     const int r = tid & (TR - 1);               // row of the tile = tensor-memory lane
     const int row = row0 + X * TR + r;
     const bool valid = row < rows;
-    const int tok = row / G;
-    const int p = valid ? rq.start + tok : -1;  // padding rows see nothing
-    const int lo = nc::window_lo(p, P.window);  // key j is visible iff lo < j <= p
-    // first split the row sees; before it (and in the first split the CTA walks) the
-    // running result is simply taken from the split, as the fold of the split kernels does
-    const int k_first = max(nc::first_key(p, P.window) / nc::kSplitLen, T0 / TPS);
+    const int p = valid ? rq.start + row / G : -1;  // padding rows see nothing
+    const int lo = nc::window_lo(p, P.window);      // key j is visible iff lo < j <= p
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t col_s = Cfg::kColS + X * 128, col_u = Cfg::kColU + X * D;
+    const uint32_t col_s = Cfg::kColS + X * 128;
     const int my_tiles = n_tiles_x[X];
     const float c = P.c;
-    // running fold of this tile in global memory ([D/4][128] float4: this thread owns column r),
-    // and the row's place in the output
-    float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + (static_cast<size_t>(blockIdx.x) * 2 + X) * (D / 4) * TR + r;
-    __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
-    float m = -INFINITY, z = 0.f, mc = 0.f, zc = 0.f;
+    float m = -INFINITY, z = 0.f;
     bool ok = true;
     for (int t = T0; t < my_tiles && ok; ++t) {
-      const int ti = t - T0, b = ti & 1, s = ti % NS;
+      const int ti = t - T0, b = ti & 1;
       const int key0 = t * KT;
       ok = __all_sync(kFullMask, wait(s_full + 8 * (2 * X + b), (ti >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
       {
-        uint32_t lo[32], hi[32];
-        tmem_ld32(tmem + lane_sel + col_s + b * KT, lo);
-        tmem_ld32(tmem + lane_sel + col_s + b * KT + 32, hi);
+        uint32_t lo32[32], hi32[32];
+        tmem_ld32(tmem + lane_sel + col_s + b * KT, lo32);
+        tmem_ld32(tmem + lane_sel + col_s + b * KT + 32, hi32);
         tmem_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) { sr[i] = lo[i]; sr[32 + i] = hi[i]; }
+        for (int i = 0; i < 32; ++i) { sr[i] = lo32[i]; sr[32 + i] = hi32[i]; }
       }
 
       // ---- the scalar rules, lanes b = 0..63 of this row --------------------------
@@ -349,38 +380,43 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       const bool all_visible = __all_sync(kFullMask, !valid || (key0 + KT - 1 <= p && key0 > lo));
       const bool h = all_visible || (key0 <= p && key0 + KT - 1 > lo);
       float mn, alpha;
-      float w[KT];
-      if (all_visible) {
+      {
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // the maximum is order-free
+        if (all_visible) {
 #pragma unroll
-        for (int i = 0; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-        mn = nc::new_max(m, mx, c);
-        alpha = nc::rescale(m, mn);
-        const float ng = -mn;
+          for (int i = 0; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
+        } else {
 #pragma unroll
-        for (int i = 0; i < KT; ++i) w[i] = nc::weight(__uint_as_float(sr[i]), c, ng);
-      } else {
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int i = 0; i < KT; ++i)
-          mx4[i & 3] = fmaxf(mx4[i & 3], (key0 + i <= p && key0 + i > lo) ? __uint_as_float(sr[i]) : -INFINITY);
+          for (int i = 0; i < KT; ++i)
+            mx4[i & 3] = fmaxf(mx4[i & 3], (key0 + i <= p && key0 + i > lo) ? __uint_as_float(sr[i]) : -INFINITY);
+        }
         const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         mn = h ? nc::new_max(m, mx, c) : m;
         alpha = h ? nc::rescale(m, mn) : 1.0f;
-        const float ng = -mn;
-#pragma unroll
-        for (int i = 0; i < KT; ++i)
-          w[i] = (key0 + i <= p && key0 + i > lo) ? nc::weight(__uint_as_float(sr[i]), c, ng) : 0.f;
       }
+      // the correction thread of this row can start on U while the exponentials are taken
+      alpha_s[(2 * X + b) * TR + r] = alpha;
+      mbar_arrive(a_full + 8 * (2 * X + b));
       {
+        const float ng = -mn;
+        if (all_visible) {
+#pragma unroll
+          for (int i = 0; i < KT; ++i) sr[i] = __float_as_uint(nc::weight(__uint_as_float(sr[i]), c, ng));
+        } else {
+#pragma unroll
+          for (int i = 0; i < KT; ++i)
+            sr[i] = (key0 + i <= p && key0 + i > lo) ? __float_as_uint(nc::weight(__uint_as_float(sr[i]), c, ng)) : 0u;
+        }
         // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3)
         float part[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           float a16[16];
 #pragma unroll
-          for (int n = 0; n < 8; ++n) { a16[2 * n] = w[8 * n + 2 * q]; a16[2 * n + 1] = w[8 * n + 2 * q + 1]; }
+          for (int n = 0; n < 8; ++n) {
+            a16[2 * n] = __uint_as_float(sr[8 * n + 2 * q]);
+            a16[2 * n + 1] = __uint_as_float(sr[8 * n + 2 * q + 1]);
+          }
           part[q] = nc::quad_partial(a16);
         }
         const float total = nc::quad_total(part[0], part[1], part[2], part[3]);
@@ -390,17 +426,57 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       uint32_t pk[32];
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        __nv_bfloat162 t2 = __floats2bfloat162_rn(w[2 * i], w[2 * i + 1]);
+        __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
         pk[i] = *reinterpret_cast<uint32_t*>(&t2);
       }
+      tmem_st32(tmem + lane_sel + col_s + b * KT, pk);  // the weights take the place of the scores read above
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(p_full + 8 * (2 * X + b));
 
-      // ---- U must be at rest before it is rescaled: PV of the previous tile done -----
-      if (ti > 0) {
+      // ---- end of a split: hand (m, z) to the correction thread, start afresh -----------
+      if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
+        const int kb = (t / TPS - T0 / TPS) & 1;
+        mz_s[(2 * X + kb) * TR + r] = make_float2(m, z);
+        mbar_arrive(mz_full + 8 * (2 * X + kb));
+        m = -INFINITY;
+        z = 0.f;
+      }
+    }
+  } else {
+    // ================= correction: one thread per row =====================================
+    reg_alloc<Cfg::kRegsCorrection>();
+    const int X = wg - 2;
+    const int r = tid & (TR - 1);
+    const int row = row0 + X * TR + r;
+    const bool valid = row < rows;
+    const int tok = row / G;
+    const int p = valid ? rq.start + tok : -1;
+    // first split the row sees; before it (and in the first split the CTA walks) the
+    // running result is simply taken from the split, as the fold of the split kernels does
+    const int k_first = max(nc::first_key(p, P.window) / nc::kSplitLen, T0 / TPS);
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const uint32_t col_u = Cfg::kColU + X * D;
+    const int my_tiles = n_tiles_x[X];
+    // running fold of this tile in global memory ([D/4][128] float4: this thread owns column r),
+    // and the row's place in the output
+    float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + (static_cast<size_t>(blockIdx.x) * 2 + X) * (D / 4) * TR + r;
+    __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
+    float mc = 0.f, zc = 0.f;
+    bool ok = true;
+    for (int t = T0; t < my_tiles && ok; ++t) {
+      const int ti = t - T0, b = ti & 1, s = ti % NS;
+      const int key0 = t * KT;
+      ok = __all_sync(kFullMask, wait(a_full + 8 * (2 * X + b), (ti >> 1) & 1));
+      if (!ok) break;
+      const float alpha = alpha_s[(2 * X + b) * TR + r];
+      // The accumulator of a split's first tile is fresh: nothing to rescale.  Otherwise U is
+      // rescaled unless alpha is exactly 1 for every row of the warp (u * 1 = u bit for bit);
+      // it must be at rest for that: PV of the previous tile done.
+      if ((t % TPS) != 0 && t != T0 && !__all_sync(kFullMask, alpha == 1.0f)) {
         ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + ((ti - 1) & 1)), ((ti - 1) >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
-      }
-      if ((t % TPS) != 0 && t != T0 && !__all_sync(kFullMask, alpha == 1.0f)) {
 #pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t ur[32];
@@ -410,35 +486,31 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           for (int i = 0; i < 32; ++i) ur[i] = __float_as_uint(nc::u_rescale(__uint_as_float(ur[i]), alpha));
           tmem_st32(tmem + lane_sel + col_u + cb, ur);
         }
+        tmem_wait_st();
       }
-      tmem_st32(tmem + lane_sel + col_s + b * KT, pk);  // the weights take the place of the scores read above
-      tmem_wait_st();
-      if (key0 + KT > n_eff) {
-        // Tail tile: zero the value rows at or beyond n_eff (not loaded, or pool garbage).  Only the
-        // last 128-row tile of a request reaches it; its 128 threads do the work.
+      if (key0 + KT > n_eff || key0 <= lo_first) {
+        // Value rows no row may see: at or beyond n_eff (not loaded, or pool garbage) in the tail
+        // tile; before the window of the item's first row (their pages may have been given back)
+        // in the first tile under a sliding window.  Zero them: 0 * non-finite would poison U.
         ok = __all_sync(kFullMask, wait(v_full + 8 * s, (ti / NS) & 1));
         if (!ok) break;
         const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
-        const int first = n_eff - key0;
-        const int per_half = (KT - first) * 8;
-        for (int xx = r; xx < per_half * (D / 64); xx += TR) {
-          const int half = xx / per_half, y = xx - half * per_half;
-          const uint32_t addr = vst + half * (KT * 128) + (first + (y >> 3)) * 128 + ((y & 7) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        if (key0 + KT > n_eff) {
+          const int first = n_eff - key0;
+          const int per_half = (KT - first) * 8;
+          for (int xx = r; xx < per_half * (D / 64); xx += TR) {
+            const int half = xx / per_half, y = xx - half * per_half;
+            const uint32_t addr = vst + half * (KT * 128) + (first + (y >> 3)) * 128 + ((y & 7) << 4);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+          }
         }
-        fence_proxy_async();
-      }
-      if (key0 <= lo_first) {
-        // First tile under a sliding window: the value rows before the window of the item's first
-        // row are visible to no row, and their pages may have been given back: zero them as well.
-        ok = __all_sync(kFullMask, wait(v_full + 8 * s, (ti / NS) & 1));
-        if (!ok) break;
-        const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
-        const int per_half = min(KT, lo_first - key0 + 1) * 8;
-        for (int xx = r; xx < per_half * (D / 64); xx += TR) {
-          const int half = xx / per_half, y = xx - half * per_half;
-          const uint32_t addr = vst + half * (KT * 128) + (y >> 3) * 128 + ((y & 7) << 4);
-          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+        if (key0 <= lo_first) {
+          const int per_half = min(KT, lo_first - key0 + 1) * 8;
+          for (int xx = r; xx < per_half * (D / 64); xx += TR) {
+            const int half = xx / per_half, y = xx - half * per_half;
+            const uint32_t addr = vst + half * (KT * 128) + (y >> 3) * 128 + ((y & 7) << 4);
+            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(addr), "r"(0u) : "memory");
+          }
         }
         fence_proxy_async();
       }
@@ -448,13 +520,17 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       // ---- end of a split: fold it into the running result (kept in global memory) -------
       if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
         const int split = t / TPS;
-        // the running-fold values do not depend on the PV in flight: request the first chunk now
+        const int kb = (split - T0 / TPS) & 1, kuse = (split - T0 / TPS) >> 1;
         const bool resume = split > T0 / TPS;  // the CTA has stored a running result before
+        // the running-fold values do not depend on the PV in flight: request the first chunk now
         float4 nxt4[8];
         if (resume) {
 #pragma unroll
           for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
         }
+        ok = __all_sync(kFullMask, wait(mz_full + 8 * (2 * X + kb), kuse & 1));
+        if (!ok) break;
+        const float2 mz = mz_s[(2 * X + kb) * TR + r];
         ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + b), (ti >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
@@ -465,10 +541,10 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         f.a = 1.f;
         f.b = 0.f;
         if (take) {
-          mc = m;
-          zc = z;
+          mc = mz.x;
+          zc = mz.y;
         } else if (sees) {
-          f = nc::fold_scalars(mc, zc, m, z);
+          f = nc::fold_scalars(mc, zc, mz.x, mz.y);
         }
         const float inv = nc::out_scale(zc);  // used on the last split only
         // chunks of 32 columns; the running-fold values of chunk c+1 are requested before chunk c is processed
@@ -515,8 +591,6 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
               ucg[static_cast<size_t>(cb / 4 + i) * TR] = make_float4(un[4 * i], un[4 * i + 1], un[4 * i + 2], un[4 * i + 3]);
           }
         }
-        m = -INFINITY;
-        z = 0.f;
       }
     }
   }

@@ -397,6 +397,11 @@ vosti_status set_kernel_attributes() {
   if (cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            TileKernelCfg<D>::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
+  // The tile kernel moves registers between its warpgroups; a request for more than the CTA
+  // was given at launch would block for ever, so refuse to run a build where that could happen.
+  cudaFuncAttributes attr;
+  if (cudaFuncGetAttributes(&attr, attn_tile_kernel<D>) != cudaSuccess) return VOSTI_ERR_CUDA;
+  if (attr.numRegs * TileKernelCfg<D>::kThreads < TileKernelCfg<D>::kRegsAfterSplit) return VOSTI_ERR_UNSUPPORTED_CONFIG;
   return VOSTI_OK;
 }
 
