@@ -1,7 +1,7 @@
-// Tile attention for long queries (prefill chunks): one CTA per (256-row super
-// tile, KV head), QK^T and PV on the 5th-generation tensor cores (tcgen05.mma,
-// M = 128) with the accumulators in tensor memory, K/V tiles gathered from the
-// page pool by TMA.
+// Tile attention for long queries (prefill chunks): one CTA per (128-row tile,
+// KV head), two CTAs per SM, QK^T and PV on the 5th-generation tensor cores
+// (tcgen05.mma, M = 128) with the accumulators in tensor memory, K/V tiles
+// gathered from the page pool by TMA.
 //
 // It executes the same numerical contract as the split-parallel kernel: key
 // tiles of 64 in ascending order; S from head-dim chunks of 16 ascending with a
@@ -14,9 +14,7 @@
 // sums for the same chunk order (measured on B200), which is what lets this
 // kernel and the warp-MMA kernels agree bit for bit.
 //
-// A CTA holds TWO 128-row tiles (X = 0, 1) that share every staged K/V tile, so
-// K/V is fetched through L2 once per 256 rows.  Work on a row is divided between
-// two threads so that neither chain is long:
+// Work on a row is divided between two threads so that neither chain is long:
 //   * a softmax thread reads the row's 64 scores, applies the scalar rules
 //     (maximum, alpha, exponentials, pinned row sum), publishes alpha and writes
 //     the bf16 weights over the scores;
@@ -24,15 +22,19 @@
 //     some alpha of its warp is not 1, zero-fills value rows no query row may
 //     see, and at the end of every split folds the split into the running
 //     result (and, at the end of the row, normalises and stores it).
-// Roles by warpgroup (640 threads): 0 / 1 = softmax of tile 0 / 1, 2 / 3 =
-// correction of tile 0 / 1, 4 = { K producer, MMA issuer of tile 0, V producer,
-// MMA issuer of tile 1 }.  Registers are moved from warpgroup 4 to the others
-// with setmaxnreg.  Each tile has its own issuer thread: the MMAs of one thread
-// run in issue order, which the aliasing of weights over scores relies on, and
-// the two tiles never wait for each other.
-// Tensor memory (512 columns): per tile S x2 (64 each; the bf16 weights P are
+// Roles by warpgroup (384 threads): 0 = softmax, 1 = correction, 2 = { K
+// producer, MMA issuer, V producer }.  Registers are moved from warpgroup 2 to
+// the others with setmaxnreg.  The MMAs of the one issuing thread run in issue
+// order, which the aliasing of weights over scores relies on.
+// Two such CTAs share an SM (half of its shared memory, tensor memory and
+// registers each) and know nothing of each other: while one of them waits --
+// for its softmax, or for the split fold, which moves 128 KB between tensor
+// memory and L2 -- the other one keeps the tensor and MUFU pipes busy.  The two
+// 128-row halves of a 256-row work item are neighbouring CTAs, so the K/V tiles
+// the second one asks for are in L2 already.
+// Tensor memory (256 columns per CTA): S x2 (64 each; the bf16 weights P are
 // written over the first 32 columns of the S buffer they were computed from)
-// and U (D).  The running fold U_c lives in global memory (per CTA and tile a
+// and U (D).  The running fold U_c lives in global memory (per CTA a
 // [D/4][128 rows] array of float4, so that a warp's rows are contiguous; touched
 // once per split): there is no room for it on chip.
 #pragma once
@@ -43,28 +45,30 @@ namespace vosti {
 
 template <int D>
 struct TileKernelCfg {
-  static constexpr int kRows = 256;                          // rows of a work item: two tiles
+  static constexpr int kItemRows = 256;                      // rows of a work item: two CTAs
   static constexpr int kTileRows = 128;
-  static constexpr int kThreads = 640;
-  static constexpr int kStages = 3;                          // K+V tile pairs in flight
-  static constexpr int kQBytes = kRows * D * 2;              // [half][row][128 B]
+  static constexpr int kThreads = 384;
+  static constexpr int kStages = 2;                          // K+V tile pairs in flight
+  static constexpr int kQBytes = kTileRows * D * 2;          // [half][row][128 B]
   static constexpr int kKBytes = nc::kKeyTile * D * 2;       // [half][key][128 B]
   static constexpr int kStageBytes = 2 * kKBytes;            // K then V
-  static constexpr int kAlphaBytes = 2 * 2 * kTileRows * 4;  // alpha[tile][buffer][row]
-  static constexpr int kMzBytes = 2 * 2 * kTileRows * 8;     // (m, z)[tile][split parity][row]
+  static constexpr int kAlphaBytes = 2 * kTileRows * 4;      // alpha[buffer][row]
+  static constexpr int kMzBytes = 2 * kTileRows * 8;         // (m, z)[split parity][row]
   static constexpr int kBarBytes = 512;
   static constexpr int kSmemBytes = kQBytes + kStages * kStageBytes + kAlphaBytes + kMzBytes + kBarBytes + 1024;
   // Registers per thread after the roles have split.  The total must not exceed what the CTA
-  // was given at launch (640 threads x 96 registers): a warpgroup asking for more than the
+  // was given at launch (384 threads x 80 registers): a warpgroup asking for more than the
   // others have released waits for ever.
-  static constexpr int kRegsSoftmax = 120;
-  static constexpr int kRegsCorrection = 104;
+  static constexpr int kRegsLaunch = 80;
+  static constexpr int kRegsSoftmax = 112;
+  static constexpr int kRegsCorrection = 96;
   static constexpr int kRegsOther = 32;
-  static constexpr int kRegsAfterSplit = 32 * (8 * kRegsSoftmax + 8 * kRegsCorrection + 4 * kRegsOther);
-  static_assert(kRegsAfterSplit <= kThreads * 96, "register split exceeds the launch allocation");
+  static constexpr int kRegsAfterSplit = 128 * (kRegsSoftmax + kRegsCorrection + kRegsOther);
+  static_assert(kRegsAfterSplit <= kThreads * kRegsLaunch, "register split exceeds the launch allocation");
   // tensor-memory columns
-  static constexpr uint32_t kColS = 0;    // tile X, buffer b: S / P at 128 X + 64 b
-  static constexpr uint32_t kColU = 256;  // tile X: U at 256 + D X
+  static constexpr uint32_t kTmemCols = 256;
+  static constexpr uint32_t kColS = 0;    // buffer b: S / P at 64 b
+  static constexpr uint32_t kColU = 128;  // U
 };
 
 template <int N>
@@ -108,6 +112,14 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
         "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
 }
+// 16 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -139,7 +151,7 @@ __host__ __device__ constexpr uint32_t umma_idesc(int m, int n, bool b_mn_major)
 }
 
 template <int D>
-__global__ void __launch_bounds__(TileKernelCfg<D>::kThreads, 1)
+__global__ void __launch_bounds__(TileKernelCfg<D>::kThreads, 2)
 attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {
   using Cfg = TileKernelCfg<D>;
   constexpr int NS = Cfg::kStages;
@@ -148,56 +160,50 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   constexpr int TR = Cfg::kTileRows;
   constexpr uint32_t kAbortAfterNs = 1000000000u;
 
-  extern __shared__ uint8_t smem_raw[];
-  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t q_smem = base;  // tile X at X * TR * D * 2
-  const uint32_t kv_smem = base + Cfg::kQBytes;
-  constexpr int kXchgOff = Cfg::kQBytes + NS * Cfg::kStageBytes;
-  float* alpha_s = reinterpret_cast<float*>(sbase + kXchgOff);                      // [X][b][row]
-  float2* mz_s = reinterpret_cast<float2*>(sbase + kXchgOff + Cfg::kAlphaBytes);     // [X][kb][row]
-  constexpr int kBarOff = kXchgOff + Cfg::kAlphaBytes + Cfg::kMzBytes;
-  const uint32_t bars = base + kBarOff;
-  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + kBarOff + 448);
-  // barrier map (8 bytes each); per tile X and buffer b: index 2 X + b
-  const uint32_t k_full = bars, v_full = bars + 8 * NS, k_empty = bars + 16 * NS, v_empty = bars + 24 * NS;
-  const uint32_t s_full = bars + 32 * NS, p_full = s_full + 32, pv_done = s_full + 64;
-  const uint32_t a_full = s_full + 96, mz_full = s_full + 128;
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int wg = warp >> 2;
-
-  const vosti_work_item item = P.items[blockIdx.x / P.Hkv];
-  const int kvh = blockIdx.x % P.Hkv;
+  // CTA -> (work item, KV head, half of the item)
+  const vosti_work_item item = P.items[(blockIdx.x >> 1) / P.Hkv];
+  const int kvh = (blockIdx.x >> 1) % P.Hkv;
   const ReqMeta rq = P.reqs[item.req];
   const int G = P.G;
-  const int row0 = item.row_group * nc::kRowsPerGroup;  // first row of the 256-row super tile
+  const int row0 = item.row_group * nc::kRowsPerGroup + (blockIdx.x & 1) * TR;  // first row of this CTA's tile
   const int rows = rq.q_len * G;
+  if (row0 >= rows) return;  // the item's second half does not exist
   const int n_eff = rq.start + rq.q_len;
-  // key tiles each 128-row tile walks (0: the tile does not exist)
-  int n_tiles_x[2];
-#pragma unroll
-  for (int X = 0; X < 2; ++X) {
-    const int first = row0 + X * TR;
-    const int last_tok = min(rq.q_len - 1, (first + TR - 1) / G);
-    n_tiles_x[X] = first < rows ? (rq.start + last_tok) / KT + 1 : 0;
-  }
-  const int n_tiles = max(n_tiles_x[0], n_tiles_x[1]);  // tile 1 holds later positions: it is the longer one
-  // Under a sliding window nothing before the first visible key of the item's first row is
-  // needed: both tiles start at key tile T0 (rows whose own window starts later take identity
+  const int n_tiles = (rq.start + min(rq.q_len - 1, (row0 + TR - 1) / G)) / KT + 1;  // key tiles walked
+  // Under a sliding window nothing before the first visible key of the tile's first row is
+  // needed: the walk starts at key tile T0 (rows whose own window starts later take identity
   // steps until it does).  Stages, S buffers and barrier phases are indexed by t - T0.
   const int p_first = rq.start + row0 / G;
   const int T0 = nc::first_key(p_first, P.window) / KT;
   const int lo_first = nc::window_lo(p_first, P.window);  // keys up to here are invisible to every row
 
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t q_smem = base;
+  const uint32_t kv_smem = base + Cfg::kQBytes;
+  constexpr int kXchgOff = Cfg::kQBytes + NS * Cfg::kStageBytes;
+  float* alpha_s = reinterpret_cast<float*>(sbase + kXchgOff);                       // [b][row]
+  float2* mz_s = reinterpret_cast<float2*>(sbase + kXchgOff + Cfg::kAlphaBytes);     // [kb][row]
+  constexpr int kBarOff = kXchgOff + Cfg::kAlphaBytes + Cfg::kMzBytes;
+  const uint32_t bars = base + kBarOff;
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + kBarOff + 448);
+  // barrier map (8 bytes each); per buffer b: index b
+  const uint32_t k_full = bars, v_full = bars + 8 * NS, k_empty = bars + 16 * NS, v_empty = bars + 24 * NS;
+  const uint32_t s_full = bars + 32 * NS, p_full = s_full + 16, pv_done = s_full + 32;
+  const uint32_t a_full = s_full + 48, mz_full = s_full + 64;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int wg = warp >> 2;
+
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
       mbar_init(k_full + 8 * i, 1);
       mbar_init(v_full + 8 * i, 1);
-      mbar_init(k_empty + 8 * i, 2);  // both issuers release a stage
-      mbar_init(v_empty + 8 * i, 2);
+      mbar_init(k_empty + 8 * i, 1);
+      mbar_init(v_empty + 8 * i, 1);
     }
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < 2; ++i) {
       mbar_init(s_full + 8 * i, 1);
       mbar_init(p_full + 8 * i, 2 * TR);  // softmax and correction thread of every row
       mbar_init(pv_done + 8 * i, 1);
@@ -209,14 +215,15 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     tma_prefetch_desc(&kv_map);
   }
   if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 456), "r"(512));
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 456),
+                 "r"(Cfg::kTmemCols));
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
   }
-  // Q tiles -> shared memory, per tile [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
-  if (warp < 8) {
+  // Q tile -> shared memory, [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
+  if (warp < 4) {
     griddep_wait();
-    const int X = warp >> 2, r = tid & (TR - 1);
-    const int row = row0 + X * TR + r;
+    const int r = tid;
+    const int row = row0 + r;
     const bool valid = row < rows;
     const int tok = row / G;
     const uint4* src = reinterpret_cast<const uint4*>(
@@ -224,7 +231,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
 #pragma unroll
     for (int c = 0; c < D / 8; ++c) {
       const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-      const uint32_t addr = q_smem + X * (TR * D * 2) + (c >> 3) * (TR * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
+      const uint32_t addr = q_smem + (c >> 3) * (TR * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
       asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
                    : "memory");
     }
@@ -253,13 +260,30 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       }
     }
   };
+  // The same for a single thread that must react at once (the MMA issuer): polls without sleeping.
+  auto wait_spin = [&](uint32_t bar, uint32_t parity) -> bool {
+    uint64_t t0 = 0;
+    for (uint32_t it = 0;; ++it) {
+      if (mbar_test_wait(bar, parity)) return true;
+      if ((it & 1023u) == 1023u) {
+        if (flags[0] != 0u) return false;
+        if (it == 1023u) {
+          t0 = global_timer_ns();
+        } else if (global_timer_ns() - t0 > kAbortAfterNs) {
+          flags[0] = 1u;
+          atomicOr(P.status, kStatusTimeout);
+          return false;
+        }
+      }
+    }
+  };
 
-  if (wg == 4) {
+  if (wg == 2) {
     reg_dealloc<Cfg::kRegsOther>();
-    if (warp == 16 || warp == 18) {
-      // ================= TMA producers: warp 16 loads the K tiles, warp 18 the V tiles =======
+    if (warp == 8 || warp == 10) {
+      // ================= TMA producers: warp 8 loads the K tiles, warp 10 the V tiles =======
       griddep_wait();
-      const int is_v = warp == 18;
+      const int is_v = warp == 10;
       const int32_t* bt = P.bt_flat + rq.bt_off;
       auto fetch_pages = [&](int split) -> int {
         const int pg = split * nc::kPagesPerSplit + lane;
@@ -284,39 +308,36 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         if (!ok) break;
         issue_stage_load<D, KT>(&kv_map, dst, full, ids, tl * nc::kPagesPerTile, n_valid, P.Hkv, kvh, is_v, lane);
       }
-    } else if (lane == 0) {
-      // ================= MMA issuers: warp 17 for tile 0, warp 19 for tile 1 ==================
+    } else if (warp == 9 && lane == 0) {
+      // ================= MMA issuer ==========================================================
       // One thread's MMAs run in issue order.  S of key tile t+2 overwrites the buffer whose
       // first columns PV of key tile t reads its weights from, so it is issued after that PV.
-      const int X = (warp - 17) >> 1;
-      const int my_tiles = n_tiles_x[X];
       constexpr uint32_t idesc_s = umma_idesc(128, KT, false);
       constexpr uint32_t idesc_pv = umma_idesc(128, D, true);
-      const uint32_t qx = q_smem + X * (TR * D * 2);
       bool ok = true;
       auto issue_s = [&](int t) {
         const int i = t - T0, s = i % NS, b = i & 1;
-        ok = ok && wait(k_full + 8 * s, (i / NS) & 1);
+        ok = ok && wait_spin(k_full + 8 * s, (i / NS) & 1);
         if (!ok) return;
         tc_fence_after();
         const uint32_t kst = kv_smem + s * Cfg::kStageBytes;
 #pragma unroll
         for (int kc = 0; kc < D / 16; ++kc) {
-          const uint64_t da = smem_desc_sw128(qx + (kc >> 2) * (TR * 128) + (kc & 3) * 32, 16, 1024);
+          const uint64_t da = smem_desc_sw128(q_smem + (kc >> 2) * (TR * 128) + (kc & 3) * 32, 16, 1024);
           const uint64_t db = smem_desc_sw128(kst + (kc >> 2) * (KT * 128) + (kc & 3) * 32, 16, 1024);
-          tc_mma_ss(tmem + Cfg::kColS + X * 128 + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
+          tc_mma_ss(tmem + Cfg::kColS + b * KT, da, db, idesc_s, kc > 0 ? 1u : 0u);
         }
-        tc_commit(s_full + 8 * (2 * X + b));
+        tc_commit(s_full + 8 * b);
         tc_commit(k_empty + 8 * s);
       };
-      if (T0 < my_tiles) issue_s(T0);
-      for (int t = T0; t < my_tiles && ok; ++t) {
-        if (t + 1 < my_tiles) issue_s(t + 1);
+      issue_s(T0);
+      for (int t = T0; t < n_tiles && ok; ++t) {
+        if (t + 1 < n_tiles) issue_s(t + 1);
         if (!ok) break;
         const int i = t - T0, s = i % NS, b = i & 1;
-        ok = wait(v_full + 8 * s, (i / NS) & 1);
+        ok = wait_spin(v_full + 8 * s, (i / NS) & 1);
         if (!ok) break;
-        ok = wait(p_full + 8 * (2 * X + b), (i >> 1) & 1);
+        ok = wait_spin(p_full + 8 * b, (i >> 1) & 1);
         if (!ok) break;
         tc_fence_after();
         const uint32_t vst = kv_smem + s * Cfg::kStageBytes + Cfg::kKBytes;
@@ -326,49 +347,35 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           const uint64_t db = smem_desc_sw128(vst + kc * 2048, KT * 128, 1024);
           // a split (and the first tile walked) starts from a fresh accumulator
           const uint32_t acc = (kc > 0 || ((t % TPS) != 0 && t != T0)) ? 1u : 0u;
-          tc_mma_ts(tmem + Cfg::kColU + X * D, tmem + Cfg::kColS + X * 128 + b * KT + kc * 8, db, idesc_pv, acc);
+          tc_mma_ts(tmem + Cfg::kColU, tmem + Cfg::kColS + b * KT + kc * 8, db, idesc_pv, acc);
         }
-        tc_commit(pv_done + 8 * (2 * X + b));
+        tc_commit(pv_done + 8 * b);
         tc_commit(v_empty + 8 * s);
       }
-      // Key tiles only the other tile walks: hand the stages back unused, each after it has
-      // been filled (so that an arrival can never count towards an earlier use of the stage).
-      for (int t = max(my_tiles, T0); t < n_tiles && ok; ++t) {
-        const int i = t - T0, s = i % NS;
-        ok = wait(k_full + 8 * s, (i / NS) & 1);
-        if (!ok) break;
-        mbar_arrive(k_empty + 8 * s);
-        ok = wait(v_full + 8 * s, (i / NS) & 1);
-        if (!ok) break;
-        mbar_arrive(v_empty + 8 * s);
-      }
     }
-  } else if (wg < 2) {
+  } else if (wg == 0) {
     // ================= softmax: one thread per row =======================================
     reg_alloc<Cfg::kRegsSoftmax>();
-    const int X = wg;                           // which 128-row tile
-    const int r = tid & (TR - 1);               // row of the tile = tensor-memory lane
-    const int row = row0 + X * TR + r;
+    const int r = tid;                          // row of the tile = tensor-memory lane
+    const int row = row0 + r;
     const bool valid = row < rows;
     const int p = valid ? rq.start + row / G : -1;  // padding rows see nothing
     const int lo = nc::window_lo(p, P.window);      // key j is visible iff lo < j <= p
-    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t col_s = Cfg::kColS + X * 128;
-    const int my_tiles = n_tiles_x[X];
+    const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
     const float c = P.c;
     float m = -INFINITY, z = 0.f;
     bool ok = true;
-    for (int t = T0; t < my_tiles && ok; ++t) {
+    for (int t = T0; t < n_tiles && ok; ++t) {
       const int ti = t - T0, b = ti & 1;
       const int key0 = t * KT;
-      ok = __all_sync(kFullMask, wait(s_full + 8 * (2 * X + b), (ti >> 1) & 1));
+      ok = __all_sync(kFullMask, wait(s_full + 8 * b, (ti >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
       uint32_t sr[64];
       {
         uint32_t lo32[32], hi32[32];
-        tmem_ld32(tmem + lane_sel + col_s + b * KT, lo32);
-        tmem_ld32(tmem + lane_sel + col_s + b * KT + 32, hi32);
+        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT, lo32);
+        tmem_ld32(tmem + lane_sel + Cfg::kColS + b * KT + 32, hi32);
         tmem_wait_ld();
 #pragma unroll
         for (int i = 0; i < 32; ++i) { sr[i] = lo32[i]; sr[32 + i] = hi32[i]; }
@@ -395,8 +402,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         alpha = h ? nc::rescale(m, mn) : 1.0f;
       }
       // the correction thread of this row can start on U while the exponentials are taken
-      alpha_s[(2 * X + b) * TR + r] = alpha;
-      mbar_arrive(a_full + 8 * (2 * X + b));
+      alpha_s[b * TR + r] = alpha;
+      mbar_arrive(a_full + 8 * b);
       {
         const float ng = -mn;
         if (all_visible) {
@@ -429,16 +436,16 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(sr[2 * i]), __uint_as_float(sr[2 * i + 1]));
         pk[i] = *reinterpret_cast<uint32_t*>(&t2);
       }
-      tmem_st32(tmem + lane_sel + col_s + b * KT, pk);  // the weights take the place of the scores read above
+      tmem_st32(tmem + lane_sel + Cfg::kColS + b * KT, pk);  // the weights take the place of the scores read above
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(p_full + 8 * (2 * X + b));
+      mbar_arrive(p_full + 8 * b);
 
       // ---- end of a split: hand (m, z) to the correction thread, start afresh -----------
-      if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
+      if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
         const int kb = (t / TPS - T0 / TPS) & 1;
-        mz_s[(2 * X + kb) * TR + r] = make_float2(m, z);
-        mbar_arrive(mz_full + 8 * (2 * X + kb));
+        mz_s[kb * TR + r] = make_float2(m, z);
+        mbar_arrive(mz_full + 8 * kb);
         m = -INFINITY;
         z = 0.f;
       }
@@ -446,9 +453,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   } else {
     // ================= correction: one thread per row =====================================
     reg_alloc<Cfg::kRegsCorrection>();
-    const int X = wg - 2;
     const int r = tid & (TR - 1);
-    const int row = row0 + X * TR + r;
+    const int row = row0 + r;
     const bool valid = row < rows;
     const int tok = row / G;
     const int p = valid ? rq.start + tok : -1;
@@ -456,41 +462,39 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     // running result is simply taken from the split, as the fold of the split kernels does
     const int k_first = max(nc::first_key(p, P.window) / nc::kSplitLen, T0 / TPS);
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const uint32_t col_u = Cfg::kColU + X * D;
-    const int my_tiles = n_tiles_x[X];
     // running fold of this tile in global memory ([D/4][128] float4: this thread owns column r),
     // and the row's place in the output
-    float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + (static_cast<size_t>(blockIdx.x) * 2 + X) * (D / 4) * TR + r;
+    float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + static_cast<size_t>(blockIdx.x) * (D / 4) * TR + r;
     __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
     float mc = 0.f, zc = 0.f;
     bool ok = true;
-    for (int t = T0; t < my_tiles && ok; ++t) {
+    for (int t = T0; t < n_tiles && ok; ++t) {
       const int ti = t - T0, b = ti & 1, s = ti % NS;
       const int key0 = t * KT;
-      ok = __all_sync(kFullMask, wait(a_full + 8 * (2 * X + b), (ti >> 1) & 1));
+      ok = __all_sync(kFullMask, wait(a_full + 8 * b, (ti >> 1) & 1));
       if (!ok) break;
-      const float alpha = alpha_s[(2 * X + b) * TR + r];
+      const float alpha = alpha_s[b * TR + r];
       // The accumulator of a split's first tile is fresh: nothing to rescale.  Otherwise U is
       // rescaled unless alpha is exactly 1 for every row of the warp (u * 1 = u bit for bit);
       // it must be at rest for that: PV of the previous tile done.
       if ((t % TPS) != 0 && t != T0 && !__all_sync(kFullMask, alpha == 1.0f)) {
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + ((ti - 1) & 1)), ((ti - 1) >> 1) & 1));
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * ((ti - 1) & 1), ((ti - 1) >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
 #pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t ur[32];
-          tmem_ld32(tmem + lane_sel + col_u + cb, ur);
+          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
           tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 32; ++i) ur[i] = __float_as_uint(nc::u_rescale(__uint_as_float(ur[i]), alpha));
-          tmem_st32(tmem + lane_sel + col_u + cb, ur);
+          tmem_st32(tmem + lane_sel + Cfg::kColU + cb, ur);
         }
         tmem_wait_st();
       }
       if (key0 + KT > n_eff || key0 <= lo_first) {
         // Value rows no row may see: at or beyond n_eff (not loaded, or pool garbage) in the tail
-        // tile; before the window of the item's first row (their pages may have been given back)
+        // tile; before the window of the tile's first row (their pages may have been given back)
         // in the first tile under a sliding window.  Zero them: 0 * non-finite would poison U.
         ok = __all_sync(kFullMask, wait(v_full + 8 * s, (ti / NS) & 1));
         if (!ok) break;
@@ -515,26 +519,26 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         fence_proxy_async();
       }
       tc_fence_before();
-      mbar_arrive(p_full + 8 * (2 * X + b));
+      mbar_arrive(p_full + 8 * b);
 
       // ---- end of a split: fold it into the running result (kept in global memory) -------
-      if ((t + 1) % TPS == 0 || t + 1 == my_tiles) {
+      if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
         const int split = t / TPS;
         const int kb = (split - T0 / TPS) & 1, kuse = (split - T0 / TPS) >> 1;
         const bool resume = split > T0 / TPS;  // the CTA has stored a running result before
         // the running-fold values do not depend on the PV in flight: request the first chunk now
-        float4 nxt4[8];
+        float4 nxt4[4];
         if (resume) {
 #pragma unroll
-          for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
+          for (int i = 0; i < 4; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
         }
-        ok = __all_sync(kFullMask, wait(mz_full + 8 * (2 * X + kb), kuse & 1));
+        ok = __all_sync(kFullMask, wait(mz_full + 8 * kb, kuse & 1));
         if (!ok) break;
-        const float2 mz = mz_s[(2 * X + kb) * TR + r];
-        ok = __all_sync(kFullMask, wait(pv_done + 8 * (2 * X + b), (ti >> 1) & 1));
+        const float2 mz = mz_s[kb * TR + r];
+        ok = __all_sync(kFullMask, wait(pv_done + 8 * b, (ti >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
-        const bool last = t + 1 == my_tiles;
+        const bool last = t + 1 == n_tiles;
         const bool take = split <= k_first;  // the row's first split: the running result starts from it
         const bool sees = p >= split * nc::kSplitLen;
         nc::FoldFactors f;
@@ -547,34 +551,34 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           f = nc::fold_scalars(mc, zc, mz.x, mz.y);
         }
         const float inv = nc::out_scale(zc);  // used on the last split only
-        // chunks of 32 columns; the running-fold values of chunk c+1 are requested before chunk c is processed
+        if (last && valid && P.lse != nullptr)
+          P.lse[static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G] = nc::lse_value(mc, zc);
+        // chunks of 16 columns; the running-fold values of chunk c+1 are requested before chunk c is processed
 #pragma unroll 1
-        for (int cb = 0; cb < D; cb += 32) {
-          uint32_t ur[32];
-          tmem_ld32(tmem + lane_sel + col_u + cb, ur);
-          float un[32];
+        for (int cb = 0; cb < D; cb += 16) {
+          uint32_t ur[16];
+          tmem_ld16(tmem + lane_sel + Cfg::kColU + cb, ur);
+          float un[16];
           if (resume) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < 4; ++i) {
               un[4 * i] = nxt4[i].x; un[4 * i + 1] = nxt4[i].y; un[4 * i + 2] = nxt4[i].z; un[4 * i + 3] = nxt4[i].w;
             }
-            if (cb + 32 < D) {
+            if (cb + 16 < D) {
 #pragma unroll
-              for (int i = 0; i < 8; ++i) nxt4[i] = ucg[static_cast<size_t>((cb + 32) / 4 + i) * TR];
+              for (int i = 0; i < 4; ++i) nxt4[i] = ucg[static_cast<size_t>((cb + 16) / 4 + i) * TR];
             }
           }
           tmem_wait_ld();
 #pragma unroll
-          for (int i = 0; i < 32; ++i) {
+          for (int i = 0; i < 16; ++i) {
             const float u = __uint_as_float(ur[i]);
             un[i] = take ? u : (sees ? nc::fold_u(un[i], u, f) : un[i]);
           }
           if (last) {
             if (valid) {
-              if (cb == 0 && P.lse != nullptr)
-                P.lse[static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G] = nc::lse_value(mc, zc);
 #pragma unroll
-              for (int i = 0; i < 32; i += 8) {
+              for (int i = 0; i < 16; i += 8) {
                 uint32_t o[4];
 #pragma unroll
                 for (int xx = 0; xx < 4; ++xx) {
@@ -587,7 +591,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
             }
           } else {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+            for (int i = 0; i < 4; ++i)
               ucg[static_cast<size_t>(cb / 4 + i) * TR] = make_float4(un[4 * i], un[4 * i + 1], un[4 * i + 2], un[4 * i + 3]);
           }
         }
@@ -598,7 +602,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   // Common exit: every role ends here, also after a timeout, so tensor memory is always released.
   tc_fence_before();
   __syncthreads();
-  if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512));
+  if (warp == 0)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
 }
 
 }  // namespace vosti

@@ -377,7 +377,8 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
     p.n_workers = static_cast<int32_t>(n_seq * Hkv);
     using TileCfg_ = TileKernelCfg<D>;
     timed(2, [&] {
-      launch_dependent(attn_tile_kernel<D>, p.n_workers, TileCfg_::kThreads, TileCfg_::kSmemBytes, stream,
+      // two CTAs (128 rows each) per item and KV head
+      launch_dependent(attn_tile_kernel<D>, 2 * p.n_workers, TileCfg_::kThreads, TileCfg_::kSmemBytes, stream,
                        ctx->kv_map, p);
     });
   }
@@ -395,7 +396,9 @@ vosti_status set_kernel_attributes() {
                            Cfg::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           TileKernelCfg<D>::kSmemBytes) != cudaSuccess)
+                           TileKernelCfg<D>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   // The tile kernel moves registers between its warpgroups; a request for more than the CTA
   // was given at launch would block for ever, so refuse to run a build where that could happen.
