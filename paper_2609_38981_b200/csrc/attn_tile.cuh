@@ -391,7 +391,11 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // the maximum is order-free
         if (all_visible) {
 #pragma unroll
-          for (int i = 0; i < KT; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(sr[i]));
+          for (int i = 0; i < KT; i += 8) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              mx4[j] = nc::max3(mx4[j], __uint_as_float(sr[i + j]), __uint_as_float(sr[i + 4 + j]));
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < KT; ++i)
@@ -407,24 +411,32 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       {
         const float ng = -mn;
         if (all_visible) {
+          const uint64_t c2 = nc::pack2(c, c), ng2 = nc::pack2(ng, ng);
 #pragma unroll
-          for (int i = 0; i < KT; ++i) sr[i] = __float_as_uint(nc::weight(__uint_as_float(sr[i]), c, ng));
+          for (int i = 0; i < KT; i += 2) {
+            float a0, a1;
+            nc::weight2(__uint_as_float(sr[i]), __uint_as_float(sr[i + 1]), c2, ng2, a0, a1);
+            sr[i] = __float_as_uint(a0);
+            sr[i + 1] = __float_as_uint(a1);
+          }
         } else {
 #pragma unroll
           for (int i = 0; i < KT; ++i)
             sr[i] = (key0 + i <= p && key0 + i > lo) ? __float_as_uint(nc::weight(__uint_as_float(sr[i]), c, ng)) : 0u;
         }
-        // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3)
+        // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3).
+        // Partials 0 and 1 advance together in one packed add, as do partials 2 and 3.
         float part[4];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          float a16[16];
+        for (int q = 0; q < 4; q += 2) {
+          uint64_t acc = nc::pack2(__uint_as_float(sr[2 * q]), __uint_as_float(sr[2 * q + 2]));
+          acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[2 * q + 1]), __uint_as_float(sr[2 * q + 3])));
 #pragma unroll
-          for (int n = 0; n < 8; ++n) {
-            a16[2 * n] = __uint_as_float(sr[8 * n + 2 * q]);
-            a16[2 * n + 1] = __uint_as_float(sr[8 * n + 2 * q + 1]);
+          for (int n = 1; n < 8; ++n) {
+            acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[8 * n + 2 * q]), __uint_as_float(sr[8 * n + 2 * q + 2])));
+            acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[8 * n + 2 * q + 1]), __uint_as_float(sr[8 * n + 2 * q + 3])));
           }
-          part[q] = nc::quad_partial(a16);
+          nc::unpack2(acc, part[q], part[q + 1]);
         }
         const float total = nc::quad_total(part[0], part[1], part[2], part[3]);
         z = h ? nc::z_update(z, alpha, total) : z;
@@ -486,8 +498,14 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           uint32_t ur[32];
           tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
           tmem_wait_ld();
+          const uint64_t alpha2 = nc::pack2(alpha, alpha);
 #pragma unroll
-          for (int i = 0; i < 32; ++i) ur[i] = __float_as_uint(nc::u_rescale(__uint_as_float(ur[i]), alpha));
+          for (int i = 0; i < 32; i += 2) {  // u * alpha, two lanes per instruction
+            float u0, u1;
+            nc::unpack2(nc::mul2(nc::pack2(__uint_as_float(ur[i]), __uint_as_float(ur[i + 1])), alpha2), u0, u1);
+            ur[i] = __float_as_uint(u0);
+            ur[i + 1] = __float_as_uint(u1);
+          }
           tmem_st32(tmem + lane_sel + Cfg::kColU + cb, ur);
         }
         tmem_wait_st();

@@ -67,6 +67,47 @@ __device__ __forceinline__ float quad_total(float s0, float s1, float s2, float 
   return __fadd_rn(__fadd_rn(s0, s1), __fadd_rn(s2, s3));
 }
 
+// Two lanes at a time.  Each half of a packed f32x2 operation is the same IEEE
+// round-to-nearest operation as its scalar form above, so a kernel may use
+// either form for any lane without changing a bit; the packed forms halve the
+// instruction count where one thread owns many lanes of a row.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// A for two lanes: 2^(s*c - m_hat) each.
+__device__ __forceinline__ void weight2(float s0, float s1, uint64_t c2, uint64_t neg_m2, float& a0, float& a1) {
+  float e0, e1;
+  unpack2(fma2(pack2(s0, s1), c2, neg_m2), e0, e1);
+  a0 = ex2(e0);
+  a1 = ex2(e1);
+}
+// maximum of three (the maximum is order-free; inputs are finite or -inf)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // Left fold of split results.  (m_c, z_c, U_c) <- fold((m_c, z_c, U_c), (m_k, z_k, U_k)).
 struct FoldFactors {
   float a, b;
