@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--no-kernel-events", action="store_true",
                     help="experiment: do not record per-kernel events in the timed region")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (experiments only)")
+    ap.add_argument("--pack-shared-splits", action="store_true",
+                    help="create the context with VOSTI_FLAG_PACK_SHARED_SPLITS (same bits, fewer tiles "
+                         "when requests share prefix pages)")
     ap.add_argument("--pool-pages", type=int, default=0,
                     help="override the pool size (small pools keep profiler captures short)")
     return ap.parse_args()
@@ -221,7 +224,8 @@ def main():
     scale = geo.head_dim ** -0.5
     max_seq = max(w.seq_lens)
     cache = DeviceCache(geo, w.num_pages, max_batch=w.batch, max_total_q=max(8192, w.total_q),
-                        max_seq_len=max_seq, device=f"cuda:{local}")
+                        max_seq_len=max_seq, device=f"cuda:{local}",
+                        flags=vb.VOSTI_FLAG_PACK_SHARED_SPLITS if args.pack_shared_splits else 0)
     cache.upload(w.requests, w.tables, upto=w.start_pos)      # cached context before the step
     bt = inputs.block_table_array(w.tables)
     ql, st, sl = (np.asarray(x, dtype=np.int32) for x in (w.q_lens, w.start_pos, w.seq_lens))
@@ -358,6 +362,9 @@ def main():
                 "timing": "value: K steps with nothing recorded between kernels; roofline: a second pass of "
                           "K steps with a CUDA event pair around each launch of the dominant kernel",
                 "ms_per_step_with_kernel_events": roof_ms / args.steps,
+                "pack_shared_splits": bool(args.pack_shared_splits),
+                "schedule": dict(zip(("split_items", "packed_items", "tile_items"),
+                                     vb.vosti_last_schedule(cache.ctx))),
             },
             "tokens_per_s": tok_all / (ms_per_step * 1e-3),
             "pct_of_8TBs": 100.0 * value / world / NOMINAL_HBM_GBS,

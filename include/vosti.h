@@ -59,7 +59,19 @@ typedef enum {
 } vosti_status;
 
 enum {
-  VOSTI_FLAG_CHECK_WRITE_SLOTS = 1 /* kv_append verifies that write slots are pairwise disjoint */
+  VOSTI_FLAG_CHECK_WRITE_SLOTS = 1, /* kv_append verifies that write slots are pairwise disjoint */
+  /* Shared-prefix row packing, a scheduling decision that cannot change a bit
+   * (Sec. "Separate cache reuse from generation": requests that reuse a cached
+   * prefix name the same physical pages).  Among the split-parallel requests of
+   * a call (decode, speculative), rows of different requests whose block tables
+   * hold the same 32 page ids for a whole 512-key split that lies wholly below
+   * their positions are packed 16 to an MMA tile: the split is fetched and
+   * multiplied once per 16 rows instead of once per request.  Every row still
+   * receives its own partial (m, z, U) for that split, computed from the same
+   * keys in the same order, and the fold is unchanged, so outputs are bitwise
+   * those of the unpacked schedule (tested by comparing the two).  Applies when
+   * window == 0. */
+  VOSTI_FLAG_PACK_SHARED_SPLITS = 2
 };
 
 /* The fixed deployment configuration (Sec. "Fixed kernel choices": tile
@@ -261,6 +273,13 @@ vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* 
 
 /* Kernels launched through this context since creation. */
 int64_t vosti_launch_count(const vosti_ctx* ctx);
+
+/* The schedule of the last attention call of this context: split-parallel work
+ * items (packed ones included), how many of them are packed items (shared-split
+ * packing, VOSTI_FLAG_PACK_SHARED_SPLITS), and 256-row tile items.  Any pointer
+ * may be NULL.  Host-side bookkeeping only. */
+vosti_status vosti_last_schedule(const vosti_ctx* ctx, int64_t* split_items, int64_t* packed_items,
+                                 int64_t* tile_items);
 
 /* Hash of the frozen numerics (tile size, split length, fold and exponent
  * rules, library version): the paper's deployment identity W.  ctx may be

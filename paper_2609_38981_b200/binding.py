@@ -25,11 +25,13 @@ _lib = ctypes.CDLL(LIB_PATH)
 VOSTI_OK, VOSTI_ERR_INVALID_ARG, VOSTI_ERR_UNSUPPORTED_CONFIG, VOSTI_ERR_OUT_OF_RANGE, \
     VOSTI_ERR_WORKSPACE, VOSTI_ERR_CUDA, VOSTI_ERR_TIMEOUT = range(7)
 VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
+VOSTI_FLAG_PACK_SHARED_SPLITS = 2
 
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
     "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
-    "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count", "vosti_fingerprint",
+    "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
+    "vosti_last_schedule", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
 )
 
@@ -97,6 +99,9 @@ _lib.vosti_profile_read.argtypes = [_vp, ctypes.POINTER(ctypes.c_double),
                                     ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_launch_count.restype = ctypes.c_int64
 _lib.vosti_launch_count.argtypes = [_vp]
+_lib.vosti_last_schedule.restype = ctypes.c_int
+_lib.vosti_last_schedule.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64),
+                                     ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_fingerprint.restype = ctypes.c_uint64
 _lib.vosti_fingerprint.argtypes = [_vp]
 _lib.vosti_constants.restype = None
@@ -315,6 +320,14 @@ def vosti_profile_read(ctx: Context):
     _check(_lib.vosti_profile_read(ctx.handle, ctypes.byref(ms), ctypes.byref(n)),
            "vosti_profile_read")
     return ms.value, n.value
+
+
+def vosti_last_schedule(ctx: "Context"):
+    """(split-parallel items, packed items among them, tile items) of the last attention call."""
+    a, b, c = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.vosti_last_schedule(ctx.handle, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c)),
+           "vosti_last_schedule")
+    return a.value, b.value, c.value
 
 
 def vosti_launch_count(ctx: Context) -> int:

@@ -86,11 +86,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     }
     if (t >= static_cast<uint32_t>(P.n_workers)) return false;
     const SplitItem si = read_item(t);
-    const int last_tok = min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
-    const int t_end = min((si.split + 1) * TPS, (si.start + last_tok) / nc::kKeyTile + 1);
-    // under a sliding window the group's first row needs nothing before this tile
-    const int first_tok = (si.row_group * nc::kRowsPerGroup) / G;
-    const int t_first = nc::first_key(si.start + first_tok, P.window) / nc::kKeyTile;
+    int t_end, t_first;
+    if (si.req < 0) {  // packed rows: every row sees the whole split
+      t_end = (si.split + 1) * TPS;
+      t_first = 0;
+    } else {
+      const int last_tok = min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
+      t_end = min((si.split + 1) * TPS, (si.start + last_tok) / nc::kKeyTile + 1);
+      // under a sliding window the group's first row needs nothing before this tile
+      const int first_tok = (si.row_group * nc::kRowsPerGroup) / G;
+      t_first = nc::first_key(si.start + first_tok, P.window) / nc::kKeyTile;
+    }
     d.ticket = t;
     d.kvh = static_cast<int>(t % P.Hkv);
     d.split_tile0 = si.split * TPS;
@@ -162,30 +168,61 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     // ---- consumer set-up for `cur` -----------------------------------------------
     const SplitItem si = read_item(cur.ticket);
     const int kvh = cur.kvh;
-    const int row_a = si.row_group * nc::kRowsPerGroup + (lane >> 2);
-    const int row_b = row_a + 8;
-    const int tok_a = row_a / G, tok_b = row_b / G;
-    const bool valid_a = tok_a < si.q_len, valid_b = tok_b < si.q_len;
+    // The warp's 16 rows: a row group of one request, or packed rows of several requests.
+    const bool packed = si.req < 0;
+    bool valid_a, valid_b, upper_rows;
+    const __nv_bfloat16 *q_a, *q_b;
+    int64_t out_a, out_b;  // partial rows the two rows write
+    int n_eff, p_min, lo_top, lo_first;
     RowPair r;
-    r.p_a = valid_a ? si.start + tok_a : -1;
-    r.p_b = valid_b ? si.start + tok_b : -1;
-    r.lo_a = nc::window_lo(r.p_a, P.window);
-    r.lo_b = nc::window_lo(r.p_b, P.window);
+    if (packed) {
+      const int ra = lane >> 2, rb = ra + 8;
+      valid_a = ra < si.q_len;
+      valid_b = rb < si.q_len;
+      const int4* rows = reinterpret_cast<const int4*>(P.packed_rows) + static_cast<size_t>(-1 - si.req) * 16;
+      const int4 da = __ldg(rows + (valid_a ? ra : 0)), db = __ldg(rows + (valid_b ? rb : 0));
+      r.p_a = valid_a ? da.y : -1;
+      r.p_b = valid_b ? db.y : -1;
+      r.lo_a = r.lo_b = nc::kNoLowerBound;
+      q_a = P.q + (static_cast<size_t>(da.x & 0xffffff) * P.Hq + kvh * G + (da.x >> 24)) * D;
+      q_b = P.q + (static_cast<size_t>(db.x & 0xffffff) * P.Hq + kvh * G + (db.x >> 24)) * D;
+      out_a = valid_a ? da.z + static_cast<int64_t>(kvh) * da.w : -1;
+      out_b = valid_b ? db.z + static_cast<int64_t>(kvh) * db.w : -1;
+      n_eff = 0x7fffffff;                           // a complete split: no tail to clear
+      p_min = (si.split + 1) * nc::kSplitLen;       // every key of the split is visible to every row
+      lo_top = lo_first = nc::kNoLowerBound;
+      upper_rows = si.q_len > 8;
+    } else {
+      const int row_a = si.row_group * nc::kRowsPerGroup + (lane >> 2);
+      const int row_b = row_a + 8;
+      const int tok_a = row_a / G, tok_b = row_b / G;
+      valid_a = tok_a < si.q_len;
+      valid_b = tok_b < si.q_len;
+      r.p_a = valid_a ? si.start + tok_a : -1;
+      r.p_b = valid_b ? si.start + tok_b : -1;
+      r.lo_a = nc::window_lo(r.p_a, P.window);
+      r.lo_b = nc::window_lo(r.p_b, P.window);
+      q_a = P.q + (static_cast<size_t>(si.q_row0 + tok_a) * P.Hq + kvh * G + row_a % G) * D;
+      q_b = P.q + (static_cast<size_t>(si.q_row0 + tok_b) * P.Hq + kvh * G + row_b % G) * D;
+      // partial (m, z, U) rows of this split, written only by rows that see some of it
+      const int64_t slab = si.part_base + (static_cast<int64_t>(kvh) * si.n_splits + (si.split - si.first_split)) *
+                                              (static_cast<int64_t>(si.q_len) * G);
+      const int first_key = si.split * nc::kSplitLen, last_key = first_key + nc::kSplitLen - 1;
+      out_a = (valid_a && r.p_a >= first_key && r.lo_a < last_key) ? slab + row_a : -1;
+      out_b = (valid_b && r.p_b >= first_key && r.lo_b < last_key) ? slab + row_b : -1;
+      n_eff = si.start + si.q_len;
+      // schedule-only facts about the group: lowest and highest real position (a tile between the
+      // highest row's window start and the lowest row's position is visible to every real row),
+      // and whether rows 8..15 hold real rows
+      p_min = si.start + (si.row_group * nc::kRowsPerGroup) / G;
+      const int p_top = si.start + min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
+      lo_top = nc::window_lo(p_top, P.window);
+      lo_first = nc::window_lo(p_min, P.window);  // keys up to here are invisible to the whole group
+      upper_rows = (si.row_group * nc::kRowsPerGroup + 8) / G < si.q_len;
+    }
     r.reset();
-    const int n_eff = si.start + si.q_len;
-    // schedule-only facts about the group: lowest and highest real position (a tile between the
-    // highest row's window start and the lowest row's position is visible to every real row),
-    // and whether rows 8..15 hold real rows
-    const int p_min = si.start + (si.row_group * nc::kRowsPerGroup) / G;
-    const int p_top = si.start + min(si.q_len - 1, (si.row_group * nc::kRowsPerGroup + 15) / G);
-    const int lo_top = nc::window_lo(p_top, P.window);
-    const int lo_first = nc::window_lo(p_min, P.window);  // keys up to here are invisible to the whole group
-    const bool upper_rows = (si.row_group * nc::kRowsPerGroup + 8) / G < si.q_len;
     uint32_t qa[C::KC][4];
-    load_q_frags<D>(qa,
-                    P.q + (static_cast<size_t>(si.q_row0 + tok_a) * P.Hq + kvh * G + row_a % G) * D,
-                    P.q + (static_cast<size_t>(si.q_row0 + tok_b) * P.Hq + kvh * G + row_b % G) * D,
-                    valid_a, valid_b, quad);
+    load_q_frags<D>(qa, q_a, q_b, valid_a, valid_b, quad);
     float u[C::NE][4];
 #pragma unroll
     for (int e = 0; e < C::NE; ++e) u[e][0] = u[e][1] = u[e][2] = u[e][3] = 0.f;
@@ -237,25 +274,17 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     if (timed_out) break;
 
     // ---- partial (m, z, U) of this split for the rows that see it -----------------
-    {
-      const int rows = si.q_len * G;
-      const int64_t slab =
-          si.part_base + (static_cast<int64_t>(kvh) * si.n_splits + (si.split - si.first_split)) * rows;
-      const int first_key = si.split * nc::kSplitLen, last_key = first_key + nc::kSplitLen - 1;
-      if (valid_a && r.p_a >= first_key && r.lo_a < last_key) {
-        float* dst = P.ws_u + (slab + row_a) * D + 2 * quad;
+    if (out_a >= 0) {
+      float* dst = P.ws_u + out_a * D + 2 * quad;
 #pragma unroll
-        for (int e = 0; e < C::NE; ++e)
-          *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][0], u[e][1]);
-        if (quad == 0) P.ws_mz[slab + row_a] = make_float2(r.m_a, r.z_a);
-      }
-      if (valid_b && r.p_b >= first_key && r.lo_b < last_key) {
-        float* dst = P.ws_u + (slab + row_b) * D + 2 * quad;
+      for (int e = 0; e < C::NE; ++e) *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][0], u[e][1]);
+      if (quad == 0) P.ws_mz[out_a] = make_float2(r.m_a, r.z_a);
+    }
+    if (out_b >= 0) {
+      float* dst = P.ws_u + out_b * D + 2 * quad;
 #pragma unroll
-        for (int e = 0; e < C::NE; ++e)
-          *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][2], u[e][3]);
-        if (quad == 0) P.ws_mz[slab + row_b] = make_float2(r.m_b, r.z_b);
-      }
+      for (int e = 0; e < C::NE; ++e) *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][2], u[e][3]);
+      if (quad == 0) P.ws_mz[out_b] = make_float2(r.m_b, r.z_b);
     }
 
     if (!has_nxt) break;

@@ -27,17 +27,28 @@ struct SplitItem {
   int32_t bt_index;  // index in the flat table of the first page of this split
   int32_t split, row_group, n_splits;
   int64_t part_base;
-  int32_t req;
+  int32_t req;          // < 0: packed item (rows from packed_rows[16 * (-1 - req) ...], q_len = rows in use)
   int32_t first_split;  // of the request: partial slabs are indexed by split - first_split
 };
 static_assert(sizeof(SplitItem) == 48, "SplitItem is read as three 16-byte words");
+
+// One row of a packed split item: rows of different requests whose block tables name the
+// same physical pages for a whole split share one 16-row MMA tile, so the split is read
+// once for all of them.  16 bytes; a packed item owns 16 consecutive entries.
+struct PackedRow {
+  int32_t q_row_g;     // packed query token row (low 24 bits) and head within the KV group (high 8 bits)
+  int32_t p;           // logical position of the row
+  int32_t slab_row;    // partial row for KV head 0: part_base + split * rows + row of the request
+  int32_t kvh_stride;  // partial rows between consecutive KV heads of the request: n_splits * rows
+};
 
 struct AttnParams {
   const __nv_bfloat16* q;
   __nv_bfloat16* out;
   const ReqMeta* reqs;
   const vosti_work_item* items;    // sequential items
-  const SplitItem* split_items;    // split-parallel items, longest first
+  const SplitItem* split_items;    // split-parallel items, longest first; req < 0: packed item -1 - req
+  const PackedRow* packed_rows;    // 16 per packed item
   uint32_t* ticket;                // next split-parallel worker index (self-resetting)
   uint32_t* done;                  // warps that have left the persistent kernel
   const int32_t* bt_flat;

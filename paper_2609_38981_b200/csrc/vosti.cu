@@ -58,7 +58,10 @@ Limits limits_of(const vosti_config& c) {
   const int64_t rows_by_batch = int64_t{c.max_batch} * nc::kSplitRowsMax;
   const int64_t rows_by_total = c.max_total_q * G;
   L.part_rows_max = std::min(rows_by_batch, rows_by_total) * c.n_kv_heads * L.k_max;
-  const size_t attn_blob = align_up(sizeof(ReqMeta) * c.max_batch, 16) +
+  // packed rows (shared-split packing only): 16 per packed item, and packing never adds items
+  const int64_t packed_rows_max = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) ? 16 * items_split : 0;
+  const size_t attn_blob = align_up(sizeof(PackedRow) * packed_rows_max, 16) +
+                           align_up(sizeof(ReqMeta) * c.max_batch, 16) +
                            align_up(sizeof(SplitItem) * items_split, 16) +
                            align_up(sizeof(vosti_work_item) * items_seq, 16) +
                            align_up(sizeof(int32_t) * L.pages_max, 16) +
@@ -81,6 +84,12 @@ Limits limits_of(const vosti_config& c) {
   L.total = at;
   return L;
 }
+
+// A (request, complete split) pair that could share its split with other requests.
+struct PackCand {
+  uint64_t key;  // from the split's index and its first and last page id
+  int32_t req, split;
+};
 
 struct Plan {
   std::vector<vosti_work_item> items;  // split-parallel items first
@@ -239,6 +248,10 @@ struct vosti_ctx {
   int64_t launches = 0;
   Plan plan;                       // reused across calls: no allocation in steady state
   std::vector<int64_t> part_base;
+  std::vector<PackCand> cands;     // shared-split packing scratch
+  std::vector<int64_t> pk_off;     // per request: first entry of its complete splits in pk_mark
+  std::vector<uint8_t> pk_mark;    // 1: the (request, split) pair is served by packed items
+  int64_t last_split_items = 0, last_packed_items = 0, last_tile_items = 0;  // schedule of the last attention call
   // profiling of the dominant kernel
   int profile_mode = 0;
   std::vector<cudaEvent_t> ev_start, ev_stop;
@@ -684,10 +697,107 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
     if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
   }
   at += align_up(sizeof(int32_t) * bt_used, 16);
+
+  // ---- shared-split packing (scheduling only) ---------------------------------------------
+  // Candidates: complete splits (all 512 keys below every row of the request) of split-parallel
+  // requests.  Requests whose 32 page ids of a split agree form a group; the rows of a group of
+  // two or more are laid out 16 to a packed item.  Packed items come first in the item list
+  // (they walk a whole split: the longest kind), the others follow in plan order.
+  int64_t n_split_final = 0, n_packed_items = 0;
+  size_t off_packed = 0;
+  std::vector<int64_t>& pk_off = ctx->pk_off;
+  std::vector<uint8_t>& pk_mark = ctx->pk_mark;
+  const bool packing = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) && window == 0 && plan.n_split > 1 &&
+                       plan.n_partial_rows < (int64_t{1} << 31) && row0 < (int64_t{1} << 24) && G <= 128;
+  if (packing) {
+    std::vector<PackCand>& cands = ctx->cands;
+    cands.clear();
+    pk_off.assign(static_cast<size_t>(batch) + 1, 0);
+    for (int r = 0; r < batch; ++r) {
+      const ReqMeta& m = reqs[r];
+      const int64_t complete =
+          (m.q_len > 0 && int64_t{m.q_len} * G <= nc::kSplitRowsMax) ? m.start / nc::kSplitLen : 0;
+      pk_off[r + 1] = pk_off[r] + complete;
+      for (int64_t k = 0; k < complete; ++k) {
+        const int32_t* ids = bt_flat + m.bt_off + k * nc::kPagesPerSplit;
+        // Grouping key: the split index with its first and last page id.  Two requests that share
+        // the whole split agree on it; agreement on all 32 ids is checked when groups are formed.
+        const uint64_t key = ((static_cast<uint64_t>(static_cast<uint32_t>(ids[0])) << 32) |
+                              static_cast<uint32_t>(ids[nc::kPagesPerSplit - 1])) * 0x9E3779B97F4A7C15ull +
+                             static_cast<uint64_t>(k);
+        cands.push_back({key, r, static_cast<int32_t>(k)});
+      }
+    }
+    pk_mark.assign(static_cast<size_t>(pk_off[batch]), 0);
+    std::sort(cands.begin(), cands.end(), [](const PackCand& a, const PackCand& b) {
+      return a.key != b.key ? a.key < b.key : a.req < b.req;
+    });
+    off_packed = at;
+    PackedRow* packed_rows = reinterpret_cast<PackedRow*>(blob + at);
+    auto same_pages = [&](const PackCand& a, const PackCand& b) {
+      return a.split == b.split &&
+             std::memcmp(bt_flat + reqs[a.req].bt_off + int64_t{a.split} * nc::kPagesPerSplit,
+                         bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
+                         sizeof(int32_t) * nc::kPagesPerSplit) == 0;
+    };
+    for (size_t lo = 0; lo < cands.size();) {
+      size_t hi = lo + 1;
+      while (hi < cands.size() && cands[hi].key == cands[lo].key) ++hi;
+      // members: the very same split and page ids as the first (a hash collision stays unpacked)
+      // and packing must save tiles: fewer 16-row tiles together than one request at a time
+      int members = 0;
+      int64_t rows_together = 0, tiles_apart = 0;
+      for (size_t i = lo; i < hi; ++i)
+        if (same_pages(cands[i], cands[lo])) {
+          const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
+          ++members;
+          rows_together += rows;
+          tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+        }
+      if (members >= 2 && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup < tiles_apart) {
+        const ReqMeta& first = reqs[cands[lo].req];
+        int in_item = 0;
+        auto close_item = [&]() {
+          PackedRow* rows16 = packed_rows + n_packed_items * 16;
+          for (int i = in_item; i < 16; ++i) rows16[i] = PackedRow{0, -1, 0, 0};
+          SplitItem& si = split_items[n_split_final++];
+          si = SplitItem{};
+          si.q_len = in_item;  // rows in use
+          si.n_pages = first.n_pages;
+          si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
+          si.split = cands[lo].split;
+          si.req = static_cast<int32_t>(-1 - n_packed_items);
+          ++n_packed_items;
+          in_item = 0;
+        };
+        for (size_t i = lo; i < hi; ++i) {
+          if (!same_pages(cands[i], cands[lo])) continue;
+          const ReqMeta& m = reqs[cands[i].req];
+          const int k = cands[i].split;
+          pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
+          const int rows = m.q_len * G;
+          for (int row = 0; row < rows; ++row) {
+            PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
+            pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
+            pr.p = m.start + row / G;
+            pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
+            pr.kvh_stride = m.n_splits * rows;
+            if (++in_item == 16) close_item();
+          }
+        }
+        if (in_item > 0) close_item();
+      }
+      lo = hi;
+    }
+    at += align_up(sizeof(PackedRow) * 16 * n_packed_items, 16);
+  }
   for (int64_t i = 0; i < plan.n_split; ++i) {
     const vosti_work_item& it = plan.items[i];
     const ReqMeta& m = reqs[it.req];
-    SplitItem& si = split_items[i];
+    if (n_packed_items > 0 && int64_t{it.split_begin} < pk_off[it.req + 1] - pk_off[it.req] &&
+        pk_mark[static_cast<size_t>(pk_off[it.req] + it.split_begin)])
+      continue;  // served by packed items
+    SplitItem& si = split_items[n_split_final++];
     si.q_row0 = m.q_row0;
     si.q_len = m.q_len;
     si.start = m.start;
@@ -721,6 +831,7 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
   p.reqs = reinterpret_cast<const ReqMeta*>(dmeta + off_reqs);
   p.items = reinterpret_cast<const vosti_work_item*>(dmeta + off_items);
   p.split_items = reinterpret_cast<const SplitItem*>(dmeta + off_split);
+  p.packed_rows = reinterpret_cast<const PackedRow*>(dmeta + off_packed);
   p.ticket = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 64);
   p.done = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 128);
   p.bt_flat = reinterpret_cast<const int32_t*>(dmeta + off_bt);
@@ -737,8 +848,11 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
   p.window = window;
   p.lse = lse;
-  st = c.head_dim == 128 ? launch_attention<128>(ctx, p, plan.n_split, n_seq, stream)
-                         : launch_attention<64>(ctx, p, plan.n_split, n_seq, stream);
+  ctx->last_split_items = n_split_final;
+  ctx->last_packed_items = n_packed_items;
+  ctx->last_tile_items = n_seq;
+  st = c.head_dim == 128 ? launch_attention<128>(ctx, p, n_split_final, n_seq, stream)
+                         : launch_attention<64>(ctx, p, n_split_final, n_seq, stream);
   if (st != VOSTI_OK) return st;
   return release_slot(slot, stream);
 }
@@ -826,5 +940,14 @@ vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* 
 }
 
 int64_t vosti_launch_count(const vosti_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+vosti_status vosti_last_schedule(const vosti_ctx* ctx, int64_t* split_items, int64_t* packed_items,
+                                 int64_t* tile_items) {
+  if (!ctx) return VOSTI_ERR_INVALID_ARG;
+  if (split_items) *split_items = ctx->last_split_items;
+  if (packed_items) *packed_items = ctx->last_packed_items;
+  if (tile_items) *tile_items = ctx->last_tile_items;
+  return VOSTI_OK;
+}
 
 }  // extern "C"
