@@ -8,8 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvosti.so")
-SOURCES = ["vosti.cu", "vosti_noalloc.cu"]
-HEADERS = ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", os.path.join("..", "..", "include", "vosti.h")]
+SOURCES = ["vosti.cu", "vosti_noalloc.cu", "prefix_cache.cpp"]
+HEADERS = ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", os.path.join("..", "..", "include", "vosti.h"),
+           os.path.join("..", "..", "include", "vosti_cache.h")]
 
 
 def _stale() -> bool:
@@ -25,8 +26,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "--use_fast_math=false" if False else "-Xcompiler", "-O2",
-           "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+           "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-O2", "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

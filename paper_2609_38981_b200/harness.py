@@ -41,6 +41,13 @@ class DeviceCache:
             pool = pat.repeat((n + 3) // 4)[:n].view(torch.bfloat16).reshape(shape).contiguous()
         else:
             raise ValueError(pool_fill)
+        if pool.data_ptr() % 1024:  # the library wants the pool 1024-byte aligned; small torch blocks are not
+            n = pool.numel()
+            raw = torch.empty(n + 512, dtype=torch.bfloat16, device=self.device)
+            off = (-raw.data_ptr() % 1024) // 2
+            aligned = raw[off:off + n].view(shape)
+            aligned.copy_(pool)
+            pool = aligned
         self.pool = pool
         self.ctx = vb.vosti_create(geo.n_q_heads, geo.n_kv_heads, geo.head_dim, geo.page_size,
                                    pool, max_batch, max_total_q, max_seq_len, flags=flags)
