@@ -44,7 +44,7 @@ def parse_args():
     ap.add_argument("--impl", default="vosti", choices=["vosti", "reference"])
     ap.add_argument("--workload", default="decode_heavy",
                     choices=["decode_heavy", "prefix_sharing", "long_context_speculative",
-                             "mixed_chunked_prefill"])
+                             "mixed_chunked_prefill", "linear"])
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-events", action="store_true",
@@ -197,10 +197,73 @@ def run_reference(args):
     }))
 
 
+def run_linear(args):
+    """Side benchmark (not the headline metric): the batch-invariant linear layer on the four
+    weight shapes of a Llama-3.1-8B decoder layer at a prefill batch of 8192 token rows, with the
+    library GEMM (torch.matmul) timed beside it for context, and the decode batch of 64 rows."""
+    import torch
+    from paper_2609_38981_b200 import linear as vl
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        src = "measured (MEASURED_PEAKS.json bf16_tflops, burst)"
+    except Exception:
+        peak, src = 1590.0, "fallback"
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+
+    def timed(fn, n):
+        for _ in range(max(3, args.warmup)):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    shapes = {"qkv": (6144, 4096), "o": (4096, 4096), "gate_up": (28672, 4096), "down": (4096, 14336)}
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    rows, flops_all, ms_all, launches = {}, 0.0, 0.0, 0
+    n = max(10, min(args.steps, 100))
+    for M in (8192, 64):
+        for name, (N, K) in shapes.items():
+            x = torch.randn(M, K, device="cuda", generator=g).bfloat16()
+            w = (torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).bfloat16()
+            y = torch.empty(M, N, device="cuda", dtype=torch.bfloat16)
+            ms = timed(lambda: vl.vosti_linear(x, w, y), n)
+            ms_lib = timed(lambda: torch.matmul(x, w.t(), out=y), n)
+            launches += n + max(3, args.warmup)
+            fl = 2.0 * M * N * K
+            rows[f"{name}_M{M}"] = {"N": N, "K": K, "us": ms * 1e3, "tflops": fl / ms / 1e9,
+                                    "weight_gbs": N * K * 2 / ms / 1e6, "library_gemm_us": ms_lib * 1e3,
+                                    "tile": list(vl.vosti_linear_tile_shape(N, K))}
+            if M == 8192:
+                flops_all += fl
+                ms_all += ms
+    clocks = sampler.stop()
+    assert vl.vosti_linear_poll_status() == 0
+    ach = flops_all / ms_all / 1e9
+    print(json.dumps({
+        "metric": "batch-invariant linear TFLOP/s (Llama-3.1-8B layer weights, 8192 token rows)", "value": ach,
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": n, "warmup": max(3, args.warmup), "ms_per_step": ms_all,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "linear", "shapes": shapes, "l2": "operands of a layer exceed L2; no flush"},
+        "gpu_launches": launches, "clocks": clocks, "per_shape": rows,
+        "roofline": {"bound": "tensor", "kernel": "linear_kernel<256>", "achieved": ach, "peak": peak,
+                     "unit": "TFLOP/s", "frac": ach / peak, "peak_source": src, "traffic": None},
+    }))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "linear":
+        return run_linear(args)
 
     import numpy as np
     import torch

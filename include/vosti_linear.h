@@ -1,0 +1,58 @@
+/* vosti_linear.h -- batch-invariant linear layer and RMS normalisation for
+ * B200 (sm_100a), the two operators that surround attention in a decoder layer.
+ *
+ * Contract (Sec. "Relational Kernel Contracts", matmul): for activations x
+ * [M, K] (one token per row), fixed weights and an output row x_i W^T, the
+ * bits of that row are the same whether x_i runs alone (M = 1) or anywhere in
+ * a batch of any size; the other rows are unconstrained.  It holds because
+ * (Sec. "Relational Structural Analysis") the tile shape is a function of
+ * (N, K) only, never of M; every output tile starts from a zero fp32
+ * accumulator and accumulates its products over the whole K range in
+ * ascending order (chunks of 16, tcgen05.mma, no split over K); and a row of
+ * an MMA tile depends on its own operand row only.
+ *
+ * All tensors are bf16, row-major, in device memory, 16-byte aligned; fp32
+ * accumulation; round-to-nearest-even to bf16 at the end.  Kernels are
+ * enqueued on `cuda_stream`; nothing is allocated.  Every device-side wait is
+ * bounded: a kernel that gives up sets a status word read by
+ * vosti_linear_poll_status.
+ */
+#ifndef VOSTI_LINEAR_H_
+#define VOSTI_LINEAR_H_
+
+#include <stdint.h>
+
+#include "vosti.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* The tile shape used for an (N, K) weight: a pure host-side function of N and
+ * K (B_M = 128, B_K = 64, B_N = 256 when N is a multiple of 256, else 128).
+ * UNSUPPORTED_CONFIG unless N is a positive multiple of 128 and K of 64. */
+vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t* b_n, int32_t* b_k);
+
+/* y [M, N] = x [M, K] * w [N, K]^T (one weight row per output feature, as a
+ * linear layer stores it).  M >= 0 is free; M = 0 does nothing.
+ * Errors: INVALID_ARG (null or misaligned pointers, negative M),
+ * UNSUPPORTED_CONFIG (see vosti_linear_tile_shape), CUDA. */
+vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
+                          void* cuda_stream);
+
+/* y [M, K] = x * rsqrt(mean_k(x^2) + eps) * weight [K], per row: the sum of
+ * squares is taken in a fixed order that depends on K only (each lane of the
+ * row's warp adds its 16-byte vectors in ascending order, lanes are combined by
+ * a butterfly), so a row's bits do not depend on M or on the row's place.
+ * K must be a multiple of 8.  y may alias x. */
+vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,
+                           void* cuda_stream);
+
+/* Waits for `cuda_stream` and reports whether a linear kernel gave up on a
+ * bounded wait since the last poll (VOSTI_ERR_TIMEOUT), clearing the word. */
+vosti_status vosti_linear_poll_status(void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VOSTI_LINEAR_H_ */

@@ -1,0 +1,334 @@
+// Batch-invariant linear layer (tcgen05.mma + TMA, persistent, warp-specialised)
+// and RMS normalisation for sm_100a: include/vosti_linear.h.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "../../include/vosti_linear.h"
+#include "ptx.cuh"
+#include "tcgen05.cuh"
+
+namespace vosti {
+namespace {
+
+__device__ uint32_t g_linear_status;  // bit 0: a bounded wait gave up
+
+template <int BN>
+struct LinearCfg {
+  static constexpr int kBM = 128, kBK = 64;
+  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static constexpr int kABytes = kBM * kBK * 2;   // [row][128 B], 128-byte swizzle
+  static constexpr int kBBytes = BN * kBK * 2;
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kThreads = 192;            // TMA warp, MMA warp, four epilogue warps
+  static constexpr int kSmemBytes = kStages * kStageBytes + 256 + 1024;
+  static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators: the epilogue of a tile overlaps the next tile's MMAs
+};
+
+// One CTA per SM walks output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...;
+// tile t covers rows 128 (t % m_tiles) and columns BN (t / m_tiles), so CTAs running
+// at the same time share a weight slab.  For every tile the K range is walked in
+// ascending 64-wide blocks, each as four K = 16 MMAs into a fresh accumulator.
+template <int BN>
+__global__ void __launch_bounds__(LinearCfg<BN>::kThreads, 1)
+linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
+              __nv_bfloat16* __restrict__ y, int M, int N, int K) {
+  using Cfg = LinearCfg<BN>;
+  constexpr int NS = Cfg::kStages;
+  constexpr uint32_t kAbortAfterNs = 1000000000u;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + NS * Cfg::kStageBytes;
+  const uint32_t full = bars, empty = bars + 8 * NS, acc_full = bars + 16 * NS, acc_empty = acc_full + 16;
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + NS * Cfg::kStageBytes + 192);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int m_tiles = (M + Cfg::kBM - 1) / Cfg::kBM;
+  const int n_tiles = m_tiles * (N / BN);
+  const int k_blocks = K / Cfg::kBK;
+
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(full + 8 * i, 1);
+      mbar_init(empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full + 8 * i, 1);
+      mbar_init(acc_empty + 8 * i, 128);
+    }
+    flags[0] = 0u;
+    mbar_fence_init();
+    tma_prefetch_desc(&x_map);
+    tma_prefetch_desc(&w_map);
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 200),
+                 "r"(Cfg::kTmemCols));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + NS * Cfg::kStageBytes + 200);
+
+  // Bounded wait: gives up after ~1 s or as soon as another thread of the CTA has given up.
+  auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 0;; ++it) {
+      if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+      if ((it & 63u) == 63u) {
+        if (flags[0] != 0u) return false;
+        if (global_timer_ns() - t0 > kAbortAfterNs) {
+          flags[0] = 1u;
+          atomicOr(&g_linear_status, 1u);
+          return false;
+        }
+      }
+    }
+  };
+
+  if (warp == 0) {
+    // ================= TMA producer ==========================================================
+    if (lane == 0) {
+      griddep_wait();
+      uint32_t it = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const int m0 = (t % m_tiles) * Cfg::kBM, n0 = (t / m_tiles) * BN;
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const uint32_t s = it % NS, use = it / NS;
+          if (use > 0) ok = wait(empty + 8 * s, (use - 1) & 1);
+          if (!ok) break;
+          const uint32_t dst = base + s * Cfg::kStageBytes;
+          mbar_expect_tx(full + 8 * s, Cfg::kStageBytes);
+          tma_load_2d(dst, &x_map, kb * Cfg::kBK, m0, full + 8 * s);           // rows beyond M arrive as zeros
+          tma_load_2d(dst + Cfg::kABytes, &w_map, kb * Cfg::kBK, n0, full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer ============================================================
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc(128, BN, false);
+      uint32_t it = 0, tile_i = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+        const uint32_t buf = tile_i & 1, acc_use = tile_i >> 1;
+        if (acc_use > 0) ok = wait(acc_empty + 8 * buf, (acc_use - 1) & 1);  // the epilogue has drained this accumulator
+        if (!ok) break;
+        tc_fence_after();
+        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
+          const uint32_t s = it % NS;
+          ok = wait(full + 8 * s, (it / NS) & 1);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t a = base + s * Cfg::kStageBytes, b = a + Cfg::kABytes;
+#pragma unroll
+          for (int kc = 0; kc < Cfg::kBK / 16; ++kc)
+            tc_mma_ss(tmem + buf * BN, smem_desc_sw128(a + kc * 32, 16, 1024), smem_desc_sw128(b + kc * 32, 16, 1024),
+                      idesc, (kb > 0 || kc > 0) ? 1u : 0u);
+          tc_commit(empty + 8 * s);
+        }
+        if (!ok) break;
+        tc_commit(acc_full + 8 * buf);
+      }
+    }
+  } else {
+    // ================= epilogue: one thread per row of the tile ================================
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int r = (warp & 3) * 32 + lane;
+    uint32_t tile_i = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
+      const uint32_t buf = tile_i & 1;
+      const int m0 = (t % m_tiles) * Cfg::kBM, n0 = (t / m_tiles) * BN;
+      ok = __all_sync(0xffffffffu, wait(acc_full + 8 * buf, (tile_i >> 1) & 1));
+      if (!ok) break;
+      tc_fence_after();
+      const bool in_range = m0 + r < M;
+      __nv_bfloat16* dst = y + static_cast<size_t>(m0 + r) * N + n0;
+#pragma unroll 1
+      for (int cb = 0; cb < BN; cb += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem + lane_sel + buf * BN + cb, v);
+        tmem_wait_ld();
+        if (cb + 32 == BN) {  // the accumulator is in registers: hand it back before the stores
+          tc_fence_before();
+          mbar_arrive(acc_empty + 8 * buf);
+        }
+        if (in_range) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint32_t o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[i + 2 * j]), __uint_as_float(v[i + 2 * j + 1]));
+              o[j] = *reinterpret_cast<uint32_t*>(&t2);
+            }
+            *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
+}
+
+// One warp per row.  Lane l adds the squares of its 8-element vectors l, l + 32, ... in
+// ascending order (elements of a vector in ascending order), the 32 partial sums are
+// combined by a butterfly (xor 16, 8, 4, 2, 1): the order depends on K only.
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const __nv_bfloat16* __restrict__ x,
+                                                      const __nv_bfloat16* __restrict__ w,
+                                                      __nv_bfloat16* __restrict__ y, int64_t M, int K, float eps) {
+  griddep_wait();
+  const int64_t row = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= M) return;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + row * K);
+  const uint4* wr = reinterpret_cast<const uint4*>(w);
+  uint4* yr = reinterpret_cast<uint4*>(y + row * K);
+  const int nv = K / 8;
+  float ss = 0.f;
+  for (int i = lane; i < nv; i += 32) {
+    const uint4 v = xr[i];
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u[j]));
+      ss = __fmaf_rn(f.x, f.x, ss);
+      ss = __fmaf_rn(f.y, f.y, ss);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss = __fadd_rn(ss, __shfl_xor_sync(0xffffffffu, ss, o));
+  const float inv = __frsqrt_rn(__fadd_rn(__fdiv_rn(ss, static_cast<float>(K)), eps));
+  for (int i = lane; i < nv; i += 32) {
+    const uint4 v = xr[i], g = wr[i];
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w}, gw[4] = {g.x, g.y, g.z, g.w};
+    uint32_t o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u[j]));
+      const float2 h = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw[j]));
+      __nv_bfloat162 t2 = __floats2bfloat162_rn(__fmul_rn(__fmul_rn(f.x, inv), h.x), __fmul_rn(__fmul_rn(f.y, inv), h.y));
+      o[j] = *reinterpret_cast<uint32_t*>(&t2);
+    }
+    yr[i] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// A [rows, K] bf16 row-major matrix as a 2-D tensor map with boxes of 64 columns x box_rows rows.
+bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int64_t rows, int64_t K, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
+                           int sm_count, cudaStream_t stream) {
+  using Cfg = LinearCfg<BN>;
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VOSTI_ERR_CUDA;
+  if (!attr_set[dev]) {
+    if (cudaFuncSetAttribute(linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
+        cudaSuccess)
+      return VOSTI_ERR_CUDA;
+    attr_set[dev] = true;
+  }
+  alignas(64) CUtensorMap x_map, w_map;
+  if (!make_map(fn, &x_map, x, M, K, Cfg::kBM) || !make_map(fn, &w_map, w, N, K, BN)) return VOSTI_ERR_CUDA;
+  const int64_t tiles = ((M + Cfg::kBM - 1) / Cfg::kBM) * (N / BN);
+  const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
+  linear_kernel<BN><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(x_map, w_map, static_cast<__nv_bfloat16*>(y),
+                                                                      static_cast<int>(M), static_cast<int>(N),
+                                                                      static_cast<int>(K));
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+}  // namespace
+}  // namespace vosti
+
+using namespace vosti;
+
+extern "C" {
+
+vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t* b_n, int32_t* b_k) {
+  if (N <= 0 || K <= 0 || N % 128 != 0 || K % 64 != 0 || N > INT32_MAX || K > INT32_MAX)
+    return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  if (b_m) *b_m = 128;
+  if (b_n) *b_n = N % 256 == 0 ? 256 : 128;
+  if (b_k) *b_k = 64;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* cuda_stream) {
+  int32_t bn = 0;
+  const vosti_status shape = vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr);
+  if (shape != VOSTI_OK) return shape;
+  if (M < 0 || M > INT32_MAX) return VOSTI_ERR_INVALID_ARG;
+  if (M == 0) return VOSTI_OK;
+  if (!x || !w || !y) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(y)) % 16)
+    return VOSTI_ERR_INVALID_ARG;
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !p)
+      return VOSTI_ERR_CUDA;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  int dev = 0, sm_count = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  return bn == 256 ? launch_linear<256>(fn, x, w, y, M, N, K, sm_count, stream)
+                   : launch_linear<128>(fn, x, w, y, M, N, K, sm_count, stream);
+}
+
+vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,
+                           void* cuda_stream) {
+  if (M < 0 || K <= 0 || K % 8 != 0 || K > INT32_MAX || !(eps >= 0.0f)) return VOSTI_ERR_INVALID_ARG;
+  if (M == 0) return VOSTI_OK;
+  if (!x || !weight || !y) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(weight) | reinterpret_cast<uintptr_t>(y)) % 16)
+    return VOSTI_ERR_INVALID_ARG;
+  const int64_t grid = (M + 7) / 8;
+  if (grid > INT32_MAX) return VOSTI_ERR_INVALID_ARG;
+  rmsnorm_kernel<<<static_cast<int>(grid), 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(weight),
+      static_cast<__nv_bfloat16*>(y), M, static_cast<int>(K), eps);
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+vosti_status vosti_linear_poll_status(void* cuda_stream) {
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0, zero = 0;
+  if (cudaStreamSynchronize(stream) != cudaSuccess ||
+      cudaMemcpyFromSymbol(&word, g_linear_status, sizeof word) != cudaSuccess ||
+      cudaMemcpyToSymbol(g_linear_status, &zero, sizeof zero) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  return (word & 1u) ? VOSTI_ERR_TIMEOUT : VOSTI_OK;
+}
+
+}  // extern "C"

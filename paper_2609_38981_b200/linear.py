@@ -1,0 +1,67 @@
+"""ctypes binding of the batch-invariant linear layer and RMS normalisation
+(``include/vosti_linear.h``): argument marshalling only."""
+from __future__ import annotations
+
+import ctypes
+
+import torch
+
+from . import binding as _vb
+
+_lib = _vb._lib
+_vp = ctypes.c_void_p
+
+EXPORTS = ("vosti_linear_tile_shape", "vosti_linear", "vosti_rmsnorm", "vosti_linear_poll_status")
+
+_lib.vosti_linear_tile_shape.restype = ctypes.c_int
+_lib.vosti_linear_tile_shape.argtypes = [ctypes.c_int64, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 3
+_lib.vosti_linear.restype = ctypes.c_int
+_lib.vosti_linear.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp]
+_lib.vosti_rmsnorm.restype = ctypes.c_int
+_lib.vosti_rmsnorm.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_float, _vp]
+_lib.vosti_linear_poll_status.restype = ctypes.c_int
+_lib.vosti_linear_poll_status.argtypes = [_vp]
+
+
+def vosti_linear_tile_shape(N: int, K: int):
+    """(B_M, B_N, B_K) for an (N, K) weight: a function of N and K only."""
+    v = [ctypes.c_int32() for _ in range(3)]
+    _vb._check(_lib.vosti_linear_tile_shape(int(N), int(K), *[ctypes.byref(x) for x in v]),
+               "vosti_linear_tile_shape")
+    return tuple(x.value for x in v)
+
+
+def _bf16_cuda(t: torch.Tensor, ndim: int) -> torch.Tensor:
+    assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.ndim == ndim
+    return t
+
+
+def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """y [M, N] = x [M, K] @ w [N, K]^T; tensors are CUDA bf16, contiguous."""
+    x, w = _bf16_cuda(x, 2), _bf16_cuda(w, 2)
+    M, K = x.shape
+    N = w.shape[0]
+    assert w.shape[1] == K
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
+    _bf16_cuda(y, 2)
+    assert y.shape == (M, N)
+    _vb._check(_lib.vosti_linear(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, _vb._stream(stream)),
+               "vosti_linear")
+    return y
+
+
+def vosti_rmsnorm(x: torch.Tensor, weight: torch.Tensor, eps: float, y: torch.Tensor = None,
+                  stream=None) -> torch.Tensor:
+    x, weight = _bf16_cuda(x, 2), _bf16_cuda(weight, 1)
+    M, K = x.shape
+    assert weight.shape == (K,)
+    if y is None:
+        y = torch.empty_like(x)
+    _vb._check(_lib.vosti_rmsnorm(_vb._dev(x), _vb._dev(weight), _vb._dev(y), M, K, float(eps),
+                                  _vb._stream(stream)), "vosti_rmsnorm")
+    return y
+
+
+def vosti_linear_poll_status(stream=None) -> int:
+    return int(_lib.vosti_linear_poll_status(_vb._stream(stream)))

@@ -35,6 +35,25 @@ def test_library_exports_every_declared_symbol(vb):
     assert sorted(vb.EXPORTS) == names
 
 
+def test_linear_header_symbols_and_tile_shape(vb):
+    """The linear layer's tile shape is a host-side function of (N, K) alone."""
+    from paper_2609_38981_b200 import linear as vl
+    text = open(os.path.join(ROOT, "include", "vosti_linear.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = sorted(set(re.findall(r"\b(vosti_[a-z_]+)\s*\(", text)))
+    lib = ctypes.CDLL(vb.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(vl.EXPORTS) == names
+    assert vl.vosti_linear_tile_shape(4096, 4096) == (128, 256, 64)
+    assert vl.vosti_linear_tile_shape(28672, 4096) == (128, 256, 64)
+    assert vl.vosti_linear_tile_shape(128, 64) == (128, 128, 64)
+    for N, K in ((0, 64), (100, 64), (128, 32), (128, 0)):
+        with pytest.raises(vb.VostiError) as e:
+            vl.vosti_linear_tile_shape(N, K)
+        assert e.value.status == vb.VOSTI_ERR_UNSUPPORTED_CONFIG
+
+
 def test_constants_and_fingerprint(vb):
     c = vb.vosti_constants()
     assert c == {"key_tile": 64, "split_len": 512, "rows_per_group": 16}
