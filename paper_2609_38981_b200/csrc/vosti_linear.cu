@@ -27,10 +27,24 @@ struct LinearCfg {
   static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators: the epilogue of a tile overlaps the next tile's MMAs
 };
 
-// One CTA per SM walks output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...;
-// tile t covers rows 128 (t % m_tiles) and columns BN (t / m_tiles), so CTAs running
-// at the same time share a weight slab.  For every tile the K range is walked in
-// ascending 64-wide blocks, each as four K = 16 MMAs into a fresh accumulator.
+// One CTA per SM walks output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  Tiles are
+// numbered in bands of 16 row tiles, column tile by column tile inside a band, so that the
+// CTAs running at the same time work on a block of about 16 x 9 tiles and both operands are
+// re-read from L2 rather than from HBM.  For every tile the K range is walked in ascending
+// 64-wide blocks, each as four K = 16 MMAs into a fresh accumulator; the order in which tiles
+// are visited has no influence on any output bit.
+struct TileCoord {
+  int m0, n0;
+};
+template <int BM, int BN>
+__device__ __forceinline__ TileCoord tile_coord(int t, int m_tiles, int n_cols) {
+  constexpr int kBand = 16;
+  const int per_band = kBand * n_cols;
+  const int band = t / per_band, in_band = t - band * per_band;
+  const int first_m = band * kBand;
+  const int rows = min(kBand, m_tiles - first_m);
+  return TileCoord{(first_m + in_band % rows) * BM, (in_band / rows) * BN};
+}
 template <int BN>
 __global__ void __launch_bounds__(LinearCfg<BN>::kThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
@@ -97,7 +111,8 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
       uint32_t it = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-        const int m0 = (t % m_tiles) * Cfg::kBM, n0 = (t / m_tiles) * BN;
+        const TileCoord tc = tile_coord<Cfg::kBM, BN>(t, m_tiles, N / BN);
+        const int m0 = tc.m0, n0 = tc.n0;
         for (int kb = 0; kb < k_blocks; ++kb, ++it) {
           const uint32_t s = it % NS, use = it / NS;
           if (use > 0) ok = wait(empty + 8 * s, (use - 1) & 1);
@@ -144,7 +159,8 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
     bool ok = true;
     for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
       const uint32_t buf = tile_i & 1;
-      const int m0 = (t % m_tiles) * Cfg::kBM, n0 = (t / m_tiles) * BN;
+      const TileCoord tc = tile_coord<Cfg::kBM, BN>(t, m_tiles, N / BN);
+        const int m0 = tc.m0, n0 = tc.n0;
       ok = __all_sync(0xffffffffu, wait(acc_full + 8 * buf, (tile_i >> 1) & 1));
       if (!ok) break;
       tc_fence_after();
