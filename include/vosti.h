@@ -200,6 +200,36 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
                                       int32_t block_table_stride, int32_t batch, float softmax_scale,
                                       int32_t window, void* cuda_stream);
 
+/* Context-parallel decode (the paper's discussion of multi-GPU determinism,
+ * Sec. "Discussion": distributed KV must not change a request's bits).  The KV
+ * pages of a long request are spread over `cp_world` GPUs by split: split k
+ * (keys 512 k .. 512 k + 511) lives on rank k mod cp_world.  Each rank runs
+ *   vosti_cp_partial   -- the partial (m, z, U) of the splits it owns, from its
+ *                         own pool and block table (entries of other ranks'
+ *                         splits are not read); the slabs of all other splits
+ *                         are set to zero;
+ *   a sum over ranks   -- of the two workspace ranges this call reports
+ *                         (fp32; an all-reduce), which assembles every split's
+ *                         partial exactly (x + 0 = x; zeros may change sign,
+ *                         which the output rule absorbs);
+ *   vosti_cp_combine   -- the left fold over all splits and the output, on any
+ *                         rank that wants the result.
+ * The fold sees the same partials in the same order as a single-GPU call, so
+ * outputs and log-sum-exp are bitwise those of vosti_paged_attention.  Only
+ * split-parallel requests (q_len * group size <= 32: decode, speculative
+ * queries) are accepted (UNSUPPORTED_CONFIG otherwise); no sliding window.
+ * *u_offset / *u_bytes and *mz_offset / *mz_bytes are byte ranges inside the
+ * context's workspace; q and the three length arrays must be the same on every
+ * rank and in both calls. */
+vosti_status vosti_cp_partial(vosti_ctx* ctx, const void* q, const int32_t* q_lens,
+                              const int32_t* start_pos, const int32_t* seq_lens,
+                              const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
+                              float softmax_scale, int32_t cp_rank, int32_t cp_world, size_t* u_offset,
+                              size_t* u_bytes, size_t* mz_offset, size_t* mz_bytes, void* cuda_stream);
+vosti_status vosti_cp_combine(vosti_ctx* ctx, void* out, float* lse, const int32_t* q_lens,
+                              const int32_t* start_pos, const int32_t* seq_lens, int32_t batch,
+                              void* cuda_stream);
+
 /* One serving step from HOST buffers: copies q, k_new, v_new to the device,
  * runs vosti_kv_append then vosti_paged_attention, copies the output back
  * and waits for it.  Same arithmetic, same kernels; exists so that a caller

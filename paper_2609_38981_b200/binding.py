@@ -29,7 +29,8 @@ VOSTI_FLAG_PACK_SHARED_SPLITS = 2
 
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
-    "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_step_host", "vosti_poll_device_status",
+    "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_cp_partial",
+    "vosti_cp_combine", "vosti_step_host", "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
     "vosti_last_schedule", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
@@ -81,6 +82,12 @@ _lib.vosti_paged_attention.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p
 _lib.vosti_paged_attention_ex.restype = ctypes.c_int
 _lib.vosti_paged_attention_ex.argtypes = [_vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_float, ctypes.c_int32, _vp]
+_szp = ctypes.POINTER(ctypes.c_size_t)
+_lib.vosti_cp_partial.restype = ctypes.c_int
+_lib.vosti_cp_partial.argtypes = [_vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32,
+                                  ctypes.c_float, ctypes.c_int32, ctypes.c_int32, _szp, _szp, _szp, _szp, _vp]
+_lib.vosti_cp_combine.restype = ctypes.c_int
+_lib.vosti_cp_combine.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, ctypes.c_int32, _vp]
 _lib.vosti_paged_attention_noalloc.restype = ctypes.c_int
 _lib.vosti_paged_attention_noalloc.argtypes = [
     ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp, ctypes.c_int64, _vp, _vp,
@@ -275,6 +282,32 @@ def vosti_paged_attention_ex(ctx: Context, q, out, lse, q_lens, start_pos, seq_l
                                          _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1], len(ql),
                                          float(softmax_scale), int(window), _stream(stream)),
            "vosti_paged_attention_ex")
+
+
+def vosti_cp_partial(ctx: Context, q, q_lens, start_pos, seq_lens, block_tables, softmax_scale: float,
+                     cp_rank: int, cp_world: int, stream=None):
+    """Context-parallel phase 1.  Returns the two fp32 views of the context's workspace
+    (partial U rows, partial (m, z) pairs) that the caller sums over ranks in place."""
+    import torch
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    assert bt.ndim == 2 and bt.shape[0] == len(ql)
+    v = [ctypes.c_size_t() for _ in range(4)]
+    _check(_lib.vosti_cp_partial(ctx.handle, _dev(q), _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1], len(ql),
+                                 float(softmax_scale), int(cp_rank), int(cp_world),
+                                 *[ctypes.byref(x) for x in v], _stream(stream)), "vosti_cp_partial")
+    ws = ctx._keep[1]
+    assert ws.dtype == torch.uint8
+    u = ws[v[0].value:v[0].value + v[1].value].view(torch.float32)
+    mz = ws[v[2].value:v[2].value + v[3].value].view(torch.float32)
+    return u, mz
+
+
+def vosti_cp_combine(ctx: Context, out, lse, q_lens, start_pos, seq_lens, stream=None) -> None:
+    """Context-parallel phase 2: the fold over all splits (after the sum over ranks)."""
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    _check(_lib.vosti_cp_combine(ctx.handle, _dev(out), _dev(lse) if lse is not None else None, _ip(ql), _ip(s),
+                                 _ip(n), len(ql), _stream(stream)), "vosti_cp_combine")
 
 
 def vosti_paged_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_size, kv_pool, q, out,

@@ -356,7 +356,7 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size
 
 template <int D>
 vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_split, int64_t n_seq,
-                              cudaStream_t stream) {
+                              cudaStream_t stream, bool run_partials = true, bool run_combine = true) {
   using Cfg = SplitKernelCfg<D>;
   const int Hkv = ctx->cfg.n_kv_heads;
   const bool prof = ctx->profile_mode != 0;
@@ -376,7 +376,7 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
     if (rec) cudaEventRecord(ctx->ev_stop[ctx->ev_used++], stream);
     ++ctx->launches;
   };
-  if (n_split > 0) {
+  if (n_split > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_split * Hkv);
     // persistent: one CTA per SM, warps draw (item, KV head) tickets
@@ -385,7 +385,7 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
       launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3, p);
     });
   }
-  if (n_seq > 0) {
+  if (n_seq > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_seq * Hkv);
     using TileCfg_ = TileKernelCfg<D>;
@@ -395,12 +395,22 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
                        ctx->kv_map, p);
     });
   }
-  if (base.n_split_tokens > 0) {
+  if (base.n_split_tokens > 0 && run_combine) {
     const int warps = base.n_split_tokens * base.Hq;
     timed(3, [&] { launch_dependent(combine_kernel<D>, (warps + 3) / 4, 128, 0, stream, base); });
   }
   return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
 }
+
+// Context-parallel decode: phase 0 = everything on this GPU; phase 1 = the partials of the splits
+// this rank owns (split k belongs to rank k mod world); phase 2 = the fold over all splits.
+struct CpMode {
+  int phase = 0, rank = 0, world = 1;
+};
+vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse, const int32_t* q_lens,
+                            const int32_t* start_pos, const int32_t* seq_lens, const int32_t* block_tables,
+                            int32_t block_table_stride, int32_t batch, float softmax_scale, int32_t window,
+                            CpMode cp, void* cuda_stream);
 
 template <int D>
 vosti_status set_kernel_attributes() {
@@ -623,9 +633,49 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
                                       const int32_t* start_pos, const int32_t* seq_lens,
                                       const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
                                       float softmax_scale, int32_t window, void* cuda_stream) {
+  return attention_impl(ctx, q, out, lse, q_lens, start_pos, seq_lens, block_tables, block_table_stride, batch,
+                        softmax_scale, window, CpMode{}, cuda_stream);
+}
+
+vosti_status vosti_cp_partial(vosti_ctx* ctx, const void* q, const int32_t* q_lens, const int32_t* start_pos,
+                              const int32_t* seq_lens, const int32_t* block_tables, int32_t block_table_stride,
+                              int32_t batch, float softmax_scale, int32_t cp_rank, int32_t cp_world,
+                              size_t* u_offset, size_t* u_bytes, size_t* mz_offset, size_t* mz_bytes,
+                              void* cuda_stream) {
+  if (cp_world < 1 || cp_rank < 0 || cp_rank >= cp_world) return VOSTI_ERR_INVALID_ARG;
+  CpMode cp;
+  cp.phase = 1;
+  cp.rank = cp_rank;
+  cp.world = cp_world;
+  const vosti_status st = attention_impl(ctx, q, nullptr, nullptr, q_lens, start_pos, seq_lens, block_tables,
+                                         block_table_stride, batch, softmax_scale, 0, cp, cuda_stream);
+  if (st != VOSTI_OK) return st;
+  if (u_offset) *u_offset = ctx->lim.off_part_u;
+  if (u_bytes) *u_bytes = sizeof(float) * static_cast<size_t>(ctx->plan.n_partial_rows) * ctx->cfg.head_dim;
+  if (mz_offset) *mz_offset = ctx->lim.off_part_mz;
+  if (mz_bytes) *mz_bytes = sizeof(float2) * static_cast<size_t>(ctx->plan.n_partial_rows);
+  return VOSTI_OK;
+}
+
+vosti_status vosti_cp_combine(vosti_ctx* ctx, void* out, float* lse, const int32_t* q_lens,
+                              const int32_t* start_pos, const int32_t* seq_lens, int32_t batch, void* cuda_stream) {
+  CpMode cp;
+  cp.phase = 2;
+  return attention_impl(ctx, nullptr, out, lse, q_lens, start_pos, seq_lens, nullptr, 0, batch, 1.0f, 0, cp,
+                        cuda_stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse, const int32_t* q_lens,
+                            const int32_t* start_pos, const int32_t* seq_lens, const int32_t* block_tables,
+                            int32_t block_table_stride, int32_t batch, float softmax_scale, int32_t window,
+                            CpMode cp, void* cuda_stream) {
   if (!ctx || batch < 0 || block_table_stride < 0 || window < 0) return VOSTI_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
-  if (batch > 0 && !block_tables) return VOSTI_ERR_INVALID_ARG;
+  if (batch > 0 && !block_tables && cp.phase != 2) return VOSTI_ERR_INVALID_ARG;
   const vosti_config& c = ctx->cfg;
   Plan& plan = ctx->plan;
   std::vector<int64_t>& part_base = ctx->part_base;
@@ -633,7 +683,9 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
   vosti_status st = plan_requests(c, q_lens, start_pos, seq_lens, batch, window, &plan, part_base.data());
   if (st != VOSTI_OK) return st;
   if (plan.items.empty()) return VOSTI_OK;
-  if (!q || !out) return VOSTI_ERR_INVALID_ARG;
+  // context-parallel phases exist for split-parallel requests only (decode, speculative queries)
+  if (cp.phase != 0 && static_cast<int64_t>(plan.items.size()) != plan.n_split) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  if ((cp.phase != 2 && !q) || (cp.phase != 1 && !out)) return VOSTI_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16) return VOSTI_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(lse) % 4) return VOSTI_ERR_INVALID_ARG;
   if (static_cast<int64_t>(plan.items.size()) > ctx->lim.items_max ||
@@ -675,9 +727,16 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
     if (q_lens[r] == 0) continue;
     const int64_t n_eff = int64_t{start_pos[r]} + q_lens[r];
     const int64_t n_pages = (n_eff + c.page_size - 1) / c.page_size;
-    if (n_pages > block_table_stride ||
-        (int64_t{seq_lens[r]} + c.page_size - 1) / c.page_size > block_table_stride)
+    if (cp.phase != 2 && (n_pages > block_table_stride ||
+                          (int64_t{seq_lens[r]} + c.page_size - 1) / c.page_size > block_table_stride))
       return VOSTI_ERR_OUT_OF_RANGE;
+    if (cp.phase == 2) {  // the fold reads no pages
+      m.n_pages = static_cast<int32_t>(n_pages);
+      m.first_split = 0;
+      m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1);
+      if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
+      continue;
+    }
     const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
     // Pages that lie wholly before the window of the request's first row are never
     // visible: their table entries are not read (the caller may have freed them);
@@ -686,6 +745,11 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
     const int64_t first_page = first_key / c.page_size;
     for (int64_t b = 0; b < first_page; ++b) bt_flat[bt_used + b] = 0;
     for (int64_t b = first_page; b < n_pages; ++b) {
+      // a context-parallel rank holds (and names) only the pages of the splits it owns
+      if (cp.phase == 1 && (b / nc::kPagesPerSplit) % cp.world != cp.rank) {
+        bt_flat[bt_used + b] = 0;
+        continue;
+      }
       const int32_t page = row[b];
       if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
       bt_flat[bt_used + b] = page;
@@ -707,7 +771,7 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
   size_t off_packed = 0;
   std::vector<int64_t>& pk_off = ctx->pk_off;
   std::vector<uint8_t>& pk_mark = ctx->pk_mark;
-  const bool packing = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) && window == 0 && plan.n_split > 1 &&
+  const bool packing = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) && window == 0 && cp.phase == 0 && plan.n_split > 1 &&
                        plan.n_partial_rows < (int64_t{1} << 31) && row0 < (int64_t{1} << 24) && G <= 128;
   if (packing) {
     std::vector<PackCand>& cands = ctx->cands;
@@ -797,6 +861,7 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
     if (n_packed_items > 0 && int64_t{it.split_begin} < pk_off[it.req + 1] - pk_off[it.req] &&
         pk_mark[static_cast<size_t>(pk_off[it.req] + it.split_begin)])
       continue;  // served by packed items
+    if (cp.phase == 2 || (cp.phase == 1 && it.split_begin % cp.world != cp.rank)) continue;  // not this rank's split
     SplitItem& si = split_items[n_split_final++];
     si.q_row0 = m.q_row0;
     si.q_len = m.q_len;
@@ -851,11 +916,23 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
   ctx->last_split_items = n_split_final;
   ctx->last_packed_items = n_packed_items;
   ctx->last_tile_items = n_seq;
-  st = c.head_dim == 128 ? launch_attention<128>(ctx, p, n_split_final, n_seq, stream)
-                         : launch_attention<64>(ctx, p, n_split_final, n_seq, stream);
+  if (cp.phase == 1) {
+    // Slabs of splits other ranks own stay zero, so that a sum over ranks assembles all partials.
+    if (cudaMemsetAsync(p.ws_u, 0, sizeof(float) * static_cast<size_t>(plan.n_partial_rows) * c.head_dim, stream) !=
+            cudaSuccess ||
+        cudaMemsetAsync(p.ws_mz, 0, sizeof(float2) * static_cast<size_t>(plan.n_partial_rows), stream) != cudaSuccess)
+      return VOSTI_ERR_CUDA;
+  }
+  st = c.head_dim == 128
+           ? launch_attention<128>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1)
+           : launch_attention<64>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1);
   if (st != VOSTI_OK) return st;
   return release_slot(slot, stream);
 }
+
+}  // namespace
+
+extern "C" {
 
 vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
                              const void* v_new_host, const int32_t* q_lens, const int32_t* start_pos,
