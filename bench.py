@@ -234,13 +234,15 @@ def run_linear(args):
             x = torch.randn(M, K, device="cuda", generator=g).bfloat16()
             w = (torch.randn(N, K, device="cuda", generator=g) * K ** -0.5).bfloat16()
             y = torch.empty(M, N, device="cuda", dtype=torch.bfloat16)
-            ms = timed(lambda: vl.vosti_linear(x, w, y), n)
+            ws = torch.empty(max(vl.vosti_linear_workspace_bytes(M, N, K), 16), dtype=torch.uint8, device="cuda")
+            ms = timed(lambda: vl.vosti_linear(x, w, y, workspace=ws), n)
             ms_lib = timed(lambda: torch.matmul(x, w.t(), out=y), n)
             launches += n + max(3, args.warmup)
             fl = 2.0 * M * N * K
             rows[f"{name}_M{M}"] = {"N": N, "K": K, "us": ms * 1e3, "tflops": fl / ms / 1e9,
                                     "weight_gbs": N * K * 2 / ms / 1e6, "library_gemm_us": ms_lib * 1e3,
-                                    "tile": list(vl.vosti_linear_tile_shape(N, K))}
+                                    "tile": list(vl.vosti_linear_tile_shape(N, K)),
+                                    "k_segments": vl.vosti_linear_segments(N, K)}
             if M == 8192:
                 flops_all += fl
                 ms_all += ms

@@ -6,10 +6,15 @@
  * bits of that row are the same whether x_i runs alone (M = 1) or anywhere in
  * a batch of any size; the other rows are unconstrained.  It holds because
  * (Sec. "Relational Structural Analysis") the tile shape is a function of
- * (N, K) only, never of M; every output tile starts from a zero fp32
- * accumulator and accumulates its products over the whole K range in
- * ascending order (chunks of 16, tcgen05.mma, no split over K); and a row of
- * an MMA tile depends on its own operand row only.
+ * (N, K) only, never of M; the K range is cut into segments that depend on
+ * (N, K) only, every segment sum starts from a zero fp32 accumulator and takes
+ * its products in ascending order (chunks of 16, tcgen05.mma), and the segment
+ * sums are added left to right in fp32; and a row of an MMA tile depends on its
+ * own operand row only.  Whether one CTA walks all segments of a tile (large
+ * batches) or the segments of a tile are spread over CTAs and added by a second
+ * kernel (small batches, so that every SM streams a slice of the weight) is a
+ * scheduling decision that may depend on M: both compute the same sums in the
+ * same order.
  *
  * All tensors are bf16, row-major, in device memory, 16-byte aligned; fp32
  * accumulation; round-to-nearest-even to bf16 at the end.  Kernels are
@@ -33,12 +38,26 @@ extern "C" {
  * UNSUPPORTED_CONFIG unless N is a positive multiple of 128 and K of 64. */
 vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t* b_n, int32_t* b_k);
 
+/* The number of K segments of an (N, K) weight, a pure host-side function of N
+ * and K: ceil(148 / column tiles), at most K / 1024 and at least 1; segment j
+ * covers the 64-wide blocks [j B / n, (j + 1) B / n) of the B = K / 64 blocks. */
+vosti_status vosti_linear_segments(int64_t N, int64_t K, int32_t* n_segments);
+
+/* Bytes of device workspace that let vosti_linear spread the K segments of a
+ * tile over CTAs when M is small (one fp32 [M, N] slab per segment); 0 for an
+ * unsupported shape. */
+size_t vosti_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
 /* y [M, N] = x [M, K] * w [N, K]^T (one weight row per output feature, as a
  * linear layer stores it).  M >= 0 is free; M = 0 does nothing.
+ * workspace: device memory, 16-byte aligned, or NULL.  With at least
+ * vosti_linear_workspace_bytes(M, N, K) bytes the call may use the split
+ * schedule; without, it always walks whole tiles.  The output bits are the same
+ * either way.
  * Errors: INVALID_ARG (null or misaligned pointers, negative M),
  * UNSUPPORTED_CONFIG (see vosti_linear_tile_shape), CUDA. */
 vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
-                          void* cuda_stream);
+                          void* workspace, size_t workspace_bytes, void* cuda_stream);
 
 /* y [M, K] = x * rsqrt(mean_k(x^2) + eps) * weight [K], per row: the sum of
  * squares is taken in a fixed order that depends on K only (each lane of the

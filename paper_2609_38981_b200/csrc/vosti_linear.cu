@@ -22,17 +22,35 @@ struct LinearCfg {
   static constexpr int kABytes = kBM * kBK * 2;   // [row][128 B], 128-byte swizzle
   static constexpr int kBBytes = BN * kBK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
-  static constexpr int kThreads = 192;            // TMA warp, MMA warp, four epilogue warps
+  static constexpr int kEpiWarps = BN / 32;       // an epilogue thread owns 128 columns of one row
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;  // TMA warp, MMA warp, epilogue warps
   static constexpr int kSmemBytes = kStages * kStageBytes + 256 + 1024;
-  static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators: the epilogue of a tile overlaps the next tile's MMAs
+  static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators: the epilogue of a segment overlaps the next one's MMAs
 };
 
-// One CTA per SM walks output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  Tiles are
-// numbered in bands of 16 row tiles, column tile by column tile inside a band, so that the
-// CTAs running at the same time work on a block of about 16 x 9 tiles and both operands are
-// re-read from L2 rather than from HBM.  For every tile the K range is walked in ascending
-// 64-wide blocks, each as four K = 16 MMAs into a fresh accumulator; the order in which tiles
-// are visited has no influence on any output bit.
+// The K range of a weight is cut into `n_seg` segments of whole 64-wide blocks, a function of
+// (N, K) alone; segment j covers blocks [j * B / n_seg, (j + 1) * B / n_seg).
+struct Segments {
+  int n_seg, k_blocks;
+  __host__ __device__ int begin(int j) const { return static_cast<int>(static_cast<int64_t>(j) * k_blocks / n_seg); }
+};
+__host__ __device__ inline Segments segments_of(int64_t N, int64_t K, int bn) {
+  const int k_blocks = static_cast<int>(K / 64);
+  const int64_t col_tiles = N / bn;
+  // enough (column tile, segment) units for every SM of a B200 when the batch is a single row tile,
+  // but segments of at least 1024 elements: every segment costs the large-batch schedule a pass
+  // over the accumulator
+  int64_t want = (148 + col_tiles - 1) / col_tiles;
+  const int64_t cap = k_blocks / 16 > 0 ? k_blocks / 16 : 1;
+  if (want > cap) want = cap;
+  if (want < 1) want = 1;
+  return Segments{static_cast<int>(want), k_blocks};
+}
+
+// Tiles are numbered in bands of 16 row tiles, column tile by column tile inside a band, so that
+// the CTAs running at the same time work on a block of about 16 x 9 tiles and both operands are
+// re-read from L2 rather than from HBM.  The order in which tiles are visited has no influence
+// on any output bit.
 struct TileCoord {
   int m0, n0;
 };
@@ -45,10 +63,22 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int m_tiles, int n_cols) 
   const int rows = min(kBand, m_tiles - first_m);
   return TileCoord{(first_m + in_band % rows) * BM, (in_band / rows) * BN};
 }
-template <int BN>
+
+// The numerical contract of an output element: for each segment of K a sum s_j that starts from
+// a zero fp32 accumulator and takes the products in ascending K order (tcgen05.mma, K = 16 per
+// instruction); then t = s_0, t = t + s_j for j = 1, 2, ... in fp32, round to nearest; then
+// bf16(t).  Two schedules compute exactly that:
+//   SPLIT = false: one CTA per SM walks output tiles and, inside a tile, the segments in order;
+//     the epilogue threads keep t in registers and add each finished segment to it while the
+//     MMAs of the next segment run into the other tensor-memory accumulator.
+//   SPLIT = true (few row tiles, e.g. a decode batch): the unit of work is a (tile, segment)
+//     pair, so that every SM streams a slice of the weight; s_j goes to a workspace and
+//     linear_fold_kernel adds the segments in the same order.
+// Which one runs is a scheduling decision that may depend on M; the bits do not.
+template <int BN, bool SPLIT>
 __global__ void __launch_bounds__(LinearCfg<BN>::kThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
-              __nv_bfloat16* __restrict__ y, int M, int N, int K) {
+              __nv_bfloat16* __restrict__ y, float* __restrict__ seg_ws, int M, int N, int K) {
   using Cfg = LinearCfg<BN>;
   constexpr int NS = Cfg::kStages;
   constexpr uint32_t kAbortAfterNs = 1000000000u;
@@ -60,8 +90,23 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
   volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + NS * Cfg::kStageBytes + 192);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int m_tiles = (M + Cfg::kBM - 1) / Cfg::kBM;
-  const int n_tiles = m_tiles * (N / BN);
-  const int k_blocks = K / Cfg::kBK;
+  const int n_cols = N / BN;
+  const int n_tiles = m_tiles * n_cols;
+  const Segments seg = segments_of(N, K, BN);
+  // A step is one segment of one tile; a CTA's steps are numbered consecutively.  Without the
+  // split a CTA owns whole tiles (steps tile-major); with it, single (tile, segment) units.
+  const int n_units = SPLIT ? n_tiles * seg.n_seg : n_tiles;
+  auto step_of = [&](int unit, int j, int& tile, int& sj) {
+    if (SPLIT) {
+      tile = unit / seg.n_seg;
+      sj = unit - tile * seg.n_seg;
+    } else {
+      tile = unit;
+      sj = j;
+    }
+  };
+  constexpr int kStepsPerUnitSplit = 1;
+  const int steps_per_unit = SPLIT ? kStepsPerUnitSplit : seg.n_seg;
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -70,7 +115,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(acc_full + 8 * i, 1);
-      mbar_init(acc_empty + 8 * i, 128);
+      mbar_init(acc_empty + 8 * i, 32 * Cfg::kEpiWarps);
     }
     flags[0] = 0u;
     mbar_fence_init();
@@ -110,17 +155,20 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
       griddep_wait();
       uint32_t it = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
-        const TileCoord tc = tile_coord<Cfg::kBM, BN>(t, m_tiles, N / BN);
-        const int m0 = tc.m0, n0 = tc.n0;
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-          const uint32_t s = it % NS, use = it / NS;
-          if (use > 0) ok = wait(empty + 8 * s, (use - 1) & 1);
-          if (!ok) break;
-          const uint32_t dst = base + s * Cfg::kStageBytes;
-          mbar_expect_tx(full + 8 * s, Cfg::kStageBytes);
-          tma_load_2d(dst, &x_map, kb * Cfg::kBK, m0, full + 8 * s);           // rows beyond M arrive as zeros
-          tma_load_2d(dst + Cfg::kABytes, &w_map, kb * Cfg::kBK, n0, full + 8 * s);
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+        for (int j = 0; j < steps_per_unit && ok; ++j) {
+          int tile, sj;
+          step_of(unit, j, tile, sj);
+          const TileCoord tc = tile_coord<Cfg::kBM, BN>(tile, m_tiles, n_cols);
+          for (int kb = seg.begin(sj); kb < seg.begin(sj + 1); ++kb, ++it) {
+            const uint32_t s = it % NS, use = it / NS;
+            if (use > 0) ok = wait(empty + 8 * s, (use - 1) & 1);
+            if (!ok) break;
+            const uint32_t dst = base + s * Cfg::kStageBytes;
+            mbar_expect_tx(full + 8 * s, Cfg::kStageBytes);
+            tma_load_2d(dst, &x_map, kb * Cfg::kBK, tc.m0, full + 8 * s);  // rows beyond M arrive as zeros
+            tma_load_2d(dst + Cfg::kABytes, &w_map, kb * Cfg::kBK, tc.n0, full + 8 * s);
+          }
         }
       }
     }
@@ -128,63 +176,101 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
     // ================= MMA issuer ============================================================
     if (lane == 0) {
       constexpr uint32_t idesc = umma_idesc(128, BN, false);
-      uint32_t it = 0, tile_i = 0;
+      uint32_t it = 0, step = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
-        const uint32_t buf = tile_i & 1, acc_use = tile_i >> 1;
-        if (acc_use > 0) ok = wait(acc_empty + 8 * buf, (acc_use - 1) & 1);  // the epilogue has drained this accumulator
-        if (!ok) break;
-        tc_fence_after();
-        for (int kb = 0; kb < k_blocks; ++kb, ++it) {
-          const uint32_t s = it % NS;
-          ok = wait(full + 8 * s, (it / NS) & 1);
+      for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+        for (int j = 0; j < steps_per_unit && ok; ++j, ++step) {
+          int tile, sj;
+          step_of(unit, j, tile, sj);
+          const uint32_t buf = step & 1, acc_use = step >> 1;
+          if (acc_use > 0) ok = wait(acc_empty + 8 * buf, (acc_use - 1) & 1);  // the epilogue has drained this accumulator
           if (!ok) break;
           tc_fence_after();
-          const uint32_t a = base + s * Cfg::kStageBytes, b = a + Cfg::kABytes;
+          const int kb0 = seg.begin(sj), kb1 = seg.begin(sj + 1);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            const uint32_t s = it % NS;
+            ok = wait(full + 8 * s, (it / NS) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a = base + s * Cfg::kStageBytes, b = a + Cfg::kABytes;
 #pragma unroll
-          for (int kc = 0; kc < Cfg::kBK / 16; ++kc)
-            tc_mma_ss(tmem + buf * BN, smem_desc_sw128(a + kc * 32, 16, 1024), smem_desc_sw128(b + kc * 32, 16, 1024),
-                      idesc, (kb > 0 || kc > 0) ? 1u : 0u);
-          tc_commit(empty + 8 * s);
+            for (int kc = 0; kc < Cfg::kBK / 16; ++kc)
+              tc_mma_ss(tmem + buf * BN, smem_desc_sw128(a + kc * 32, 16, 1024),
+                        smem_desc_sw128(b + kc * 32, 16, 1024), idesc, (kb > kb0 || kc > 0) ? 1u : 0u);
+            tc_commit(empty + 8 * s);
+          }
+          if (!ok) break;
+          tc_commit(acc_full + 8 * buf);
         }
-        if (!ok) break;
-        tc_commit(acc_full + 8 * buf);
       }
     }
   } else {
-    // ================= epilogue: one thread per row of the tile ================================
+    // ================= epilogue: a thread owns 128 columns of one row of the tile ===============
+    const int e = warp - 2;
     const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const int r = (warp & 3) * 32 + lane;
-    uint32_t tile_i = 0;
+    const int r = (warp & 3) * 32 + lane;   // row of the tile = tensor-memory lane
+    const int c0 = (e >> 2) * 128;          // first of the thread's columns
+    float total[128];
+    uint32_t step = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile_i) {
-      const uint32_t buf = tile_i & 1;
-      const TileCoord tc = tile_coord<Cfg::kBM, BN>(t, m_tiles, N / BN);
-        const int m0 = tc.m0, n0 = tc.n0;
-      ok = __all_sync(0xffffffffu, wait(acc_full + 8 * buf, (tile_i >> 1) & 1));
-      if (!ok) break;
-      tc_fence_after();
-      const bool in_range = m0 + r < M;
-      __nv_bfloat16* dst = y + static_cast<size_t>(m0 + r) * N + n0;
+    for (int unit = blockIdx.x; unit < n_units && ok; unit += gridDim.x) {
+      for (int j = 0; j < steps_per_unit && ok; ++j, ++step) {
+        int tile, sj;
+        step_of(unit, j, tile, sj);
+        const uint32_t buf = step & 1;
+        const TileCoord tc = tile_coord<Cfg::kBM, BN>(tile, m_tiles, n_cols);
+        ok = __all_sync(0xffffffffu, wait(acc_full + 8 * buf, (step >> 1) & 1));
+        if (!ok) break;
+        tc_fence_after();
+        const bool in_range = tc.m0 + r < M;
+        if (SPLIT) {
+          // s_j of this unit -> workspace [column tile][segment][row][BN]
+          float* dst = seg_ws + ((static_cast<size_t>(tc.n0 / BN) * seg.n_seg + sj) * M + (tc.m0 + r)) * BN + c0;
 #pragma unroll 1
-      for (int cb = 0; cb < BN; cb += 32) {
-        uint32_t v[32];
-        tmem_ld32(tmem + lane_sel + buf * BN + cb, v);
-        tmem_wait_ld();
-        if (cb + 32 == BN) {  // the accumulator is in registers: hand it back before the stores
-          tc_fence_before();
-          mbar_arrive(acc_empty + 8 * buf);
-        }
-        if (in_range) {
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint32_t o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(v[i + 2 * j]), __uint_as_float(v[i + 2 * j + 1]));
-              o[j] = *reinterpret_cast<uint32_t*>(&t2);
+          for (int cb = 0; cb < 128; cb += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_sel + buf * BN + c0 + cb, v);
+            tmem_wait_ld();
+            if (cb + 32 == 128) {
+              tc_fence_before();
+              mbar_arrive(acc_empty + 8 * buf);
             }
-            *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(o[0], o[1], o[2], o[3]);
+            if (in_range) {
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<uint4*>(dst + cb + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int cb = 0; cb < 128; cb += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_sel + buf * BN + c0 + cb, v);
+            tmem_wait_ld();
+            if (cb + 32 == 128) {  // the accumulator is in registers: hand it back
+              tc_fence_before();
+              mbar_arrive(acc_empty + 8 * buf);
+            }
+            if (sj == 0) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) total[cb + i] = __uint_as_float(v[i]);
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i) total[cb + i] = __fadd_rn(total[cb + i], __uint_as_float(v[i]));
+            }
+          }
+          if (sj == seg.n_seg - 1 && in_range) {
+            __nv_bfloat16* dst = y + static_cast<size_t>(tc.m0 + r) * N + tc.n0 + c0;
+#pragma unroll
+            for (int i = 0; i < 128; i += 8) {
+              uint32_t o[4];
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                __nv_bfloat162 t2 = __floats2bfloat162_rn(total[i + 2 * q], total[i + 2 * q + 1]);
+                o[q] = *reinterpret_cast<uint32_t*>(&t2);
+              }
+              *reinterpret_cast<uint4*>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
           }
         }
       }
@@ -195,6 +281,37 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
   __syncthreads();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
+}
+
+// The second half of the split schedule: y = bf16(((s_0 + s_1) + s_2) + ...), eight columns per thread.
+__global__ void __launch_bounds__(256) linear_fold_kernel(const float* __restrict__ seg_ws,
+                                                          __nv_bfloat16* __restrict__ y, int M, int N, int bn,
+                                                          int n_seg) {
+  griddep_wait();
+  const int64_t idx = (static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x) * 8;
+  if (idx >= static_cast<int64_t>(M) * N) return;
+  const int m = static_cast<int>(idx / N), n = static_cast<int>(idx - static_cast<int64_t>(m) * N);
+  const int ct = n / bn, c = n - ct * bn;
+  const float* src = seg_ws + ((static_cast<size_t>(ct) * n_seg) * M + m) * bn + c;
+  const size_t seg_stride = static_cast<size_t>(M) * bn;
+  float t[8];
+  {
+    const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+    t[0] = a.x; t[1] = a.y; t[2] = a.z; t[3] = a.w; t[4] = b.x; t[5] = b.y; t[6] = b.z; t[7] = b.w;
+  }
+  for (int j = 1; j < n_seg; ++j) {
+    const float4 a = *reinterpret_cast<const float4*>(src + j * seg_stride);
+    const float4 b = *reinterpret_cast<const float4*>(src + j * seg_stride + 4);
+    t[0] = __fadd_rn(t[0], a.x); t[1] = __fadd_rn(t[1], a.y); t[2] = __fadd_rn(t[2], a.z); t[3] = __fadd_rn(t[3], a.w);
+    t[4] = __fadd_rn(t[4], b.x); t[5] = __fadd_rn(t[5], b.y); t[6] = __fadd_rn(t[6], b.z); t[7] = __fadd_rn(t[7], b.w);
+  }
+  uint32_t o[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    __nv_bfloat162 t2 = __floats2bfloat162_rn(t[2 * q], t[2 * q + 1]);
+    o[q] = *reinterpret_cast<uint32_t*>(&t2);
+  }
+  *reinterpret_cast<uint4*>(y + idx) = make_uint4(o[0], o[1], o[2], o[3]);
 }
 
 // One warp per row.  Lane l adds the squares of its 8-element vectors l, l + 32, ... in
@@ -256,26 +373,61 @@ bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int64_t rows,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Workspace the split schedule needs: one fp32 [M, N] slab per segment.
+size_t split_workspace_bytes(int64_t M, int64_t N, int64_t K, int bn) {
+  return sizeof(float) * static_cast<size_t>(segments_of(N, K, bn).n_seg) * M * N;
+}
+
 template <int BN>
 vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
-                           int sm_count, cudaStream_t stream) {
+                           void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream) {
   using Cfg = LinearCfg<BN>;
   static bool attr_set[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return VOSTI_ERR_CUDA;
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(linear_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) !=
-        cudaSuccess)
+    if (cudaFuncSetAttribute(linear_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(linear_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::kSmemBytes) != cudaSuccess)
       return VOSTI_ERR_CUDA;
     attr_set[dev] = true;
   }
   alignas(64) CUtensorMap x_map, w_map;
   if (!make_map(fn, &x_map, x, M, K, Cfg::kBM) || !make_map(fn, &w_map, w, N, K, BN)) return VOSTI_ERR_CUDA;
   const int64_t tiles = ((M + Cfg::kBM - 1) / Cfg::kBM) * (N / BN);
-  const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
-  linear_kernel<BN><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(x_map, w_map, static_cast<__nv_bfloat16*>(y),
-                                                                      static_cast<int>(M), static_cast<int>(N),
-                                                                      static_cast<int>(K));
+  const Segments seg = segments_of(N, K, BN);
+  // Scheduling only: split the segments over CTAs when whole tiles would leave most SMs idle
+  // and the caller has provided room for the segment sums.
+  const bool split = seg.n_seg > 1 && tiles * 2 <= sm_count && workspace != nullptr &&
+                     workspace_bytes >= split_workspace_bytes(M, N, K, BN) &&
+                     reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
+  __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(y);
+  if (!split) {
+    const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
+    linear_kernel<BN, false><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
+        x_map, w_map, yb, nullptr, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+  } else {
+    const int64_t units = tiles * seg.n_seg;
+    const int grid = static_cast<int>(units < sm_count ? units : sm_count);
+    float* ws = static_cast<float*>(workspace);
+    linear_kernel<BN, true><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(
+        x_map, w_map, yb, ws, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+    // the fold may be scheduled while the segment kernel drains; it waits for it on the device
+    const int64_t threads = M * N / 8;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>((threads + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, linear_fold_kernel, static_cast<const float*>(ws), yb, static_cast<int>(M),
+                           static_cast<int>(N), BN, seg.n_seg) != cudaSuccess)
+      return VOSTI_ERR_CUDA;
+  }
   return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
 }
 
@@ -295,7 +447,22 @@ vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t
   return VOSTI_OK;
 }
 
-vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* cuda_stream) {
+vosti_status vosti_linear_segments(int64_t N, int64_t K, int32_t* n_segments) {
+  int32_t bn = 0;
+  const vosti_status shape = vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr);
+  if (shape != VOSTI_OK) return shape;
+  if (n_segments) *n_segments = segments_of(N, K, bn).n_seg;
+  return VOSTI_OK;
+}
+
+size_t vosti_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  int32_t bn = 0;
+  if (M <= 0 || vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr) != VOSTI_OK) return 0;
+  return split_workspace_bytes(M, N, K, bn);
+}
+
+vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* workspace,
+                          size_t workspace_bytes, void* cuda_stream) {
   int32_t bn = 0;
   const vosti_status shape = vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr);
   if (shape != VOSTI_OK) return shape;
@@ -318,8 +485,8 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
       cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  return bn == 256 ? launch_linear<256>(fn, x, w, y, M, N, K, sm_count, stream)
-                   : launch_linear<128>(fn, x, w, y, M, N, K, sm_count, stream);
+  return bn == 256 ? launch_linear<256>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream)
+                   : launch_linear<128>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream);
 }
 
 vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,

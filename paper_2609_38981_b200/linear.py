@@ -11,12 +11,17 @@ from . import binding as _vb
 _lib = _vb._lib
 _vp = ctypes.c_void_p
 
-EXPORTS = ("vosti_linear_tile_shape", "vosti_linear", "vosti_rmsnorm", "vosti_linear_poll_status")
+EXPORTS = ("vosti_linear_tile_shape", "vosti_linear_segments", "vosti_linear_workspace_bytes", "vosti_linear",
+           "vosti_rmsnorm", "vosti_linear_poll_status")
 
 _lib.vosti_linear_tile_shape.restype = ctypes.c_int
 _lib.vosti_linear_tile_shape.argtypes = [ctypes.c_int64, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 3
 _lib.vosti_linear.restype = ctypes.c_int
-_lib.vosti_linear.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp]
+_lib.vosti_linear.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp, ctypes.c_size_t, _vp]
+_lib.vosti_linear_segments.restype = ctypes.c_int
+_lib.vosti_linear_segments.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.POINTER(ctypes.c_int32)]
+_lib.vosti_linear_workspace_bytes.restype = ctypes.c_size_t
+_lib.vosti_linear_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64]
 _lib.vosti_rmsnorm.restype = ctypes.c_int
 _lib.vosti_rmsnorm.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_float, _vp]
 _lib.vosti_linear_poll_status.restype = ctypes.c_int
@@ -31,13 +36,25 @@ def vosti_linear_tile_shape(N: int, K: int):
     return tuple(x.value for x in v)
 
 
+def vosti_linear_segments(N: int, K: int) -> int:
+    v = ctypes.c_int32()
+    _vb._check(_lib.vosti_linear_segments(int(N), int(K), ctypes.byref(v)), "vosti_linear_segments")
+    return v.value
+
+
+def vosti_linear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(_lib.vosti_linear_workspace_bytes(int(M), int(N), int(K)))
+
+
 def _bf16_cuda(t: torch.Tensor, ndim: int) -> torch.Tensor:
     assert t.is_cuda and t.dtype == torch.bfloat16 and t.is_contiguous() and t.ndim == ndim
     return t
 
 
-def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
-    """y [M, N] = x [M, K] @ w [N, K]^T; tensors are CUDA bf16, contiguous."""
+def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, workspace: torch.Tensor = None,
+                 stream=None) -> torch.Tensor:
+    """y [M, N] = x [M, K] @ w [N, K]^T; tensors are CUDA bf16, contiguous.  workspace: an optional
+    CUDA byte tensor (see vosti_linear_workspace_bytes) that allows the split schedule for small M."""
     x, w = _bf16_cuda(x, 2), _bf16_cuda(w, 2)
     M, K = x.shape
     N = w.shape[0]
@@ -46,8 +63,9 @@ def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, strea
         y = torch.empty((M, N), dtype=torch.bfloat16, device=x.device)
     _bf16_cuda(y, 2)
     assert y.shape == (M, N)
-    _vb._check(_lib.vosti_linear(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, _vb._stream(stream)),
-               "vosti_linear")
+    ws_ptr, ws_bytes = (0, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
+    _vb._check(_lib.vosti_linear(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, ws_ptr, ws_bytes,
+                                 _vb._stream(stream)), "vosti_linear")
     return y
 
 

@@ -48,6 +48,8 @@ def test_linear_header_symbols_and_tile_shape(vb):
     assert vl.vosti_linear_tile_shape(4096, 4096) == (128, 256, 64)
     assert vl.vosti_linear_tile_shape(28672, 4096) == (128, 256, 64)
     assert vl.vosti_linear_tile_shape(128, 64) == (128, 128, 64)
+    assert vl.vosti_linear_segments(4096, 4096) == 4 and vl.vosti_linear_segments(6144, 4096) == 4
+    assert vl.vosti_linear_workspace_bytes(3, 128, 64) == 3 * 128 * 4 and vl.vosti_linear_workspace_bytes(3, 100, 64) == 0
     for N, K in ((0, 64), (100, 64), (128, 32), (128, 0)):
         with pytest.raises(vb.VostiError) as e:
             vl.vosti_linear_tile_shape(N, K)

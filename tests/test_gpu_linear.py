@@ -26,6 +26,12 @@ def widen(t):
     return t.float().double().cpu().numpy()
 
 
+def workspace(M, N, K):
+    """Room for the split schedule (the library decides whether to use it)."""
+    from paper_2609_38981_b200 import linear as vl
+    return torch.empty(max(vl.vosti_linear_workspace_bytes(M, N, K), 16), dtype=torch.uint8, device="cuda")
+
+
 @pytest.mark.parametrize("N,K", SHAPES)
 def test_linear_parity_with_the_oracle(N, K):
     """fp32 accumulation of exact bf16 products over K terms, one rounding to bf16: the error is
@@ -35,7 +41,7 @@ def test_linear_parity_with_the_oracle(N, K):
     from paper_2609_38981_b200 import linear as vl
     for M in (1, 130, 517):
         x, w = data(N, K, M, 11)
-        y = vl.vosti_linear(x.cuda(), w.cuda())
+        y = vl.vosti_linear(x.cuda(), w.cuda(), workspace=workspace(M, N, K) if M != 130 else None)
         ref = lo.linear(inputs.bits(x), inputs.bits(w))
         mag = np.abs(widen(x)) @ np.abs(widen(w)).T
         err = np.abs(widen(y) - ref)
@@ -46,18 +52,24 @@ def test_linear_parity_with_the_oracle(N, K):
 
 @pytest.mark.parametrize("N,K", SHAPES)
 def test_row_level_contract(N, K):
-    """Every row of every batch equals its singleton run bit for bit, wherever it sits."""
+    """Every row of every batch equals its singleton run bit for bit, wherever it sits, and
+    whichever schedule computes it: whole tiles per CTA (no workspace) or the K segments of a
+    tile spread over CTAs (workspace given, few row tiles)."""
     from paper_2609_38981_b200 import linear as vl
     from paper_2609_38981_b200.harness import bf16_bits
     x, w = data(N, K, 1000, 12)
     xd, wd = x.cuda(), w.cuda()
-    single = torch.cat([bf16_bits(vl.vosti_linear(xd[i:i + 1].contiguous(), wd)) for i in range(0, 1000, 37)])
     rows = list(range(0, 1000, 37))
+    single = torch.cat([bf16_bits(vl.vosti_linear(xd[i:i + 1].contiguous(), wd)) for i in rows])
+    single_split = torch.cat([bf16_bits(vl.vosti_linear(xd[i:i + 1].contiguous(), wd, workspace=workspace(1, N, K)))
+                              for i in rows])
+    assert torch.equal(single, single_split), "the two schedules disagree on a singleton run"
     for M in BATCHES:
-        y = bf16_bits(vl.vosti_linear(xd[:M].contiguous(), wd))
-        for j, i in enumerate(rows):
-            if i < M:
-                assert torch.equal(y[i], single[j]), (N, K, M, i)
+        for ws in (None, workspace(M, N, K)):
+            y = bf16_bits(vl.vosti_linear(xd[:M].contiguous(), wd, workspace=ws))
+            for j, i in enumerate(rows):
+                if i < M:
+                    assert torch.equal(y[i], single[j]), (N, K, M, i, ws is not None)
     # the same rows in another order and with strangers in between
     perm = torch.randperm(1000, generator=inputs.generator(5))
     y = bf16_bits(vl.vosti_linear(xd[perm.cuda()].contiguous(), wd))
@@ -67,10 +79,16 @@ def test_row_level_contract(N, K):
         assert torch.equal(y[inv[i]], single[j]), (N, K, "permuted", i)
 
 
-def test_tile_shape_is_a_function_of_the_weight_only():
+def test_tile_shape_and_segments_are_functions_of_the_weight_only():
     from paper_2609_38981_b200 import linear as vl
     assert vl.vosti_linear_tile_shape(4096, 4096) == (128, 256, 64)
     assert vl.vosti_linear_tile_shape(384, 64) == (128, 128, 64)
+    # ceil(148 / column tiles), at most K / 1024
+    assert vl.vosti_linear_segments(4096, 4096) == 4        # 16 column tiles -> 10, capped by 4096 / 1024
+    assert vl.vosti_linear_segments(4096, 14336) == 10
+    assert vl.vosti_linear_segments(28672, 4096) == 2
+    assert vl.vosti_linear_segments(256, 64) == 1
+    assert vl.vosti_linear_workspace_bytes(64, 4096, 4096) == 4 * 64 * 4096 * 4
 
 
 def test_rmsnorm_parity_and_row_independence():
