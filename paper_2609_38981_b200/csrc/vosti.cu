@@ -669,6 +669,97 @@ vosti_status vosti_cp_combine(vosti_ctx* ctx, void* out, float* lse, const int32
 
 namespace {
 
+// Shared-split packing (scheduling only).  Candidates: complete splits (all 512 keys below every
+// row of the request) of split-parallel requests.  Requests whose 32 page ids of a split agree
+// form a group; the rows of a group of two or more are laid out 16 to a packed item, if that
+// saves tiles.  Writes the packed rows at `packed_rows`, one SplitItem per packed item at the
+// front of `split_items`, marks the (request, split) pairs it has taken over in ctx->pk_mark,
+// and returns the number of packed items.
+int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, int G, const int32_t* bt_flat,
+                           PackedRow* packed_rows, SplitItem* split_items) {
+  std::vector<int64_t>& pk_off = ctx->pk_off;
+  std::vector<uint8_t>& pk_mark = ctx->pk_mark;
+  int64_t n_split_final = 0, n_packed_items = 0;
+  std::vector<PackCand>& cands = ctx->cands;
+  cands.clear();
+  pk_off.assign(static_cast<size_t>(batch) + 1, 0);
+  for (int r = 0; r < batch; ++r) {
+    const ReqMeta& m = reqs[r];
+    const int64_t complete =
+        (m.q_len > 0 && int64_t{m.q_len} * G <= nc::kSplitRowsMax) ? m.start / nc::kSplitLen : 0;
+    pk_off[r + 1] = pk_off[r] + complete;
+    for (int64_t k = 0; k < complete; ++k) {
+      const int32_t* ids = bt_flat + m.bt_off + k * nc::kPagesPerSplit;
+      // Grouping key: the split index with its first and last page id.  Two requests that share
+      // the whole split agree on it; agreement on all 32 ids is checked when groups are formed.
+      const uint64_t key = ((static_cast<uint64_t>(static_cast<uint32_t>(ids[0])) << 32) |
+                            static_cast<uint32_t>(ids[nc::kPagesPerSplit - 1])) * 0x9E3779B97F4A7C15ull +
+                           static_cast<uint64_t>(k);
+      cands.push_back({key, r, static_cast<int32_t>(k)});
+    }
+  }
+  pk_mark.assign(static_cast<size_t>(pk_off[batch]), 0);
+  std::sort(cands.begin(), cands.end(), [](const PackCand& a, const PackCand& b) {
+    return a.key != b.key ? a.key < b.key : a.req < b.req;
+  });
+  auto same_pages = [&](const PackCand& a, const PackCand& b) {
+    return a.split == b.split &&
+           std::memcmp(bt_flat + reqs[a.req].bt_off + int64_t{a.split} * nc::kPagesPerSplit,
+                       bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
+                       sizeof(int32_t) * nc::kPagesPerSplit) == 0;
+  };
+  for (size_t lo = 0; lo < cands.size();) {
+    size_t hi = lo + 1;
+    while (hi < cands.size() && cands[hi].key == cands[lo].key) ++hi;
+    // members: the very same split and page ids as the first (a hash collision stays unpacked)
+    // and packing must save tiles: fewer 16-row tiles together than one request at a time
+    int members = 0;
+    int64_t rows_together = 0, tiles_apart = 0;
+    for (size_t i = lo; i < hi; ++i)
+      if (same_pages(cands[i], cands[lo])) {
+        const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
+        ++members;
+        rows_together += rows;
+        tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+      }
+    if (members >= 2 && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup < tiles_apart) {
+      const ReqMeta& first = reqs[cands[lo].req];
+      int in_item = 0;
+      auto close_item = [&]() {
+        PackedRow* rows16 = packed_rows + n_packed_items * 16;
+        for (int i = in_item; i < 16; ++i) rows16[i] = PackedRow{0, -1, 0, 0};
+        SplitItem& si = split_items[n_split_final++];
+        si = SplitItem{};
+        si.q_len = in_item;  // rows in use
+        si.n_pages = first.n_pages;
+        si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
+        si.split = cands[lo].split;
+        si.req = static_cast<int32_t>(-1 - n_packed_items);
+        ++n_packed_items;
+        in_item = 0;
+      };
+      for (size_t i = lo; i < hi; ++i) {
+        if (!same_pages(cands[i], cands[lo])) continue;
+        const ReqMeta& m = reqs[cands[i].req];
+        const int k = cands[i].split;
+        pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
+        const int rows = m.q_len * G;
+        for (int row = 0; row < rows; ++row) {
+          PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
+          pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
+          pr.p = m.start + row / G;
+          pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
+          pr.kvh_stride = m.n_splits * rows;
+          if (++in_item == 16) close_item();
+        }
+      }
+      if (in_item > 0) close_item();
+    }
+    lo = hi;
+  }
+  return n_packed_items;
+}
+
 vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse, const int32_t* q_lens,
                             const int32_t* start_pos, const int32_t* seq_lens, const int32_t* block_tables,
                             int32_t block_table_stride, int32_t batch, float softmax_scale, int32_t window,
@@ -762,11 +853,8 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
   }
   at += align_up(sizeof(int32_t) * bt_used, 16);
 
-  // ---- shared-split packing (scheduling only) ---------------------------------------------
-  // Candidates: complete splits (all 512 keys below every row of the request) of split-parallel
-  // requests.  Requests whose 32 page ids of a split agree form a group; the rows of a group of
-  // two or more are laid out 16 to a packed item.  Packed items come first in the item list
-  // (they walk a whole split: the longest kind), the others follow in plan order.
+  // ---- shared-split packing (scheduling only): packed items first in the item list (they walk a
+  // whole split: the longest kind), the others follow in plan order ---------------------------
   int64_t n_split_final = 0, n_packed_items = 0;
   size_t off_packed = 0;
   std::vector<int64_t>& pk_off = ctx->pk_off;
@@ -774,85 +862,10 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
   const bool packing = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) && window == 0 && cp.phase == 0 && plan.n_split > 1 &&
                        plan.n_partial_rows < (int64_t{1} << 31) && row0 < (int64_t{1} << 24) && G <= 128;
   if (packing) {
-    std::vector<PackCand>& cands = ctx->cands;
-    cands.clear();
-    pk_off.assign(static_cast<size_t>(batch) + 1, 0);
-    for (int r = 0; r < batch; ++r) {
-      const ReqMeta& m = reqs[r];
-      const int64_t complete =
-          (m.q_len > 0 && int64_t{m.q_len} * G <= nc::kSplitRowsMax) ? m.start / nc::kSplitLen : 0;
-      pk_off[r + 1] = pk_off[r] + complete;
-      for (int64_t k = 0; k < complete; ++k) {
-        const int32_t* ids = bt_flat + m.bt_off + k * nc::kPagesPerSplit;
-        // Grouping key: the split index with its first and last page id.  Two requests that share
-        // the whole split agree on it; agreement on all 32 ids is checked when groups are formed.
-        const uint64_t key = ((static_cast<uint64_t>(static_cast<uint32_t>(ids[0])) << 32) |
-                              static_cast<uint32_t>(ids[nc::kPagesPerSplit - 1])) * 0x9E3779B97F4A7C15ull +
-                             static_cast<uint64_t>(k);
-        cands.push_back({key, r, static_cast<int32_t>(k)});
-      }
-    }
-    pk_mark.assign(static_cast<size_t>(pk_off[batch]), 0);
-    std::sort(cands.begin(), cands.end(), [](const PackCand& a, const PackCand& b) {
-      return a.key != b.key ? a.key < b.key : a.req < b.req;
-    });
     off_packed = at;
-    PackedRow* packed_rows = reinterpret_cast<PackedRow*>(blob + at);
-    auto same_pages = [&](const PackCand& a, const PackCand& b) {
-      return a.split == b.split &&
-             std::memcmp(bt_flat + reqs[a.req].bt_off + int64_t{a.split} * nc::kPagesPerSplit,
-                         bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
-                         sizeof(int32_t) * nc::kPagesPerSplit) == 0;
-    };
-    for (size_t lo = 0; lo < cands.size();) {
-      size_t hi = lo + 1;
-      while (hi < cands.size() && cands[hi].key == cands[lo].key) ++hi;
-      // members: the very same split and page ids as the first (a hash collision stays unpacked)
-      // and packing must save tiles: fewer 16-row tiles together than one request at a time
-      int members = 0;
-      int64_t rows_together = 0, tiles_apart = 0;
-      for (size_t i = lo; i < hi; ++i)
-        if (same_pages(cands[i], cands[lo])) {
-          const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
-          ++members;
-          rows_together += rows;
-          tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
-        }
-      if (members >= 2 && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup < tiles_apart) {
-        const ReqMeta& first = reqs[cands[lo].req];
-        int in_item = 0;
-        auto close_item = [&]() {
-          PackedRow* rows16 = packed_rows + n_packed_items * 16;
-          for (int i = in_item; i < 16; ++i) rows16[i] = PackedRow{0, -1, 0, 0};
-          SplitItem& si = split_items[n_split_final++];
-          si = SplitItem{};
-          si.q_len = in_item;  // rows in use
-          si.n_pages = first.n_pages;
-          si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
-          si.split = cands[lo].split;
-          si.req = static_cast<int32_t>(-1 - n_packed_items);
-          ++n_packed_items;
-          in_item = 0;
-        };
-        for (size_t i = lo; i < hi; ++i) {
-          if (!same_pages(cands[i], cands[lo])) continue;
-          const ReqMeta& m = reqs[cands[i].req];
-          const int k = cands[i].split;
-          pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
-          const int rows = m.q_len * G;
-          for (int row = 0; row < rows; ++row) {
-            PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
-            pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
-            pr.p = m.start + row / G;
-            pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
-            pr.kvh_stride = m.n_splits * rows;
-            if (++in_item == 16) close_item();
-          }
-        }
-        if (in_item > 0) close_item();
-      }
-      lo = hi;
-    }
+    n_packed_items = pack_shared_splits(ctx, reqs, batch, G, bt_flat, reinterpret_cast<PackedRow*>(blob + at),
+                                        split_items);
+    n_split_final = n_packed_items;
     at += align_up(sizeof(PackedRow) * 16 * n_packed_items, 16);
   }
   for (int64_t i = 0; i < plan.n_split; ++i) {
