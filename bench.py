@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--pack-shared-splits", action="store_true",
                     help="create the context with VOSTI_FLAG_PACK_SHARED_SPLITS (same bits, fewer tiles "
                          "when requests share prefix pages)")
+    ap.add_argument("--window", type=int, default=0,
+                    help="sliding window (keys); experiments with vosti_paged_attention_ex, the e2e and "
+                         "cpu_baseline legs stay unwindowed")
     ap.add_argument("--pool-pages", type=int, default=0,
                     help="override the pool size (small pools keep profiler captures short)")
     return ap.parse_args()
@@ -303,7 +306,11 @@ def main():
 
     def step():
         vb.vosti_kv_append(cache.ctx, kn, vn, ql, st, bt, stream=stream)
-        vb.vosti_paged_attention(cache.ctx, q, out, ql, st, sl, bt, scale, stream=stream)
+        if args.window:
+            vb.vosti_paged_attention_ex(cache.ctx, q, out, None, ql, st, sl, bt, scale, window=args.window,
+                                        stream=stream)
+        else:
+            vb.vosti_paged_attention(cache.ctx, q, out, ql, st, sl, bt, scale, stream=stream)
 
     def sync_all():
         torch.cuda.synchronize()
@@ -373,6 +380,9 @@ def main():
     out_match = bool(torch.equal(outh.view(torch.int16), out.cpu().view(torch.int16)))
 
     kv_bytes = float(w.kv_bytes())
+    if args.window:  # keys some row of the request sees: from the first row's window start to the last position
+        kv_bytes = float(sum(min(s + n, args.window + n - 1) for s, n in zip(w.start_pos, w.q_lens) if n > 0)
+                         * geo.kv_bytes_per_token)
     t_max, e2e_max, bytes_all, tok_all = elapsed_ms, e2e_ms, kv_bytes, float(w.total_q)
     if dist is not None:
         t = torch.tensor([elapsed_ms, e2e_ms], device=dev, dtype=torch.float64)
@@ -428,6 +438,7 @@ def main():
                           "K steps with a CUDA event pair around each launch of the dominant kernel",
                 "ms_per_step_with_kernel_events": roof_ms / args.steps,
                 "pack_shared_splits": bool(args.pack_shared_splits),
+                "window": int(args.window),
                 "schedule": dict(zip(("split_items", "packed_items", "tile_items"),
                                      vb.vosti_last_schedule(cache.ctx))),
             },
