@@ -251,6 +251,7 @@ struct vosti_ctx {
   std::vector<PackCand> cands;     // shared-split packing scratch
   std::vector<int64_t> pk_off;     // per request: first entry of its complete splits in pk_mark
   std::vector<uint8_t> pk_mark;    // 1: the (request, split) pair is served by packed items
+  std::vector<int32_t> pk_table, pk_next, pk_head, pk_tail;  // grouping of the candidates by key
   int64_t last_split_items = 0, last_packed_items = 0, last_tile_items = 0;  // schedule of the last attention call
   // profiling of the dominant kernel
   int profile_mode = 0;
@@ -699,63 +700,83 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
     }
   }
   pk_mark.assign(static_cast<size_t>(pk_off[batch]), 0);
-  std::sort(cands.begin(), cands.end(), [](const PackCand& a, const PackCand& b) {
-    return a.key != b.key ? a.key < b.key : a.req < b.req;
-  });
+  // Group the candidates by key without sorting: an open-addressing table from key to group, the
+  // members of a group chained in the order they were generated (ascending request index).
+  const int n = static_cast<int>(cands.size());
+  int table_size = 64;
+  while (table_size < 2 * n) table_size *= 2;
+  std::vector<int32_t>& table = ctx->pk_table;
+  std::vector<int32_t>& next = ctx->pk_next;
+  std::vector<int32_t>& head = ctx->pk_head;
+  std::vector<int32_t>& tail = ctx->pk_tail;
+  table.assign(static_cast<size_t>(table_size), -1);
+  next.assign(static_cast<size_t>(n), -1);
+  head.clear();
+  tail.clear();
+  for (int i = 0; i < n; ++i) {
+    uint32_t h = static_cast<uint32_t>((cands[i].key * 0xD6E8FEB86659FD93ull) >> 40) & (table_size - 1);
+    while (table[h] >= 0 && cands[head[table[h]]].key != cands[i].key) h = (h + 1) & (table_size - 1);
+    if (table[h] < 0) {
+      table[h] = static_cast<int32_t>(head.size());
+      head.push_back(i);
+      tail.push_back(i);
+    } else {
+      next[tail[table[h]]] = i;
+      tail[table[h]] = i;
+    }
+  }
   auto same_pages = [&](const PackCand& a, const PackCand& b) {
     return a.split == b.split &&
            std::memcmp(bt_flat + reqs[a.req].bt_off + int64_t{a.split} * nc::kPagesPerSplit,
                        bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
                        sizeof(int32_t) * nc::kPagesPerSplit) == 0;
   };
-  for (size_t lo = 0; lo < cands.size();) {
-    size_t hi = lo + 1;
-    while (hi < cands.size() && cands[hi].key == cands[lo].key) ++hi;
-    // members: the very same split and page ids as the first (a hash collision stays unpacked)
+  for (size_t g = 0; g < head.size(); ++g) {
+    const int lo = head[g];
+    if (next[lo] < 0) continue;  // alone
+    // members: the very same split and page ids as the first (a key collision stays unpacked)
     // and packing must save tiles: fewer 16-row tiles together than one request at a time
     int members = 0;
     int64_t rows_together = 0, tiles_apart = 0;
-    for (size_t i = lo; i < hi; ++i)
+    for (int i = lo; i >= 0; i = next[i])
       if (same_pages(cands[i], cands[lo])) {
         const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
         ++members;
         rows_together += rows;
         tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
       }
-    if (members >= 2 && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup < tiles_apart) {
-      const ReqMeta& first = reqs[cands[lo].req];
-      int in_item = 0;
-      auto close_item = [&]() {
-        PackedRow* rows16 = packed_rows + n_packed_items * 16;
-        for (int i = in_item; i < 16; ++i) rows16[i] = PackedRow{0, -1, 0, 0};
-        SplitItem& si = split_items[n_split_final++];
-        si = SplitItem{};
-        si.q_len = in_item;  // rows in use
-        si.n_pages = first.n_pages;
-        si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
-        si.split = cands[lo].split;
-        si.req = static_cast<int32_t>(-1 - n_packed_items);
-        ++n_packed_items;
-        in_item = 0;
-      };
-      for (size_t i = lo; i < hi; ++i) {
-        if (!same_pages(cands[i], cands[lo])) continue;
-        const ReqMeta& m = reqs[cands[i].req];
-        const int k = cands[i].split;
-        pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
-        const int rows = m.q_len * G;
-        for (int row = 0; row < rows; ++row) {
-          PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
-          pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
-          pr.p = m.start + row / G;
-          pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
-          pr.kvh_stride = m.n_splits * rows;
-          if (++in_item == 16) close_item();
-        }
+    if (members < 2 || (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup >= tiles_apart) continue;
+    const ReqMeta& first = reqs[cands[lo].req];
+    int in_item = 0;
+    auto close_item = [&]() {
+      PackedRow* rows16 = packed_rows + n_packed_items * 16;
+      for (int i = in_item; i < 16; ++i) rows16[i] = PackedRow{0, -1, 0, 0};
+      SplitItem& si = split_items[n_split_final++];
+      si = SplitItem{};
+      si.q_len = in_item;  // rows in use
+      si.n_pages = first.n_pages;
+      si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
+      si.split = cands[lo].split;
+      si.req = static_cast<int32_t>(-1 - n_packed_items);
+      ++n_packed_items;
+      in_item = 0;
+    };
+    for (int i = lo; i >= 0; i = next[i]) {
+      if (!same_pages(cands[i], cands[lo])) continue;
+      const ReqMeta& m = reqs[cands[i].req];
+      const int k = cands[i].split;
+      pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
+      const int rows = m.q_len * G;
+      for (int row = 0; row < rows; ++row) {
+        PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
+        pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
+        pr.p = m.start + row / G;
+        pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
+        pr.kvh_stride = m.n_splits * rows;
+        if (++in_item == 16) close_item();
       }
-      if (in_item > 0) close_item();
     }
-    lo = hi;
+    if (in_item > 0) close_item();
   }
   return n_packed_items;
 }
