@@ -243,6 +243,29 @@ vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host,
                              const int32_t* block_tables, int32_t block_table_stride, int32_t batch,
                              float softmax_scale, void* cuda_stream);
 
+/* The same step without the wait, for callers that keep several steps in
+ * flight: inputs go up on a stream of the context while the previous step's
+ * kernels run on `cuda_stream`, and the output comes down on another while the
+ * next step's kernels run.  Steps execute in the order issued (KV appended by
+ * one is visible to the next); the kernels, the plan and therefore the bits
+ * are those of vosti_step_host.  The int32 arrays are read before the call
+ * returns; q_host, k_new_host, v_new_host must stay unchanged, and out_host is
+ * not valid, until vosti_step_host_wait(ctx, *ticket) has returned.  Up to
+ * VOSTI_HOST_STEPS_IN_FLIGHT steps may be pending; issuing one more first
+ * waits for the oldest.  Host buffers should be pinned (pageable memory makes
+ * the copies synchronous).  All steps of a context must use one cuda_stream. */
+#define VOSTI_HOST_STEPS_IN_FLIGHT 3
+vosti_status vosti_step_host_async(vosti_ctx* ctx, const void* q_host, void* out_host,
+                                   const void* k_new_host, const void* v_new_host,
+                                   const int32_t* q_lens, const int32_t* start_pos,
+                                   const int32_t* seq_lens, const int32_t* block_tables,
+                                   int32_t block_table_stride, int32_t batch, float softmax_scale,
+                                   void* cuda_stream, int64_t* ticket);
+/* Blocks until the step's out_host is complete.  A ticket already waited for
+ * (explicitly, or because a later step reused its staging) returns at once;
+ * INVALID_ARG for a ticket never issued. */
+vosti_status vosti_step_host_wait(vosti_ctx* ctx, int64_t ticket);
+
 /* Split-parallel paged attention for callers that must not allocate.  (The
  * paper has no counterpart: this is a packaging variant of the operation
  * above, not a different computation.)

@@ -26,11 +26,13 @@ VOSTI_OK, VOSTI_ERR_INVALID_ARG, VOSTI_ERR_UNSUPPORTED_CONFIG, VOSTI_ERR_OUT_OF_
     VOSTI_ERR_WORKSPACE, VOSTI_ERR_CUDA, VOSTI_ERR_TIMEOUT = range(7)
 VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
 VOSTI_FLAG_PACK_SHARED_SPLITS = 2
+VOSTI_HOST_STEPS_IN_FLIGHT = 3
 
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
     "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_cp_partial",
-    "vosti_cp_combine", "vosti_step_host", "vosti_poll_device_status",
+    "vosti_cp_combine", "vosti_step_host", "vosti_step_host_async", "vosti_step_host_wait",
+    "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
     "vosti_last_schedule", "vosti_fingerprint",
     "vosti_constants", "vosti_status_string",
@@ -95,6 +97,10 @@ _lib.vosti_paged_attention_noalloc.argtypes = [
 _lib.vosti_step_host.restype = ctypes.c_int
 _lib.vosti_step_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p,
                                  ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_step_host_async.restype = ctypes.c_int
+_lib.vosti_step_host_async.argtypes = _lib.vosti_step_host.argtypes + [ctypes.POINTER(ctypes.c_int64)]
+_lib.vosti_step_host_wait.restype = ctypes.c_int
+_lib.vosti_step_host_wait.argtypes = [_vp, ctypes.c_int64]
 _lib.vosti_poll_device_status.restype = ctypes.c_int
 _lib.vosti_poll_device_status.argtypes = [_vp, _vp]
 _lib.vosti_selftest_bounded_wait.restype = ctypes.c_int
@@ -335,6 +341,23 @@ def vosti_step_host(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_le
     _check(_lib.vosti_step_host(ctx.handle, _dev(q_host), _dev(out_host), _dev(k_new_host),
                                 _dev(v_new_host), _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1],
                                 len(ql), float(softmax_scale), _stream(stream)), "vosti_step_host")
+
+
+def vosti_step_host_async(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_lens, start_pos,
+                          seq_lens, block_tables, softmax_scale: float, stream=None) -> int:
+    """Returns the step's ticket; the host buffers belong to the library until it is waited for."""
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    bt = _host_i32(block_tables)
+    ticket = ctypes.c_int64(-1)
+    _check(_lib.vosti_step_host_async(ctx.handle, _dev(q_host), _dev(out_host), _dev(k_new_host),
+                                      _dev(v_new_host), _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1],
+                                      len(ql), float(softmax_scale), _stream(stream), ctypes.byref(ticket)),
+           "vosti_step_host_async")
+    return ticket.value
+
+
+def vosti_step_host_wait(ctx: Context, ticket: int) -> None:
+    _check(_lib.vosti_step_host_wait(ctx.handle, int(ticket)), "vosti_step_host_wait")
 
 
 def vosti_poll_device_status(ctx: Context, stream=None) -> int:

@@ -16,6 +16,7 @@ namespace vosti {
 namespace {
 
 constexpr int kHostSlots = 8;        // ring of pinned staging buffers
+constexpr int kHostSteps = 3;        // host-buffer steps that may be in flight (vosti_step_host_async)
 constexpr size_t kAlign = 1024;
 constexpr int kTileRows = 256;       // rows of one tile-kernel work item (16 row groups)
 
@@ -42,8 +43,7 @@ struct Limits {
   int64_t part_rows_max;
   size_t meta_bytes;     // one metadata blob (attention or append)
   // workspace offsets
-  size_t off_status, off_meta, off_part_u, off_part_mz, off_uc, off_stage_q, off_stage_o, off_stage_k,
-      off_stage_v, total;
+  size_t off_status, off_meta, off_part_u, off_part_mz, off_uc, off_stage, stage_q, stage_kv, total;
 };
 
 Limits limits_of(const vosti_config& c) {
@@ -77,10 +77,10 @@ Limits limits_of(const vosti_config& c) {
   at += align_up(sizeof(float) * items_seq * c.n_kv_heads * kTileRows * c.head_dim);
   const size_t qbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_q_heads * c.head_dim;
   const size_t kbytes = sizeof(__nv_bfloat16) * c.max_total_q * c.n_kv_heads * c.head_dim;
-  L.off_stage_q = at; at += align_up(qbytes);
-  L.off_stage_o = at; at += align_up(qbytes);
-  L.off_stage_k = at; at += align_up(kbytes);
-  L.off_stage_v = at; at += align_up(kbytes);
+  // staging of the host-buffer steps: one set of (q, out, k_new, v_new) per step in flight
+  L.stage_q = align_up(qbytes);
+  L.stage_kv = align_up(kbytes);
+  L.off_stage = at; at += kHostSteps * (2 * L.stage_q + 2 * L.stage_kv);
   L.total = at;
   return L;
 }
@@ -229,6 +229,15 @@ struct HostSlot {
   bool has_release = false;
 };
 
+// One host-buffer step in flight: its staging set in the workspace and the three
+// points of its life (inputs on the device, kernels done, output on the host).
+struct HostStep {
+  cudaEvent_t in_done = nullptr;
+  cudaEvent_t computed = nullptr;
+  cudaEvent_t out_done = nullptr;
+  int64_t ticket = -1;  // -1: nothing pending in this set
+};
+
 }  // namespace
 }  // namespace vosti
 
@@ -244,6 +253,10 @@ struct vosti_ctx {
   HostSlot slots[kHostSlots];
   int next_slot = 0;
   cudaStream_t copy_stream = nullptr;  // metadata uploads overlap the previous call's kernels
+  cudaStream_t in_stream = nullptr;    // host-buffer steps: inputs of the next step while this one computes
+  cudaStream_t out_stream = nullptr;   // host-buffer steps: output of the last step while this one computes
+  HostStep host_steps[kHostSteps];
+  int64_t host_steps_issued = 0;
   uint8_t* ws = nullptr;
   int64_t launches = 0;
   Plan plan;                       // reused across calls: no allocation in steady state
@@ -520,6 +533,16 @@ vosti_status vosti_create(vosti_ctx** out, const vosti_config* config) {
   if (st == VOSTI_OK) st = config->head_dim == 128 ? set_kernel_attributes<128>() : set_kernel_attributes<64>();
   if (st == VOSTI_OK && cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
     st = VOSTI_ERR_CUDA;
+  if (st == VOSTI_OK && (cudaStreamCreateWithFlags(&ctx->in_stream, cudaStreamNonBlocking) != cudaSuccess ||
+                         cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking) != cudaSuccess))
+    st = VOSTI_ERR_CUDA;
+  for (int i = 0; st == VOSTI_OK && i < kHostSteps; ++i) {
+    HostStep& h = ctx->host_steps[i];
+    if (cudaEventCreateWithFlags(&h.in_done, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.computed, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h.out_done, cudaEventDisableTiming) != cudaSuccess)
+      st = VOSTI_ERR_CUDA;
+  }
   for (int i = 0; st == VOSTI_OK && i < kHostSlots; ++i) {
     ctx->slots[i].device = ctx->ws + lim.off_meta + static_cast<size_t>(i) * lim.meta_bytes;
     if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->slots[i].pinned), lim.meta_bytes, cudaHostAllocDefault) !=
@@ -546,10 +569,14 @@ vosti_status vosti_destroy(vosti_ctx* ctx) {
     if (s.released) cudaEventDestroy(s.released);
     if (s.pinned) cudaFreeHost(s.pinned);
   }
-  if (ctx->copy_stream) {
-    cudaStreamSynchronize(ctx->copy_stream);
-    cudaStreamDestroy(ctx->copy_stream);
+  for (cudaStream_t cs : {ctx->in_stream, ctx->out_stream, ctx->copy_stream}) {
+    if (!cs) continue;
+    cudaStreamSynchronize(cs);
+    cudaStreamDestroy(cs);
   }
+  for (auto& h : ctx->host_steps)
+    for (cudaEvent_t e : {h.in_done, h.computed, h.out_done})
+      if (e) cudaEventDestroy(e);
   for (auto e : ctx->ev_start) cudaEventDestroy(e);
   for (auto e : ctx->ev_stop) cudaEventDestroy(e);
   delete ctx;
@@ -968,12 +995,20 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
 
 extern "C" {
 
-vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
-                             const void* v_new_host, const int32_t* q_lens, const int32_t* start_pos,
-                             const int32_t* seq_lens, const int32_t* block_tables,
-                             int32_t block_table_stride, int32_t batch, float softmax_scale,
-                             void* cuda_stream) {
-  if (!ctx || batch < 0) return VOSTI_ERR_INVALID_ARG;
+vosti_status vosti_step_host_wait(vosti_ctx* ctx, int64_t ticket) {
+  if (!ctx || ticket < 0 || ticket >= ctx->host_steps_issued) return VOSTI_ERR_INVALID_ARG;
+  HostStep& h = ctx->host_steps[ticket % kHostSteps];
+  if (h.ticket != ticket) return VOSTI_OK;  // a later step took the set, which waited for this one first
+  h.ticket = -1;
+  return cudaEventSynchronize(h.out_done) == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+vosti_status vosti_step_host_async(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
+                                   const void* v_new_host, const int32_t* q_lens, const int32_t* start_pos,
+                                   const int32_t* seq_lens, const int32_t* block_tables,
+                                   int32_t block_table_stride, int32_t batch, float softmax_scale,
+                                   void* cuda_stream, int64_t* ticket) {
+  if (!ctx || batch < 0 || !ticket) return VOSTI_ERR_INVALID_ARG;
   if (batch > 0 && !q_lens) return VOSTI_ERR_INVALID_ARG;
   const vosti_config& c = ctx->cfg;
   int64_t total = 0;
@@ -982,29 +1017,63 @@ vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host,
     total += q_lens[r];
   }
   if (total > c.max_total_q) return VOSTI_ERR_OUT_OF_RANGE;
-  if (total == 0) return VOSTI_OK;
-  if (!q_host || !out_host || !k_new_host || !v_new_host) return VOSTI_ERR_INVALID_ARG;
+  if (total > 0 && (!q_host || !out_host || !k_new_host || !v_new_host)) return VOSTI_ERR_INVALID_ARG;
+  // The set of the step issued kHostSteps ago is reused: that step must be wholly done.
+  HostStep& h = ctx->host_steps[ctx->host_steps_issued % kHostSteps];
+  if (h.ticket >= 0) {
+    const vosti_status w = vosti_step_host_wait(ctx, h.ticket);
+    if (w != VOSTI_OK) return w;
+  }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t qbytes = sizeof(__nv_bfloat16) * total * c.n_q_heads * c.head_dim;
   const size_t kbytes = sizeof(__nv_bfloat16) * total * c.n_kv_heads * c.head_dim;
-  uint8_t* dq = ctx->ws + ctx->lim.off_stage_q;
-  uint8_t* dout = ctx->ws + ctx->lim.off_stage_o;
-  uint8_t* dk = ctx->ws + ctx->lim.off_stage_k;
-  uint8_t* dv = ctx->ws + ctx->lim.off_stage_v;
-  if (cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(dk, k_new_host, kbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-      cudaMemcpyAsync(dv, v_new_host, kbytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-    return VOSTI_ERR_CUDA;
-  vosti_status st =
-      vosti_kv_append(ctx, dk, dv, q_lens, start_pos, block_tables, block_table_stride, batch, stream);
-  if (st != VOSTI_OK) return st;
-  st = vosti_paged_attention(ctx, dq, dout, q_lens, start_pos, seq_lens, block_tables, block_table_stride,
-                             batch, softmax_scale, stream);
-  if (st != VOSTI_OK) return st;
-  if (cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaStreamSynchronize(stream) != cudaSuccess)
-    return VOSTI_ERR_CUDA;
+  uint8_t* dq = ctx->ws + ctx->lim.off_stage +
+                (ctx->host_steps_issued % kHostSteps) * (2 * ctx->lim.stage_q + 2 * ctx->lim.stage_kv);
+  uint8_t* dout = dq + ctx->lim.stage_q;
+  uint8_t* dk = dout + ctx->lim.stage_q;
+  uint8_t* dv = dk + ctx->lim.stage_kv;
+  if (total > 0) {
+    // Inputs go up on their own stream, so that they overlap the kernels of the step before.
+    if (cudaMemcpyAsync(dq, q_host, qbytes, cudaMemcpyHostToDevice, ctx->in_stream) != cudaSuccess ||
+        cudaMemcpyAsync(dk, k_new_host, kbytes, cudaMemcpyHostToDevice, ctx->in_stream) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v_new_host, kbytes, cudaMemcpyHostToDevice, ctx->in_stream) != cudaSuccess ||
+        cudaEventRecord(h.in_done, ctx->in_stream) != cudaSuccess ||
+        cudaStreamWaitEvent(stream, h.in_done, 0) != cudaSuccess)
+      return VOSTI_ERR_CUDA;
+    vosti_status st =
+        vosti_kv_append(ctx, dk, dv, q_lens, start_pos, block_tables, block_table_stride, batch, stream);
+    if (st == VOSTI_OK)
+      st = vosti_paged_attention(ctx, dq, dout, q_lens, start_pos, seq_lens, block_tables, block_table_stride,
+                                 batch, softmax_scale, stream);
+    if (st != VOSTI_OK) {
+      // Nothing of this step is reported as pending; what was enqueued is drained so that the
+      // caller may free its buffers.
+      cudaStreamSynchronize(ctx->in_stream);
+      cudaStreamSynchronize(stream);
+      return st;
+    }
+    // The output goes down on a third stream, under the kernels of the next step.
+    if (cudaEventRecord(h.computed, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(ctx->out_stream, h.computed, 0) != cudaSuccess ||
+        cudaMemcpyAsync(out_host, dout, qbytes, cudaMemcpyDeviceToHost, ctx->out_stream) != cudaSuccess)
+      return VOSTI_ERR_CUDA;
+  }
+  if (cudaEventRecord(h.out_done, ctx->out_stream) != cudaSuccess) return VOSTI_ERR_CUDA;
+  h.ticket = ctx->host_steps_issued;
+  *ticket = ctx->host_steps_issued++;
   return VOSTI_OK;
+}
+
+vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host, const void* k_new_host,
+                             const void* v_new_host, const int32_t* q_lens, const int32_t* start_pos,
+                             const int32_t* seq_lens, const int32_t* block_tables,
+                             int32_t block_table_stride, int32_t batch, float softmax_scale,
+                             void* cuda_stream) {
+  int64_t ticket = -1;
+  const vosti_status st =
+      vosti_step_host_async(ctx, q_host, out_host, k_new_host, v_new_host, q_lens, start_pos, seq_lens,
+                            block_tables, block_table_stride, batch, softmax_scale, cuda_stream, &ticket);
+  return st == VOSTI_OK ? vosti_step_host_wait(ctx, ticket) : st;
 }
 
 vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
