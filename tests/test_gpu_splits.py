@@ -15,6 +15,9 @@ GEOS = {
     "d128_g4": inputs.Geometry(8, 2, 128, 16),
     "d128_g8": inputs.Geometry(8, 1, 128, 16),
     "d64_g1": inputs.Geometry(2, 2, 64, 16),
+    "d128_g16": inputs.Geometry(16, 1, 128, 16),
+    "d64_g8": inputs.Geometry(8, 1, 64, 16),
+    "d128_g1": inputs.Geometry(2, 2, 128, 16),
 }
 # around split edges (512 k), tile edges (64 k), page edges (16 k), and the degenerate 1
 CONTEXTS = (1, 16, 511, 512, 513, 1023, 1024, 1025, 1600)
