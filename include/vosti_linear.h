@@ -39,7 +39,7 @@ extern "C" {
 vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t* b_n, int32_t* b_k);
 
 /* The number of K segments of an (N, K) weight, a pure host-side function of N
- * and K: ceil(148 / column tiles), at most K / 1024 and at least 1; segment j
+ * and K: floor(148 / column tiles), at most K / 1024 and at least 1; segment j
  * covers the 64-wide blocks [j B / n, (j + 1) B / n) of the B = K / 64 blocks. */
 vosti_status vosti_linear_segments(int64_t N, int64_t K, int32_t* n_segments);
 

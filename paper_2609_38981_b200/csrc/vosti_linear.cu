@@ -37,10 +37,10 @@ struct Segments {
 __host__ __device__ inline Segments segments_of(int64_t N, int64_t K, int bn) {
   const int k_blocks = static_cast<int>(K / 64);
   const int64_t col_tiles = N / bn;
-  // enough (column tile, segment) units for every SM of a B200 when the batch is a single row tile,
-  // but segments of at least 1024 elements: every segment costs the large-batch schedule a pass
-  // over the accumulator
-  int64_t want = (148 + col_tiles - 1) / col_tiles;
+  // as many (column tile, segment) units as fit one wave over the 148 SMs of a B200 when the batch
+  // is a single row tile, but segments of at least 1024 elements: every segment costs the
+  // large-batch schedule a pass over the accumulator
+  int64_t want = 148 / col_tiles;
   const int64_t cap = k_blocks / 16 > 0 ? k_blocks / 16 : 1;
   if (want > cap) want = cap;
   if (want < 1) want = 1;

@@ -83,10 +83,10 @@ def test_tile_shape_and_segments_are_functions_of_the_weight_only():
     from paper_2609_38981_b200 import linear as vl
     assert vl.vosti_linear_tile_shape(4096, 4096) == (128, 256, 64)
     assert vl.vosti_linear_tile_shape(384, 64) == (128, 128, 64)
-    # ceil(148 / column tiles), at most K / 1024
-    assert vl.vosti_linear_segments(4096, 4096) == 4        # 16 column tiles -> 10, capped by 4096 / 1024
-    assert vl.vosti_linear_segments(4096, 14336) == 10
-    assert vl.vosti_linear_segments(28672, 4096) == 2
+    # floor(148 / column tiles), at most K / 1024, at least 1
+    assert vl.vosti_linear_segments(4096, 4096) == 4        # 16 column tiles -> 9, capped by 4096 / 1024
+    assert vl.vosti_linear_segments(4096, 14336) == 9       # 144 (column tile, segment) units: one wave of 148 SMs
+    assert vl.vosti_linear_segments(28672, 4096) == 1       # 112 column tiles already fill the SMs
     assert vl.vosti_linear_segments(256, 64) == 1
     assert vl.vosti_linear_workspace_bytes(64, 4096, 4096) == 4 * 64 * 4096 * 4
 
