@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--pack-shared-splits", action="store_true",
                     help="create the context with VOSTI_FLAG_PACK_SHARED_SPLITS (same bits, fewer tiles "
                          "when requests share prefix pages)")
+    ap.add_argument("--device-plan", action="store_true",
+                    help="time the step as a CUDA-graph replay of vosti_plan_device + vosti_kv_append_planned + "
+                         "vosti_paged_attention_planned (metadata in device memory); same bits")
     ap.add_argument("--window", type=int, default=0,
                     help="sliding window (keys); experiments with vosti_paged_attention_ex, the e2e and "
                          "cpu_baseline legs stay unwindowed")
@@ -313,6 +316,32 @@ def main():
         else:
             vb.vosti_paged_attention(cache.ctx, q, out, ql, st, sl, bt, scale, stream=stream)
 
+    host_step = step
+    if args.device_plan:
+        # The same step with its metadata in device memory, planned by a kernel, captured once in a
+        # CUDA graph: the host's share of a step is one graph launch.
+        if max(w.q_lens) * (geo.n_q_heads // geo.n_kv_heads) > 32 or args.window:
+            raise SystemExit("--device-plan covers split-parallel batches (decode, speculative) without a window")
+        plan = torch.empty(vb.vosti_device_plan_bytes(cache.ctx), dtype=torch.uint8, device=dev)
+        ql_d, st_d, bt_d = (torch.from_numpy(np.ascontiguousarray(x)).to(dev) for x in (ql, st, bt))
+        max_q = int(max(w.q_lens))
+
+        def planned_step():
+            vb.vosti_plan_device(cache.ctx, plan, ql_d, st_d, bt_d, max_q)
+            vb.vosti_kv_append_planned(cache.ctx, plan, kn, vn, bt_d, max_q)
+            vb.vosti_paged_attention_planned(cache.ctx, plan, q, out, None, bt_d, max_q, scale)
+
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            planned_step()
+        stream.wait_stream(side)
+        torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            planned_step()
+        step = graph.replay
+
     def sync_all():
         torch.cuda.synchronize()
         if dist is not None:
@@ -335,7 +364,7 @@ def main():
         h_us.append((time.perf_counter() - t0) * 1e6 / 2)
     torch.cuda.synchronize()
 
-    def timed_pass(profile_mode):
+    def timed_pass(profile_mode, step=step):
         """K steps bracketed by barrier + synchronize, timed with CUDA events on the stream."""
         vb.vosti_profile_enable(cache.ctx, profile_mode)
         l0 = vb.vosti_launch_count(cache.ctx)
@@ -360,7 +389,15 @@ def main():
     # Pass 2, same K steps, records a CUDA event pair around every launch of the dominant kernel
     # (on the launching stream) for the roofline.  The event nodes sit between the step's kernels
     # and defeat their dependent launch, which is why they are kept out of pass 1.
-    roof_ms, _, kernel_ms, kernels_timed = timed_pass(0 if args.no_kernel_events else (2 if tile_bound else 1))
+    # (Always the host-planned step: the library records its events around its own launches.)
+    roof_ms, _, kernel_ms, kernels_timed = timed_pass(0 if args.no_kernel_events else (2 if tile_bound else 1),
+                                                      step=host_step)
+    if args.device_plan:
+        launches = 4 * args.steps        # plan, append, attention, combine per replay
+        out_graph = out.clone()
+        host_step()
+        torch.cuda.synchronize()
+        assert torch.equal(out_graph.view(torch.int16), out.view(torch.int16)), "device-planned output differs"
     assert vb.vosti_poll_device_status(cache.ctx) == vb.VOSTI_OK
 
     # end to end: host buffers in, host buffer out, every step
@@ -469,6 +506,7 @@ def main():
                           "K steps with a CUDA event pair around each launch of the dominant kernel",
                 "ms_per_step_with_kernel_events": roof_ms / args.steps,
                 "pack_shared_splits": bool(args.pack_shared_splits),
+                "device_plan": bool(args.device_plan),
                 "window": int(args.window),
                 "schedule": dict(zip(("split_items", "packed_items", "tile_items"),
                                      vb.vosti_last_schedule(cache.ctx))),

@@ -266,6 +266,54 @@ vosti_status vosti_step_host_async(vosti_ctx* ctx, const void* q_host, void* out
  * INVALID_ARG for a ticket never issued. */
 vosti_status vosti_step_host_wait(vosti_ctx* ctx, int64_t ticket);
 
+/* Device-planned steps, for decode loops replayed from a CUDA graph.  (The
+ * paper has no counterpart: this is the planning of the operation above moved
+ * to the GPU, not a different computation.)
+ *
+ * vosti_paged_attention reads its lengths and block tables on the host, so a
+ * captured graph would replay the metadata of the step it was captured on.
+ * Here q_lens, start_pos and block_tables live in DEVICE memory and may change
+ * between replays; a planning kernel turns them into the same work items the
+ * host planner makes, and the append / attention / combine kernels read those.
+ * None of the three calls below synchronises, allocates, creates events or
+ * reads device memory on the host: all may be issued while a stream is being
+ * captured, and the captured graph replayed with other metadata, Q, K/V rows
+ * and output contents at the same addresses.  Output bits are those of
+ * vosti_kv_append + vosti_paged_attention for the same logical requests.
+ *
+ * Only split-parallel requests: every q_len * (n_q_heads / n_kv_heads) <= 32
+ * (decode, speculative queries); max_q_len bounds every q_len and must satisfy
+ * the same limit (UNSUPPORTED_CONFIG otherwise).  No sliding window.  Rows of
+ * q / k_new / v_new / out are packed in request order (sum of q_lens rows),
+ * as in the host-planned calls; seq_len of a request is start_pos + q_len.
+ *
+ *   plan            device, vosti_device_plan_bytes(config) bytes, 16-byte
+ *                   aligned; written by vosti_plan_device, read by the other
+ *                   two; may be shared by contexts of equal configuration
+ *                   limits (one plan per step, one context per layer)
+ *   q_lens_dev, start_pos_dev   device [batch] int32
+ *   block_tables_dev            device [batch][block_table_stride] int32
+ *   batch, max_q_len, block_table_stride   host values, fixed at capture
+ * Metadata cannot be checked on the host.  The planning kernel checks it:
+ * a request with lengths outside the premises (negative, q_len > max_q_len,
+ * start_pos + q_len > max_seq_len or beyond block_table_stride pages) is
+ * treated as empty, a page id outside the pool is never written to (reads of
+ * it return zeros), a batch that exceeds the workspace runs nothing; in each
+ * case the device status word is set and the next vosti_poll_device_status
+ * returns VOSTI_ERR_OUT_OF_RANGE.  Errors detectable from the host values are
+ * returned by the call as usual. */
+size_t vosti_device_plan_bytes(const vosti_config* config);
+vosti_status vosti_plan_device(vosti_ctx* ctx, void* plan, const int32_t* q_lens_dev,
+                               const int32_t* start_pos_dev, const int32_t* block_tables_dev,
+                               int32_t block_table_stride, int32_t batch, int32_t max_q_len,
+                               void* cuda_stream);
+vosti_status vosti_kv_append_planned(vosti_ctx* ctx, const void* plan, const void* k_new,
+                                     const void* v_new, const int32_t* block_tables_dev, int32_t batch,
+                                     int32_t max_q_len, void* cuda_stream);
+vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, const void* q, void* out,
+                                           float* lse, const int32_t* block_tables_dev, int32_t batch,
+                                           int32_t max_q_len, float softmax_scale, void* cuda_stream);
+
 /* Split-parallel paged attention for callers that must not allocate.  (The
  * paper has no counterpart: this is a packaging variant of the operation
  * above, not a different computation.)
@@ -301,9 +349,10 @@ vosti_status vosti_paged_attention_noalloc(int32_t n_q_heads, int32_t n_kv_heads
                                            const int32_t* block_tables, int32_t block_table_stride,
                                            int32_t batch, float softmax_scale, void* cuda_stream);
 
-/* Waits for the stream and reads the device status word: VOSTI_OK, or
+/* Waits for the stream and reads the device status word: VOSTI_OK,
  * VOSTI_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is
- * then undefined).  The word is cleared by the read. */
+ * then undefined), or VOSTI_ERR_OUT_OF_RANGE if a device-planned step met
+ * metadata outside the premises.  The word is cleared by the read. */
 vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream);
 
 /* Failure-detection self-test (no GPU fault involved): launches one warp that

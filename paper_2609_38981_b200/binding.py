@@ -32,6 +32,7 @@ EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
     "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_cp_partial",
     "vosti_cp_combine", "vosti_step_host", "vosti_step_host_async", "vosti_step_host_wait",
+    "vosti_device_plan_bytes", "vosti_plan_device", "vosti_kv_append_planned", "vosti_paged_attention_planned",
     "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
     "vosti_last_schedule", "vosti_fingerprint",
@@ -101,6 +102,15 @@ _lib.vosti_step_host_async.restype = ctypes.c_int
 _lib.vosti_step_host_async.argtypes = _lib.vosti_step_host.argtypes + [ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_step_host_wait.restype = ctypes.c_int
 _lib.vosti_step_host_wait.argtypes = [_vp, ctypes.c_int64]
+_lib.vosti_device_plan_bytes.restype = ctypes.c_size_t
+_lib.vosti_device_plan_bytes.argtypes = [_cfgp]
+_lib.vosti_plan_device.restype = ctypes.c_int
+_lib.vosti_plan_device.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp]
+_lib.vosti_kv_append_planned.restype = ctypes.c_int
+_lib.vosti_kv_append_planned.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32, _vp]
+_lib.vosti_paged_attention_planned.restype = ctypes.c_int
+_lib.vosti_paged_attention_planned.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32,
+                                               ctypes.c_float, _vp]
 _lib.vosti_poll_device_status.restype = ctypes.c_int
 _lib.vosti_poll_device_status.argtypes = [_vp, _vp]
 _lib.vosti_selftest_bounded_wait.restype = ctypes.c_int
@@ -358,6 +368,33 @@ def vosti_step_host_async(ctx: Context, q_host, out_host, k_new_host, v_new_host
 
 def vosti_step_host_wait(ctx: Context, ticket: int) -> None:
     _check(_lib.vosti_step_host_wait(ctx.handle, int(ticket)), "vosti_step_host_wait")
+
+
+def vosti_device_plan_bytes(ctx: Context) -> int:
+    return int(_lib.vosti_device_plan_bytes(ctypes.byref(ctx.cfg)))
+
+
+def vosti_plan_device(ctx: Context, plan, q_lens_dev, start_pos_dev, block_tables_dev, max_q_len: int,
+                      stream=None) -> None:
+    """All array arguments are int32 CUDA tensors; `plan` a CUDA byte tensor of vosti_device_plan_bytes."""
+    _check(_lib.vosti_plan_device(ctx.handle, _dev(plan), _dev(q_lens_dev), _dev(start_pos_dev),
+                                  _dev(block_tables_dev), block_tables_dev.shape[1], q_lens_dev.shape[0],
+                                  int(max_q_len), _stream(stream)), "vosti_plan_device")
+
+
+def vosti_kv_append_planned(ctx: Context, plan, k_new, v_new, block_tables_dev, max_q_len: int,
+                            stream=None) -> None:
+    _check(_lib.vosti_kv_append_planned(ctx.handle, _dev(plan), _dev(k_new), _dev(v_new), _dev(block_tables_dev),
+                                        block_tables_dev.shape[0], int(max_q_len), _stream(stream)),
+           "vosti_kv_append_planned")
+
+
+def vosti_paged_attention_planned(ctx: Context, plan, q, out, lse, block_tables_dev, max_q_len: int,
+                                  softmax_scale: float, stream=None) -> None:
+    _check(_lib.vosti_paged_attention_planned(ctx.handle, _dev(plan), _dev(q), _dev(out), _dev(lse),
+                                              _dev(block_tables_dev), block_tables_dev.shape[0], int(max_q_len),
+                                              float(softmax_scale), _stream(stream)),
+           "vosti_paged_attention_planned")
 
 
 def vosti_poll_device_status(ctx: Context, stream=None) -> int:

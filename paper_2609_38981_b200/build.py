@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libvosti.so")
 SOURCES = ["vosti.cu", "vosti_noalloc.cu", "vosti_linear.cu", "prefix_cache.cpp"]
-HEADERS = ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", "tcgen05.cuh", os.path.join("..", "..", "include", "vosti.h"),
+HEADERS = ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "device_plan.cuh", "tile_math.cuh", "meta.cuh", "nc_math.cuh", "ptx.cuh", "tcgen05.cuh", os.path.join("..", "..", "include", "vosti.h"),
            os.path.join("..", "..", "include", "vosti_cache.h"),
            os.path.join("..", "..", "include", "vosti_linear.h")]
 

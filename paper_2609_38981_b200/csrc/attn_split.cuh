@@ -15,8 +15,6 @@
 
 namespace vosti {
 
-constexpr uint32_t kStatusTimeout = 1u;
-
 // Eight workers per SM (two per scheduler, so one worker's instruction latency
 // hides behind the other's); each owns kStages stages of 32 keys (K or V).
 template <int D>
@@ -58,6 +56,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
 
   const int G = P.G;
   const float c = P.c;
+  // A device-planned call reads items a kernel earlier in the stream wrote: nothing before it is done.
+  if (P.counts != nullptr) griddep_wait();
 
   // ---- tickets ---------------------------------------------------------------
   // Producer-side description of an item: enough to issue its loads.
@@ -84,7 +84,8 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
       if (lane == 0) t = n_static + atomicAdd(P.ticket, 1u);
       t = __shfl_sync(kFullMask, t, 0);
     }
-    if (t >= static_cast<uint32_t>(P.n_workers)) return false;
+    const uint32_t n_workers = P.counts != nullptr ? static_cast<uint32_t>(__ldg(P.counts)) : static_cast<uint32_t>(P.n_workers);
+    if (t >= n_workers) return false;
     const SplitItem si = read_item(t);
     int t_end, t_first;
     if (si.req < 0) {  // packed rows: every row sees the whole split
@@ -104,6 +105,12 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     d.n_loads = LPT * (t_end - d.t_begin);
     d.n_pages = si.n_pages;
     d.ids = (si.split * nc::kPagesPerSplit + lane < si.n_pages) ? __ldg(P.bt_flat + si.bt_index + lane) : -1;
+    if (P.counts != nullptr) {  // nobody has looked at these page ids yet: report strays, read page 0 instead
+      const bool stray = d.ids < -1 || d.ids >= P.num_pages ||
+                         (d.ids == -1 && si.split * nc::kPagesPerSplit + lane < si.n_pages);
+      if (__any_sync(kFullMask, stray) && lane == 0) atomicOr(P.status, kStatusBadMetadata);
+      if (stray) d.ids = 0;
+    }
     return true;
   };
   auto leave = [&]() {

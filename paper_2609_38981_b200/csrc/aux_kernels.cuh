@@ -15,7 +15,8 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
   constexpr int BATCH = 8;    // partial rows whose loads are in flight together
   const int lane = threadIdx.x & 31;
   const int widx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (widx >= P.n_split_tokens * P.Hq) return;
+  if (P.counts != nullptr) griddep_wait();  // device-planned: the metadata too comes from the stream
+  if (widx >= (P.counts != nullptr ? P.counts[1] : P.n_split_tokens) * P.Hq) return;
   // Metadata does not depend on the kernel before this one: read it first, so that
   // only the partial rows themselves wait for the attention kernel to finish.
   const int2 rt = P.split_tokens[widx / P.Hq];

@@ -7,6 +7,10 @@
 
 namespace vosti {
 
+// Bits of the device status word.
+constexpr uint32_t kStatusTimeout = 1u;      // a bounded wait gave up
+constexpr uint32_t kStatusBadMetadata = 2u;  // a device-planned step met lengths / page ids outside the premises
+
 // One request of a call, as the kernels see it.
 struct ReqMeta {
   int32_t q_row0;     // first packed row of the request
@@ -63,6 +67,10 @@ struct AttnParams {
   float c;                   // sigma * log2(e), rounded once on the host
   int32_t window;            // sliding window w: key j visible iff p - w < j <= p; 0 = no window
   float* lse;                // optional [T][Hq] natural-log log-sum-exp output, or nullptr
+  // Device-planned calls: {n_workers, n_split_tokens} written by the planning kernel earlier in
+  // the stream (the two fields above are then only upper bounds for the grids); nullptr otherwise.
+  const int32_t* counts;
+  int32_t num_pages;         // device-planned calls: page ids are checked against it when an item is drawn
 };
 
 struct AppendParams {

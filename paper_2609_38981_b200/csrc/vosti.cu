@@ -11,6 +11,7 @@
 #include "attn_split.cuh"
 #include "attn_tile.cuh"
 #include "aux_kernels.cuh"
+#include "device_plan.cuh"
 
 namespace vosti {
 namespace {
@@ -974,6 +975,8 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
   p.window = window;
   p.lse = lse;
+  p.counts = nullptr;
+  p.num_pages = 0;
   ctx->last_split_items = n_split_final;
   ctx->last_packed_items = n_packed_items;
   ctx->last_tile_items = n_seq;
@@ -1076,6 +1079,157 @@ vosti_status vosti_step_host(vosti_ctx* ctx, const void* q_host, void* out_host,
   return st == VOSTI_OK ? vosti_step_host_wait(ctx, ticket) : st;
 }
 
+// ---- device-planned steps (graph capture) ------------------------------------------------------
+
+size_t vosti_device_plan_bytes(const vosti_config* config) {
+  if (!config || !geometry_ok(*config)) return 0;
+  return device_plan_layout(config->max_batch, config->max_total_q, config->max_seq_len).total;
+}
+
+namespace {
+// Premises every device-planned call shares; host-side, so they are reported at once.
+vosti_status planned_call_ok(const vosti_ctx* ctx, const void* plan, const int32_t* block_tables_dev,
+                             int32_t batch, int32_t max_q_len) {
+  if (!ctx || !plan || batch < 0 || max_q_len < 1) return VOSTI_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(plan) % 16) return VOSTI_ERR_INVALID_ARG;
+  if (batch > 0 && !block_tables_dev) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  if (batch > c.max_batch) return VOSTI_ERR_OUT_OF_RANGE;
+  if (int64_t{max_q_len} * (c.n_q_heads / c.n_kv_heads) > nc::kSplitRowsMax) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  if (ctx->lim.part_rows_max >= (int64_t{1} << 31)) return VOSTI_ERR_WORKSPACE;  // the planner counts in 32 bits
+  return VOSTI_OK;
+}
+}  // namespace
+
+vosti_status vosti_plan_device(vosti_ctx* ctx, void* plan, const int32_t* q_lens_dev,
+                               const int32_t* start_pos_dev, const int32_t* block_tables_dev,
+                               int32_t block_table_stride, int32_t batch, int32_t max_q_len,
+                               void* cuda_stream) {
+  vosti_status st = planned_call_ok(ctx, plan, block_tables_dev, batch, max_q_len);
+  if (st != VOSTI_OK) return st;
+  if (block_table_stride < 0 || (batch > 0 && (!q_lens_dev || !start_pos_dev))) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  const DevicePlanLayout L = device_plan_layout(c.max_batch, c.max_total_q, c.max_seq_len);
+  uint8_t* base = static_cast<uint8_t*>(plan);
+  DevicePlanArgs a{};
+  a.q_lens = q_lens_dev;
+  a.start_pos = start_pos_dev;
+  a.block_tables = block_tables_dev;
+  a.stride = block_table_stride;
+  a.batch = batch;
+  a.max_q_len = max_q_len;
+  a.G = c.n_q_heads / c.n_kv_heads;
+  a.Hkv = c.n_kv_heads;
+  a.num_pages = c.num_pages;
+  a.max_seq_len = c.max_seq_len;
+  a.items_max = std::min(L.items_max, ctx->lim.items_max);
+  a.toks_max = L.toks_max;
+  a.part_rows_max = ctx->lim.part_rows_max;
+  a.header = reinterpret_cast<DevicePlanHeader*>(base);
+  a.reqs = reinterpret_cast<ReqMeta*>(base + L.off_reqs);
+  a.items = reinterpret_cast<SplitItem*>(base + L.off_items);
+  a.toks = reinterpret_cast<int2*>(base + L.off_toks);
+  a.scratch = reinterpret_cast<DevicePlanScratch*>(base + L.off_scratch);
+  a.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (launch_dependent(device_plan_kernel, 1, batch <= 256 ? 256 : kPlanThreads, 0, stream, a) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  ++ctx->launches;
+  return VOSTI_OK;
+}
+
+vosti_status vosti_kv_append_planned(vosti_ctx* ctx, const void* plan, const void* k_new, const void* v_new,
+                                     const int32_t* block_tables_dev, int32_t batch, int32_t max_q_len,
+                                     void* cuda_stream) {
+  vosti_status st = planned_call_ok(ctx, plan, block_tables_dev, batch, max_q_len);
+  if (st != VOSTI_OK) return st;
+  if (batch == 0) return VOSTI_OK;
+  if (!k_new || !v_new) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(k_new) | reinterpret_cast<uintptr_t>(v_new)) % 16) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  const DevicePlanLayout L = device_plan_layout(c.max_batch, c.max_total_q, c.max_seq_len);
+  AppendPlannedParams p{};
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.pool = static_cast<__nv_bfloat16*>(c.kv_pool);
+  p.reqs = reinterpret_cast<const ReqMeta*>(static_cast<const uint8_t*>(plan) + L.off_reqs);
+  p.block_tables = block_tables_dev;
+  p.batch = batch;
+  p.max_q_len = max_q_len;
+  p.Hkv = c.n_kv_heads;
+  p.num_pages = c.num_pages;
+  p.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status);
+  const int64_t warps = int64_t{batch} * max_q_len * c.n_kv_heads;
+  const int grid = static_cast<int>((warps + 3) / 4);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const cudaError_t e = c.head_dim == 128
+                            ? launch_dependent(kv_append_planned_kernel<128>, grid, 128, 0, stream, p)
+                            : launch_dependent(kv_append_planned_kernel<64>, grid, 128, 0, stream, p);
+  if (e != cudaSuccess) return VOSTI_ERR_CUDA;
+  ++ctx->launches;
+  return VOSTI_OK;
+}
+
+extern "C++" {
+namespace {
+template <int D>
+vosti_status launch_attention_planned(vosti_ctx* ctx, const AttnParams& p, cudaStream_t stream) {
+  using Cfg = SplitKernelCfg<D>;
+  // The item count is known to the device only: a full persistent grid, whose idle workers leave at once.
+  if (launch_dependent(attn_split_kernel<D>, ctx->sm_count, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3,
+                       p) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  const int64_t warps = int64_t{p.n_split_tokens} * p.Hq;
+  if (launch_dependent(combine_kernel<D>, static_cast<int>((warps + 3) / 4), 128, 0, stream, p) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  ctx->launches += 2;
+  return VOSTI_OK;
+}
+}  // namespace
+}  // extern "C++"
+
+vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, const void* q, void* out, float* lse,
+                                           const int32_t* block_tables_dev, int32_t batch, int32_t max_q_len,
+                                           float softmax_scale, void* cuda_stream) {
+  vosti_status st = planned_call_ok(ctx, plan, block_tables_dev, batch, max_q_len);
+  if (st != VOSTI_OK) return st;
+  if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
+  if (batch == 0) return VOSTI_OK;
+  if (!q || !out) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16) return VOSTI_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(lse) % 4) return VOSTI_ERR_INVALID_ARG;
+  const vosti_config& c = ctx->cfg;
+  const DevicePlanLayout L = device_plan_layout(c.max_batch, c.max_total_q, c.max_seq_len);
+  const uint8_t* base = static_cast<const uint8_t*>(plan);
+  AttnParams p{};
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.reqs = reinterpret_cast<const ReqMeta*>(base + L.off_reqs);
+  p.items = nullptr;
+  p.split_items = reinterpret_cast<const SplitItem*>(base + L.off_items);
+  p.packed_rows = nullptr;
+  p.ticket = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 64);
+  p.done = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status + 128);
+  p.bt_flat = block_tables_dev;
+  p.split_tokens = reinterpret_cast<const int2*>(base + L.off_toks);
+  p.ws_u = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_part_u);
+  p.ws_mz = reinterpret_cast<float2*>(ctx->ws + ctx->lim.off_part_mz);
+  p.ws_uc = reinterpret_cast<float*>(ctx->ws + ctx->lim.off_uc);
+  p.status = reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status);
+  p.n_workers = 0;
+  p.n_split_tokens = static_cast<int32_t>(std::min<int64_t>(int64_t{batch} * max_q_len, L.toks_max));  // grid bound
+  p.Hq = c.n_q_heads;
+  p.Hkv = c.n_kv_heads;
+  p.G = c.n_q_heads / c.n_kv_heads;
+  p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
+  p.window = 0;
+  p.lse = lse;
+  p.counts = reinterpret_cast<const int32_t*>(base);
+  p.num_pages = static_cast<int32_t>(c.num_pages);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  return c.head_dim == 128 ? launch_attention_planned<128>(ctx, p, stream) : launch_attention_planned<64>(ctx, p, stream);
+}
+
 vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
   if (!ctx) return VOSTI_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -1085,7 +1239,8 @@ vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
       cudaMemsetAsync(d, 0, kAlign, stream) != cudaSuccess ||
       cudaStreamSynchronize(stream) != cudaSuccess)
     return VOSTI_ERR_CUDA;
-  return (word & kStatusTimeout) ? VOSTI_ERR_TIMEOUT : VOSTI_OK;
+  if (word & kStatusTimeout) return VOSTI_ERR_TIMEOUT;
+  return (word & kStatusBadMetadata) ? VOSTI_ERR_OUT_OF_RANGE : VOSTI_OK;
 }
 
 vosti_status vosti_selftest_bounded_wait(vosti_ctx* ctx, uint32_t limit_us, void* cuda_stream) {

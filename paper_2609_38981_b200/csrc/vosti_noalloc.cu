@@ -235,6 +235,8 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
   p.window = 0;
   p.lse = nullptr;
+  p.counts = nullptr;
+  p.num_pages = 0;
   p.packed_rows = nullptr;
   return head_dim == 128 ? launch<128>(map, p, sm_count, stream) : launch<64>(map, p, sm_count, stream);
 }

@@ -1,0 +1,222 @@
+"""Device-planned decode steps: lengths, start positions and block tables in
+device memory, planned by a kernel, so that a step can be captured once in a
+CUDA graph and replayed with other metadata.  The outputs, the log-sum-exp and
+the KV written to the pool must be, bit for bit, those of the host-planned
+calls for the same logical requests; metadata outside the premises sets the
+device status word and faults nothing."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_38981_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+GEOS = {
+    "d128_g4": (inputs.Geometry(8, 2, 128, 16), 4),      # geometry, largest q_len that stays split-parallel (tested)
+    "d64_g2": (inputs.TINY, 4),
+    "d128_g8": (inputs.Geometry(8, 1, 128, 16), 4),
+    "d128_g16": (inputs.Geometry(16, 1, 128, 16), 2),
+}
+# contexts around page, tile and split edges; each request also has a tail of positions to decode
+CONTEXTS = (1, 17, 64, 300, 511, 512, 513, 1030, 1600)
+TAIL = 13
+NUM_PAGES = 1024
+MAXLEN = 2048
+
+
+class Env:
+    def __init__(self, geo):
+        from paper_2609_38981_b200.harness import DeviceCache
+        self.geo = geo
+        self.scale = geo.head_dim ** -0.5
+        self.reqs = [inputs.make_request(geo, 777, i, n + TAIL) for i, n in enumerate(CONTEXTS)]
+        self.tables = inputs._assign_private_pages(inputs.generator(777), geo, NUM_PAGES, [r.n for r in self.reqs])
+        self.bt = inputs.block_table_array(self.tables)
+        self.new_cache = lambda: DeviceCache(geo, NUM_PAGES, max_batch=16, max_total_q=2048, max_seq_len=MAXLEN,
+                                             pool_fill="nan")
+
+    def prefill(self, cache):
+        cache.upload(self.reqs, self.tables, upto=list(CONTEXTS))
+
+    def rows(self, call):
+        q = torch.cat([self.reqs[i].q_rows(s, n) for i, s, n in call if n > 0]).cuda().contiguous()
+        k = torch.cat([self.reqs[i].k[s:s + n] for i, s, n in call if n > 0]).cuda().contiguous()
+        v = torch.cat([self.reqs[i].v[s:s + n] for i, s, n in call if n > 0]).cuda().contiguous()
+        return q, k, v
+
+
+@pytest.fixture(scope="module", params=list(GEOS))
+def env(request):
+    geo, max_q = GEOS[request.param]
+    e = Env(geo)
+    e.max_q = max_q
+    return e
+
+
+def host_step(env, cache, call):
+    from paper_2609_38981_b200 import binding as vb
+    q, k, v = env.rows(call)
+    ql, st = [n for _, _, n in call], [s for _, s, _ in call]
+    vb.vosti_kv_append(cache.ctx, k, v, ql, st, env.bt)
+    out = torch.empty_like(q)
+    out.view(torch.int16).fill_(0x7FC1)
+    lse = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+    vb.vosti_paged_attention_ex(cache.ctx, q, out, lse, ql, st, [s + n for _, s, n in call], env.bt, env.scale)
+    return out, lse
+
+
+def device_step(env, cache, plan, call, max_q_len):
+    from paper_2609_38981_b200 import binding as vb
+    q, k, v = env.rows(call)
+    ql = torch.tensor([n for _, _, n in call], dtype=torch.int32, device="cuda")
+    st = torch.tensor([s for _, s, _ in call], dtype=torch.int32, device="cuda")
+    bt = torch.from_numpy(env.bt).cuda()
+    out = torch.empty_like(q)
+    out.view(torch.int16).fill_(0x7FC1)
+    lse = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+    vb.vosti_plan_device(cache.ctx, plan, ql, st, bt, max_q_len)
+    vb.vosti_kv_append_planned(cache.ctx, plan, k, v, bt, max_q_len)
+    vb.vosti_paged_attention_planned(cache.ctx, plan, q, out, lse, bt, max_q_len, env.scale)
+    return out, lse
+
+
+def new_plan(cache):
+    from paper_2609_38981_b200 import binding as vb
+    n = vb.vosti_device_plan_bytes(cache.ctx)
+    assert n > 0
+    return torch.empty(n, dtype=torch.uint8, device="cuda")
+
+
+def same(a, b, what):
+    assert torch.equal(a.view(torch.int16), b.view(torch.int16)), f"{what}: outputs differ bitwise"
+
+
+def test_decode_and_speculative_steps_equal_the_host_planned_calls(env):
+    from paper_2609_38981_b200 import binding as vb
+    host, dev = env.new_cache(), env.new_cache()
+    env.prefill(host)
+    env.prefill(dev)
+    plan = new_plan(dev)
+    done = list(CONTEXTS)
+    rng = np.random.default_rng(5)
+    for step in range(6):
+        # a mix of query lengths per request, zero included (a request that sits a step out)
+        ql = [int(rng.integers(0, env.max_q + 1)) for _ in CONTEXTS] if step else [1] * len(CONTEXTS)
+        ql = [min(n, c + TAIL - d) for n, c, d in zip(ql, CONTEXTS, done)]
+        if sum(ql) == 0:
+            ql[0] = 1
+        call = [(i, done[i], ql[i]) for i in range(len(CONTEXTS))]
+        oh, lh = host_step(env, host, call)
+        od, ld = device_step(env, dev, plan, call, env.max_q)
+        same(od, oh, f"step {step}, q_lens {ql}")
+        assert torch.equal(ld.view(torch.int32), lh.view(torch.int32)), f"step {step}: log-sum-exp differs bitwise"
+        assert not (od.view(torch.int16) == 0x7FC1).any()
+        done = [d + n for d, n in zip(done, ql)]
+    used = sorted({p for t in env.tables for p in t})
+    assert torch.equal(host.pool[used].view(torch.int16), dev.pool[used].view(torch.int16))   # appended KV
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK
+    host.close()
+    dev.close()
+
+
+def test_a_captured_graph_replays_with_new_metadata(env):
+    """One capture of plan + append + attention; every replay advances the device-side start
+    positions and refills the static Q / K / V buffers."""
+    from paper_2609_38981_b200 import binding as vb
+    geo, B = env.geo, len(CONTEXTS)
+    host, dev = env.new_cache(), env.new_cache()
+    env.prefill(host)
+    env.prefill(dev)
+    plan = new_plan(dev)
+    ql = torch.ones(B, dtype=torch.int32, device="cuda")
+    st = torch.tensor(CONTEXTS, dtype=torch.int32, device="cuda")
+    bt = torch.from_numpy(env.bt).cuda()
+    q = torch.zeros((B, geo.n_q_heads, geo.head_dim), dtype=torch.bfloat16, device="cuda")
+    k = torch.zeros((B, geo.n_kv_heads, geo.head_dim), dtype=torch.bfloat16, device="cuda")
+    v = torch.zeros_like(k)
+    out = torch.zeros_like(q)
+    lse = torch.zeros((B, geo.n_q_heads), dtype=torch.float32, device="cuda")
+
+    def fill(step):
+        call = [(i, CONTEXTS[i] + step, 1) for i in range(B)]
+        qs, ks, vs = env.rows(call)
+        q.copy_(qs)
+        k.copy_(ks)
+        v.copy_(vs)
+        st.copy_(torch.tensor([s for _, s, _ in call], dtype=torch.int32))
+        return call
+
+    fill(0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):          # one eager run first: lazy module loading must not happen under capture
+        vb.vosti_plan_device(dev.ctx, plan, ql, st, bt, 1)
+        vb.vosti_paged_attention_planned(dev.ctx, plan, q, out, lse, bt, 1, env.scale)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        vb.vosti_plan_device(dev.ctx, plan, ql, st, bt, 1)
+        vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt, 1)
+        vb.vosti_paged_attention_planned(dev.ctx, plan, q, out, lse, bt, 1, env.scale)
+    for step in range(TAIL):
+        call = fill(step)
+        out.view(torch.int16).fill_(0x7FC1)
+        graph.replay()
+        oh, lh = host_step(env, host, call)
+        same(out, oh, f"replay {step}")
+        assert torch.equal(lse.view(torch.int32), lh.view(torch.int32)), f"replay {step}: log-sum-exp differs"
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK
+    host.close()
+    dev.close()
+
+
+def test_bad_metadata_sets_the_status_word_and_spares_the_rest(env):
+    from paper_2609_38981_b200 import binding as vb
+    host, dev = env.new_cache(), env.new_cache()
+    env.prefill(host)
+    env.prefill(dev)
+    plan = new_plan(dev)
+    call = [(i, CONTEXTS[i], 1) for i in range(len(CONTEXTS))]
+    oh, _ = host_step(env, host, call)
+    q, k, v = env.rows(call)
+    st = torch.tensor(CONTEXTS, dtype=torch.int32, device="cuda")
+    bt = torch.from_numpy(env.bt).cuda()
+    # request 3 claims more query rows than the call allows, request 5 a negative start
+    ql = torch.ones(len(CONTEXTS), dtype=torch.int32, device="cuda")
+    for bad_ql, bad_st in (({3: env.max_q + 1}, {}), ({}, {5: -4}), ({2: -1}, {}), ({}, {6: MAXLEN})):
+        ql2, st2 = ql.clone(), st.clone()
+        for i, x in bad_ql.items():
+            ql2[i] = x
+        for i, x in bad_st.items():
+            st2[i] = x
+        out = torch.empty_like(q)
+        out.view(torch.int16).fill_(0x7FC1)
+        vb.vosti_plan_device(dev.ctx, plan, ql2, st2, bt, env.max_q)
+        vb.vosti_paged_attention_planned(dev.ctx, plan, q, out, None, bt, env.max_q, env.scale)
+        assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_ERR_OUT_OF_RANGE
+        assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK          # cleared by the read
+    # a page id outside the pool: reported, never written through
+    bt_bad = bt.clone()
+    bt_bad[4, CONTEXTS[4] // 16] = NUM_PAGES + 5
+    snapshot = dev.pool.clone()
+    vb.vosti_plan_device(dev.ctx, plan, ql, st, bt_bad, 1)
+    vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt_bad, 1)
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_ERR_OUT_OF_RANGE
+    touched = sorted({env.tables[i][CONTEXTS[i] // 16] for i in range(len(CONTEXTS)) if i != 4})
+    rest = [p for p in range(NUM_PAGES) if p not in touched]
+    assert torch.equal(dev.pool[rest].view(torch.int16), snapshot[rest].view(torch.int16))
+    # and a clean step afterwards is right again (the append above wrote every request but the fourth)
+    vb.vosti_plan_device(dev.ctx, plan, ql, st, bt, 1)
+    vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt, 1)
+    out = torch.empty_like(q)
+    vb.vosti_paged_attention_planned(dev.ctx, plan, q, out, None, bt, 1, env.scale)
+    same(out, oh, "after the rejected steps")
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK
+    # host-detectable errors are returned by the call
+    with pytest.raises(vb.VostiError) as e:
+        vb.vosti_plan_device(dev.ctx, plan, ql, st, bt, 40)
+    assert e.value.status == vb.VOSTI_ERR_UNSUPPORTED_CONFIG
+    host.close()
+    dev.close()
