@@ -528,8 +528,10 @@ def main():
         }
         if world == 1 and not args.no_cpu_baseline:
             ostep, cores = oracle_step_factory(w)
+            c0 = time.perf_counter()
             ostep()
-            reps = 8
+            # about ten seconds of host work: enough repetitions to average out the box's other tenants
+            reps = int(min(400, max(8, 10.0 / max(time.perf_counter() - c0, 1e-3))))
             c0 = time.perf_counter()
             for _ in range(reps):
                 ref = ostep()
