@@ -135,6 +135,9 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
   __shared__ int warp_totals[32][NV];
   __shared__ int bucket_base[TPS + 1];
   __shared__ int bad;
+  // full_prefix of every request, for the binary searches of phase B2 (global scratch beyond 1024 requests)
+  __shared__ int full_prefix_s[kPlanThreads];
+  const bool prefix_in_smem = A.batch <= kPlanThreads;
   const int tid = threadIdx.x, n_threads = blockDim.x;
   if (tid == 0) bad = 0;
   griddep_wait();  // the metadata may come from a kernel earlier in the stream
@@ -189,6 +192,7 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
       A.reqs[r] = m;
       DevicePlanScratch s;
       s.full_prefix = carry[2] + pre[2];
+      if (prefix_in_smem) full_prefix_s[r] = s.full_prefix;
       s.tail_rel[0] = s.tail_rel[1] = -1;
 #pragma unroll
       for (int t = 1; t < TPS; ++t) {
@@ -263,11 +267,12 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
     int lo = 0, hi = A.batch - 1;  // last request whose full_prefix <= j and that owns full items
     while (lo < hi) {
       const int mid = (lo + hi + 1) >> 1;
-      if (A.scratch[mid].full_prefix <= j) lo = mid; else hi = mid - 1;
+      const int at_mid = prefix_in_smem ? full_prefix_s[mid] : A.scratch[mid].full_prefix;
+      if (at_mid <= j) lo = mid; else hi = mid - 1;
     }
     const int r = lo;
     const ReqMeta m = A.reqs[r];
-    const int local = j - A.scratch[r].full_prefix;
+    const int local = j - (prefix_in_smem ? full_prefix_s[r] : A.scratch[r].full_prefix);
     const int groups = (m.q_len * A.G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
     int f[2] = {0, 0};
     for (int x = 0; x < groups; ++x) {
