@@ -220,3 +220,29 @@ def test_bad_metadata_sets_the_status_word_and_spares_the_rest(env):
     assert e.value.status == vb.VOSTI_ERR_UNSUPPORTED_CONFIG
     host.close()
     dev.close()
+
+
+def test_one_plan_serves_the_contexts_of_several_layers(env):
+    """A plan written through one context drives another context of the same configuration
+    (another layer's pool): planning happens once per step, not once per layer."""
+    from paper_2609_38981_b200 import binding as vb
+    host, layer_a, layer_b = env.new_cache(), env.new_cache(), env.new_cache()
+    env.prefill(host)
+    env.prefill(layer_b)
+    plan = new_plan(layer_a)
+    call = [(i, CONTEXTS[i], 1) for i in range(len(CONTEXTS))]
+    oh, lh = host_step(env, host, call)
+    q, k, v = env.rows(call)
+    ql = torch.ones(len(CONTEXTS), dtype=torch.int32, device="cuda")
+    st = torch.tensor(CONTEXTS, dtype=torch.int32, device="cuda")
+    bt = torch.from_numpy(env.bt).cuda()
+    out = torch.empty_like(q)
+    lse = torch.empty(q.shape[:2], dtype=torch.float32, device="cuda")
+    vb.vosti_plan_device(layer_a.ctx, plan, ql, st, bt, 1)
+    vb.vosti_kv_append_planned(layer_b.ctx, plan, k, v, bt, 1)
+    vb.vosti_paged_attention_planned(layer_b.ctx, plan, q, out, lse, bt, 1, env.scale)
+    same(out, oh, "plan from another context")
+    assert torch.equal(lse.view(torch.int32), lh.view(torch.int32))
+    for c in (host, layer_a, layer_b):
+        assert vb.vosti_poll_device_status(c.ctx) == vb.VOSTI_OK
+        c.close()
