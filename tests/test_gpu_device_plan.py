@@ -246,3 +246,52 @@ def test_one_plan_serves_the_contexts_of_several_layers(env):
     for c in (host, layer_a, layer_b):
         assert vb.vosti_poll_device_status(c.ctx) == vb.VOSTI_OK
         c.close()
+
+
+@pytest.mark.parametrize("batch", [300, 1500])
+def test_large_batches_are_planned_in_chunks(batch):
+    """More requests than the planner has threads (and than its shared-memory prefix holds):
+    the scan carries over chunks of requests and the item search falls back to global memory."""
+    from paper_2609_38981_b200 import binding as vb
+    from paper_2609_38981_b200.harness import DeviceCache
+    geo = inputs.Geometry(8, 2, 128, 16)
+    scale = geo.head_dim ** -0.5
+    rng = np.random.default_rng(batch)
+    ctx = [int(x) for x in rng.integers(1, 700, size=batch)]
+    ctx[:4] = [511, 512, 513, 1]
+    qls = [int(x) for x in rng.integers(0, 5, size=batch)]          # decode, speculative, idle
+    qls[:4] = [4, 1, 2, 1]
+    n_pages = sum(inputs.pages_needed(c + q, geo.page_size) for c, q in zip(ctx, qls))
+    num_pages = n_pages + 64
+    reqs = [inputs.make_request(geo, 4321, i, c + q) for i, (c, q) in enumerate(zip(ctx, qls))]
+    tables = inputs._assign_private_pages(inputs.generator(batch), geo, num_pages, [r.n for r in reqs])
+    bt = inputs.block_table_array(tables)
+    mk = lambda: DeviceCache(geo, num_pages, max_batch=2048, max_total_q=8192, max_seq_len=1024, pool_fill="nan")
+    host, dev = mk(), mk()
+    for c in (host, dev):
+        c.upload(reqs, tables, upto=ctx)
+    call = [(i, ctx[i], qls[i]) for i in range(batch)]
+    q = torch.cat([reqs[i].q_rows(s, n) for i, s, n in call if n > 0]).cuda().contiguous()
+    k = torch.cat([reqs[i].k[s:s + n] for i, s, n in call if n > 0]).cuda().contiguous()
+    v = torch.cat([reqs[i].v[s:s + n] for i, s, n in call if n > 0]).cuda().contiguous()
+    oh, od = torch.empty_like(q), torch.empty_like(q)
+    for o in (oh, od):
+        o.view(torch.int16).fill_(0x7FC1)
+    lh = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+    ld = lh.clone()
+    vb.vosti_kv_append(host.ctx, k, v, qls, ctx, bt)
+    vb.vosti_paged_attention_ex(host.ctx, q, oh, lh, qls, ctx, [c + n for c, n in zip(ctx, qls)], bt, scale)
+    plan = new_plan(dev)
+    ql_d = torch.tensor(qls, dtype=torch.int32, device="cuda")
+    st_d = torch.tensor(ctx, dtype=torch.int32, device="cuda")
+    bt_d = torch.from_numpy(bt).cuda()
+    vb.vosti_plan_device(dev.ctx, plan, ql_d, st_d, bt_d, 4)
+    vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt_d, 4)
+    vb.vosti_paged_attention_planned(dev.ctx, plan, q, od, ld, bt_d, 4, scale)
+    same(od, oh, f"batch {batch}")
+    assert torch.equal(ld.view(torch.int32), lh.view(torch.int32))
+    assert not (od.view(torch.int16) == 0x7FC1).any()
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK
+    assert vb.vosti_last_schedule(host.ctx)[0] > batch          # more items than requests: several splits and groups
+    host.close()
+    dev.close()
