@@ -283,6 +283,242 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
 }
 
+// ---- the same contract on CTA pairs -------------------------------------------------------------
+// Two CTAs of a cluster (the two SMs of a TPC) compute one 256 x 256 tile with tcgen05.mma
+// cta_group::2: each loads its own 128 rows of x and its own 128 of the tile's 256 weight rows,
+// the pair's instruction reads both halves of the weight tile, and each SM's tensor memory
+// receives its 128 rows of the result.  Per SM and K block that is 32 KB from L2 instead of 48 KB,
+// so six stages fit where four did.  An output element is still the same chain of K = 16
+// products in ascending K order, segment by segment: the bits are those of linear_kernel
+// (tested), and which kernel runs is a scheduling decision.
+struct PairCfg {
+  static constexpr int kBM = 128, kBN = 256, kBK = 64;   // kBM: rows per CTA; the pair's tile is 256 x 256
+  static constexpr int kStages = 6;
+  static constexpr int kABytes = kBM * kBK * 2;
+  static constexpr int kBBytes = (kBN / 2) * kBK * 2;    // this CTA's half of the weight tile
+  static constexpr int kStageBytes = kABytes + kBBytes;
+  static constexpr int kEpiWarps = 8;
+  static constexpr int kThreads = 64 + 32 * kEpiWarps;
+  static constexpr int kSmemBytes = kStages * kStageBytes + 256 + 1024;
+  static constexpr uint32_t kTmemCols = 2 * kBN;
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// The address, in the cluster's shared window, of `addr` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA load into this CTA's shared memory whose bytes are counted on the leader CTA's mbarrier.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y,
+                                                 uint32_t leader_bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(leader_bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive, once the pair's MMAs issued so far have completed, on the barrier at this offset in both CTAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  const uint16_t both = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::
+                   "r"(bar), "h"(both)
+               : "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(PairCfg::kThreads, 1)
+linear_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
+                   __nv_bfloat16* __restrict__ y, int M, int N, int K) {
+  using Cfg = PairCfg;
+  constexpr int NS = Cfg::kStages;
+  constexpr int BN = Cfg::kBN;
+  constexpr uint32_t kAbortAfterNs = 1000000000u;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t bars = base + NS * Cfg::kStageBytes;
+  // full, acc_empty: the leader's copies are used; empty, acc_full: each CTA's own
+  const uint32_t full = bars, empty = bars + 8 * NS, acc_full = bars + 16 * NS, acc_empty = acc_full + 16;
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(sbase + NS * Cfg::kStageBytes + 192);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles = (M + 2 * Cfg::kBM - 1) / (2 * Cfg::kBM);
+  const int n_cols = N / BN;
+  const int n_tiles = m_tiles * n_cols;
+  const Segments seg = segments_of(N, K, BN);
+
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) {
+      mbar_init(full + 8 * i, 1);
+      mbar_init(empty + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(acc_full + 8 * i, 1);
+      mbar_init(acc_empty + 8 * i, 2 * Cfg::kEpiWarps);  // one arrival per epilogue warp of either CTA
+    }
+    flags[0] = 0u;
+    mbar_fence_init();
+    tma_prefetch_desc(&x_map);
+    tma_prefetch_desc(&w_map);
+  }
+  if (warp == 1) {  // the same warp of both CTAs, the same shared-memory offset
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(bars + 200),
+                 "r"(Cfg::kTmemCols));
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers exist before anything is sent to them
+  tc_fence_after();
+  const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(sbase + NS * Cfg::kStageBytes + 200);
+
+  auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 0;; ++it) {
+      if (mbar_try_wait_hint(bar, parity, 2000u)) return true;
+      if ((it & 63u) == 63u) {
+        if (flags[0] != 0u) return false;
+        if (global_timer_ns() - t0 > kAbortAfterNs) {
+          flags[0] = 1u;
+          atomicOr(&g_linear_status, 1u);
+          return false;
+        }
+      }
+    }
+  };
+
+  if (warp == 0) {
+    // ================= TMA producer (both CTAs) ==============================================
+    if (lane == 0) {
+      griddep_wait();
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        const TileCoord tc = tile_coord<2 * Cfg::kBM, BN>(tile, m_tiles, n_cols);
+        for (int kb = 0; kb < seg.k_blocks; ++kb, ++it) {
+          const uint32_t s = it % NS, use = it / NS;
+          if (use > 0) ok = wait(empty + 8 * s, (use - 1) & 1);
+          if (!ok) break;
+          const uint32_t dst = base + s * Cfg::kStageBytes;
+          const uint32_t leader_full = map_to_cta(full + 8 * s, 0);
+          if (rank == 0) mbar_expect_tx(full + 8 * s, 2 * Cfg::kStageBytes);  // both CTAs' bytes
+          tma_load_2d_pair(dst, &x_map, kb * Cfg::kBK, tc.m0 + static_cast<int>(rank) * Cfg::kBM, leader_full);
+          tma_load_2d_pair(dst + Cfg::kABytes, &w_map, kb * Cfg::kBK, tc.n0 + static_cast<int>(rank) * (BN / 2),
+                           leader_full);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ================= MMA issuer (one thread of the leader CTA) ==============================
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = umma_idesc(2 * Cfg::kBM, BN, false);
+      uint32_t it = 0, step = 0;
+      bool ok = true;
+      for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+        for (int sj = 0; sj < seg.n_seg && ok; ++sj, ++step) {
+          const uint32_t buf = step & 1, acc_use = step >> 1;
+          if (acc_use > 0) ok = wait(acc_empty + 8 * buf, (acc_use - 1) & 1);  // both epilogues have drained it
+          if (!ok) break;
+          tc_fence_after();
+          const int kb0 = seg.begin(sj), kb1 = seg.begin(sj + 1);
+          for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            const uint32_t s = it % NS;
+            ok = wait(full + 8 * s, (it / NS) & 1);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a = base + s * Cfg::kStageBytes, b = a + Cfg::kABytes;
+#pragma unroll
+            for (int kc = 0; kc < Cfg::kBK / 16; ++kc)
+              tc_mma_ss_pair(tmem + buf * BN, smem_desc_sw128(a + kc * 32, 16, 1024),
+                             smem_desc_sw128(b + kc * 32, 16, 1024), idesc, (kb > kb0 || kc > 0) ? 1u : 0u);
+            tc_commit_pair(empty + 8 * s);
+          }
+          if (!ok) break;
+          tc_commit_pair(acc_full + 8 * buf);
+        }
+      }
+    }
+  } else {
+    // ================= epilogue (both CTAs): a thread owns 128 columns of one of its CTA's rows =
+    const int e = warp - 2;
+    const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int r = (warp & 3) * 32 + lane;
+    const int c0 = (e >> 2) * 128;
+    float total[128];
+    uint32_t step = 0;
+    bool ok = true;
+    for (int tile = pair; tile < n_tiles && ok; tile += n_pairs) {
+      const TileCoord tc = tile_coord<2 * Cfg::kBM, BN>(tile, m_tiles, n_cols);
+      const int row = tc.m0 + static_cast<int>(rank) * Cfg::kBM + r;
+      for (int sj = 0; sj < seg.n_seg && ok; ++sj, ++step) {
+        const uint32_t buf = step & 1;
+        ok = __all_sync(0xffffffffu, wait(acc_full + 8 * buf, (step >> 1) & 1));
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll
+        for (int cb = 0; cb < 128; cb += 32) {
+          uint32_t v[32];
+          tmem_ld32(tmem + lane_sel + buf * BN + c0 + cb, v);
+          tmem_wait_ld();
+          if (cb + 32 == 128) {  // the accumulator is in registers: hand it back to the issuer
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty + 8 * buf, 0));
+          }
+          if (sj == 0) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) total[cb + i] = __uint_as_float(v[i]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) total[cb + i] = __fadd_rn(total[cb + i], __uint_as_float(v[i]));
+          }
+        }
+        if (sj == seg.n_seg - 1 && row < M) {
+          __nv_bfloat16* dst = y + static_cast<size_t>(row) * N + tc.n0 + c0;
+#pragma unroll
+          for (int i = 0; i < 128; i += 8) {
+            uint32_t o[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __nv_bfloat162 t2 = __floats2bfloat162_rn(total[i + 2 * q], total[i + 2 * q + 1]);
+              o[q] = *reinterpret_cast<uint32_t*>(&t2);
+            }
+            *reinterpret_cast<uint4*>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+          }
+        }
+      }
+    }
+  }
+
+  // Neither CTA leaves while the other may still send to its barriers or read its shared memory.
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
+}
+
 // The second half of the split schedule: y = bf16(((s_0 + s_1) + s_2) + ...), eight columns per thread.
 __global__ void __launch_bounds__(256) linear_fold_kernel(const float* __restrict__ seg_ws,
                                                           __nv_bfloat16* __restrict__ y, int M, int N, int bn,
@@ -403,6 +639,26 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
                      workspace_bytes >= split_workspace_bytes(M, N, K, BN) &&
                      reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
   __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(y);
+  if constexpr (BN == 256) {
+    // Scheduling only: with more than one row tile and enough 256 x 256 tiles for every pair of
+    // SMs, CTA pairs compute them (less operand traffic per SM, deeper pipeline).
+    const int n_pairs = sm_count / 2;
+    const int64_t pair_tiles = ((M + 2 * PairCfg::kBM - 1) / (2 * PairCfg::kBM)) * (N / BN);
+    if (!split && n_pairs > 0 && M > PairCfg::kBM && pair_tiles >= int64_t{n_pairs}) {
+      static bool pair_attr_set[64] = {};
+      if (!pair_attr_set[dev]) {
+        if (cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 PairCfg::kSmemBytes) != cudaSuccess)
+          return VOSTI_ERR_CUDA;
+        pair_attr_set[dev] = true;
+      }
+      alignas(64) CUtensorMap w_half_map;  // this CTA's 128 of the tile's 256 weight rows
+      if (!make_map(fn, &w_half_map, w, N, K, BN / 2)) return VOSTI_ERR_CUDA;
+      linear_pair_kernel<<<2 * n_pairs, PairCfg::kThreads, PairCfg::kSmemBytes, stream>>>(
+          x_map, w_half_map, yb, static_cast<int>(M), static_cast<int>(N), static_cast<int>(K));
+      return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+    }
+  }
   if (!split) {
     const int grid = static_cast<int>(tiles < sm_count ? tiles : sm_count);
     linear_kernel<BN, false><<<grid, Cfg::kThreads, Cfg::kSmemBytes, stream>>>(

@@ -126,3 +126,28 @@ def test_argument_checks():
                             torch.zeros(N, K, dtype=torch.bfloat16, device="cuda"))
         assert e.value.status == vb.VOSTI_ERR_UNSUPPORTED_CONFIG
     assert vl.vosti_linear(x[:0].contiguous(), torch.zeros(128, 64, dtype=torch.bfloat16, device="cuda")).shape == (0, 128)
+
+
+@pytest.mark.parametrize("N,K,M", [(4096, 1024, 4096), (4096, 4096, 3900), (6144, 2048, 2500)])
+def test_cta_pair_kernel_gives_the_bits_of_the_single_cta_kernel(N, K, M):
+    """Large problems run on CTA pairs (tcgen05.mma cta_group::2, 256 x 256 tiles); small ones on
+    single CTAs.  The choice depends on M, so the bits must not: every row of the large call
+    equals the same row computed in a call of 128 rows.  Ragged M: the last pair of the second
+    shape has 60 rows, so its second CTA owns no row at all."""
+    from oracle import linear_oracle as lo
+    from paper_2609_38981_b200 import linear as vl
+    from paper_2609_38981_b200.harness import bf16_bits
+    x, w = data(N, K, M, 13)
+    xd, wd = x.cuda(), w.cuda()
+    y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    vl.vosti_linear(xd, wd, y)
+    assert vl.vosti_linear_poll_status() == 0
+    big = bf16_bits(y)
+    for r0 in list(range(0, M, 1024)) + [M - 128]:
+        part = bf16_bits(vl.vosti_linear(xd[r0:r0 + 128].contiguous(), wd))
+        assert torch.equal(big[r0:r0 + 128], part), f"rows {r0}..{r0 + 127} differ between the two kernels"
+    rows = [0, 127, 128, 255, 256, M - 1]
+    ref = lo.linear(inputs.bits(x[rows]), inputs.bits(w))
+    mag = np.abs(widen(x[rows])) @ np.abs(widen(w)).T
+    err = np.abs(widen(y[rows]) - ref)
+    assert (err <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -20 * mag).all(), float(err.max())
