@@ -10,11 +10,14 @@
  * (N, K) only, every segment sum starts from a zero fp32 accumulator and takes
  * its products in ascending order (chunks of 16, tcgen05.mma), and the segment
  * sums are added left to right in fp32; and a row of an MMA tile depends on its
- * own operand row only.  Whether one CTA walks all segments of a tile (large
- * batches) or the segments of a tile are spread over CTAs and added by a second
- * kernel (small batches, so that every SM streams a slice of the weight) is a
- * scheduling decision that may depend on M: both compute the same sums in the
- * same order.
+ * own operand row only.  Whether a pair of CTAs computes 256 x 256 tiles with
+ * two-SM MMA instructions (large batches), one CTA walks all segments of a
+ * 128-row tile, or the segments of a tile are spread over CTAs and added by a
+ * second kernel (one row tile, so that every SM streams a slice of the weight)
+ * is a scheduling decision that may depend on M: all compute the same sums in
+ * the same order.  The tile shape reported by vosti_linear_tile_shape is the
+ * unit of that arithmetic (one CTA's rows, one instruction's columns and K
+ * block); a pair kernel works on two such row tiles at a time.
  *
  * All tensors are bf16, row-major, in device memory, 16-byte aligned; fp32
  * accumulation; round-to-nearest-even to bf16 at the end.  Kernels are
