@@ -34,9 +34,9 @@ struct Segments {
   int n_seg, k_blocks;
   __host__ __device__ int begin(int j) const { return static_cast<int>(static_cast<int64_t>(j) * k_blocks / n_seg); }
 };
-__host__ __device__ inline Segments segments_of(int64_t N, int64_t K, int bn) {
+__host__ __device__ inline Segments segments_of(int64_t N, int64_t K) {
   const int k_blocks = static_cast<int>(K / 64);
-  const int64_t col_tiles = N / bn;
+  const int64_t col_tiles = N % 256 == 0 ? N / 256 : N / 128;  // columns of the widest instruction that divides N
   // as many (column tile, segment) units as fit one wave over the 148 SMs of a B200 when the batch
   // is a single row tile, but segments of at least 1024 elements: every segment costs the
   // large-batch schedule a pass over the accumulator
@@ -92,7 +92,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
   const int m_tiles = (M + Cfg::kBM - 1) / Cfg::kBM;
   const int n_cols = N / BN;
   const int n_tiles = m_tiles * n_cols;
-  const Segments seg = segments_of(N, K, BN);
+  const Segments seg = segments_of(N, K);
   // A step is one segment of one tile; a CTA's steps are numbered consecutively.  Without the
   // split a CTA owns whole tiles (steps tile-major); with it, single (tile, segment) units.
   const int n_units = SPLIT ? n_tiles * seg.n_seg : n_tiles;
@@ -365,7 +365,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
   const int m_tiles = (M + 2 * Cfg::kBM - 1) / (2 * Cfg::kBM);
   const int n_cols = N / BN;
   const int n_tiles = m_tiles * n_cols;
-  const Segments seg = segments_of(N, K, BN);
+  const Segments seg = segments_of(N, K);
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) {
@@ -610,13 +610,14 @@ bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int64_t rows,
 }
 
 // Workspace the split schedule needs: one fp32 [M, N] slab per segment.
-size_t split_workspace_bytes(int64_t M, int64_t N, int64_t K, int bn) {
-  return sizeof(float) * static_cast<size_t>(segments_of(N, K, bn).n_seg) * M * N;
+size_t split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  return sizeof(float) * static_cast<size_t>(segments_of(N, K).n_seg) * M * N;
 }
 
 template <int BN>
 vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
-                           void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream) {
+                           void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream,
+                           bool use_pairs = false) {
   using Cfg = LinearCfg<BN>;
   static bool attr_set[64] = {};
   int dev = 0;
@@ -632,19 +633,17 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
   alignas(64) CUtensorMap x_map, w_map;
   if (!make_map(fn, &x_map, x, M, K, Cfg::kBM) || !make_map(fn, &w_map, w, N, K, BN)) return VOSTI_ERR_CUDA;
   const int64_t tiles = ((M + Cfg::kBM - 1) / Cfg::kBM) * (N / BN);
-  const Segments seg = segments_of(N, K, BN);
+  const Segments seg = segments_of(N, K);
   // Scheduling only: split the segments over CTAs when whole tiles would leave most SMs idle
   // and the caller has provided room for the segment sums.
   const bool split = seg.n_seg > 1 && tiles * 2 <= sm_count && workspace != nullptr &&
-                     workspace_bytes >= split_workspace_bytes(M, N, K, BN) &&
+                     workspace_bytes >= split_workspace_bytes(M, N, K) &&
                      reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
   __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(y);
   if constexpr (BN == 256) {
-    // Scheduling only: with more than one row tile and enough 256 x 256 tiles for every pair of
-    // SMs, CTA pairs compute them (less operand traffic per SM, deeper pipeline).
+    // CTA pairs (less operand traffic per SM, deeper pipeline) when the caller's estimate favours them.
     const int n_pairs = sm_count / 2;
-    const int64_t pair_tiles = ((M + 2 * PairCfg::kBM - 1) / (2 * PairCfg::kBM)) * (N / BN);
-    if (!split && n_pairs > 0 && M > PairCfg::kBM && pair_tiles >= int64_t{n_pairs}) {
+    if (!split && n_pairs > 0 && use_pairs) {
       static bool pair_attr_set[64] = {};
       if (!pair_attr_set[dev]) {
         if (cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -707,14 +706,14 @@ vosti_status vosti_linear_segments(int64_t N, int64_t K, int32_t* n_segments) {
   int32_t bn = 0;
   const vosti_status shape = vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr);
   if (shape != VOSTI_OK) return shape;
-  if (n_segments) *n_segments = segments_of(N, K, bn).n_seg;
+  if (n_segments) *n_segments = segments_of(N, K).n_seg;
   return VOSTI_OK;
 }
 
 size_t vosti_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   int32_t bn = 0;
   if (M <= 0 || vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr) != VOSTI_OK) return 0;
-  return split_workspace_bytes(M, N, K, bn);
+  return split_workspace_bytes(M, N, K);
 }
 
 vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* workspace,
@@ -741,8 +740,17 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
       cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  return bn == 256 ? launch_linear<256>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream)
-                   : launch_linear<128>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream);
+  if (bn != 256) return launch_linear<128>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream);
+  // Scheduling only (the bits are the same either way): CTA pairs when there is more than one
+  // row tile, the pairs have at least three rounds of 256 x 256 tiles (below that a round of
+  // single CTAs is measured to be as fast or faster), and their rounds, a little cheaper each,
+  // do not take longer than the single CTAs' rounds of 128 x 256 tiles.
+  const int64_t m128 = (M + 127) / 128, m256 = (M + 255) / 256;
+  auto rounds = [](int64_t tiles, int64_t slots) { return (tiles + slots - 1) / slots; };
+  const int64_t r_single = rounds(m128 * (N / 256), sm_count);
+  const int64_t r_pair = sm_count >= 2 ? rounds(m256 * (N / 256), sm_count / 2) : 0;
+  const bool use_pairs = M > 128 && r_pair >= 3 && 0.93 * static_cast<double>(r_pair) <= static_cast<double>(r_single);
+  return launch_linear<256>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream, use_pairs);
 }
 
 vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,
