@@ -54,6 +54,11 @@ def parse_args():
     ap.add_argument("--pack-shared-splits", action="store_true",
                     help="create the context with VOSTI_FLAG_PACK_SHARED_SPLITS (same bits, fewer tiles "
                          "when requests share prefix pages)")
+    ap.add_argument("--pack-through-tiles", action="store_true",
+                    help="with --pack-shared-splits: VOSTI_FLAG_PACK_THROUGH_TILES (large sharing groups always "
+                         "go through the tile kernel)")
+    ap.add_argument("--shared-prefix", type=int, default=0,
+                    help="prefix_sharing workload: length of the common prefix (experiments; default 2048)")
     ap.add_argument("--device-plan", action="store_true",
                     help="time the step as a CUDA-graph replay of vosti_plan_device + vosti_kv_append_planned + "
                          "vosti_paged_attention_planned (metadata in device memory); same bits")
@@ -65,7 +70,7 @@ def parse_args():
     return ap.parse_args()
 
 
-def make_workload(name: str, rank: int, pool_pages: int = 0, batch: int = 0):
+def make_workload(name: str, rank: int, pool_pages: int = 0, batch: int = 0, shared_prefix: int = 0):
     from paper_2609_38981_b200 import inputs
     fn = getattr(inputs, name)
     base = {"decode_heavy": 2, "mixed_chunked_prefill": 3, "prefix_sharing": 4,
@@ -73,6 +78,8 @@ def make_workload(name: str, rank: int, pool_pages: int = 0, batch: int = 0):
     kw = {"num_pages": pool_pages} if pool_pages else {}
     if batch:
         kw["batch"] = batch
+    if shared_prefix:
+        kw["prefix"] = shared_prefix
     return fn(seed=inputs.BASE_SEED * 10 + base + 1000 * rank, **kw)
 
 
@@ -291,13 +298,14 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = make_workload(args.workload, rank, args.pool_pages, args.batch)
+    w = make_workload(args.workload, rank, args.pool_pages, args.batch, args.shared_prefix)
     geo = w.geo
     scale = geo.head_dim ** -0.5
     max_seq = max(w.seq_lens)
     cache = DeviceCache(geo, w.num_pages, max_batch=w.batch, max_total_q=max(8192, w.total_q),
                         max_seq_len=max_seq, device=f"cuda:{local}",
-                        flags=vb.VOSTI_FLAG_PACK_SHARED_SPLITS if args.pack_shared_splits else 0)
+                        flags=(vb.VOSTI_FLAG_PACK_SHARED_SPLITS if args.pack_shared_splits else 0) |
+                        (vb.VOSTI_FLAG_PACK_THROUGH_TILES if args.pack_through_tiles else 0))
     cache.upload(w.requests, w.tables, upto=w.start_pos)      # cached context before the step
     bt = inputs.block_table_array(w.tables)
     ql, st, sl = (np.asarray(x, dtype=np.int32) for x in (w.q_lens, w.start_pos, w.seq_lens))
@@ -506,6 +514,8 @@ def main():
                           "K steps with a CUDA event pair around each launch of the dominant kernel",
                 "ms_per_step_with_kernel_events": roof_ms / args.steps,
                 "pack_shared_splits": bool(args.pack_shared_splits),
+                "pack_through_tiles": bool(args.pack_through_tiles),
+                "shared_prefix": int(args.shared_prefix) or None,
                 "device_plan": bool(args.device_plan),
                 "window": int(args.window),
                 "schedule": dict(zip(("split_items", "packed_items", "tile_items"),

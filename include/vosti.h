@@ -70,8 +70,15 @@ enum {
    * receives its own partial (m, z, U) for that split, computed from the same
    * keys in the same order, and the fold is unchanged, so outputs are bitwise
    * those of the unpacked schedule (tested by comparing the two).  Applies when
-   * window == 0. */
-  VOSTI_FLAG_PACK_SHARED_SPLITS = 2
+   * window == 0.  When the groups of 48 rows or more hold at least 4096 rows x
+   * splits between them, those groups are packed 128 rows to a tile of the
+   * tensor-memory kernel instead (one more kernel launch per call, an eighth
+   * of the reads of the shared pages); same partials, same bits. */
+  VOSTI_FLAG_PACK_SHARED_SPLITS = 2,
+  /* With PACK_SHARED_SPLITS: groups of 48 rows or more always go through the
+   * tensor-memory kernel, however little they hold (tests; callers that know
+   * their steps are bound by the GPU and not by the host). */
+  VOSTI_FLAG_PACK_THROUGH_TILES = 4
 };
 
 /* The fixed deployment configuration (Sec. "Fixed kernel choices": tile
@@ -377,9 +384,11 @@ vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* 
 int64_t vosti_launch_count(const vosti_ctx* ctx);
 
 /* The schedule of the last attention call of this context: split-parallel work
- * items (packed ones included), how many of them are packed items (shared-split
- * packing, VOSTI_FLAG_PACK_SHARED_SPLITS), and 256-row tile items.  Any pointer
- * may be NULL.  Host-side bookkeeping only. */
+ * items (16-row packed ones included), how many of them are packed items
+ * (shared-split packing, VOSTI_FLAG_PACK_SHARED_SPLITS), and tile items: the
+ * 256-row items of long queries plus the 128-row packed tiles that large
+ * sharing groups are routed to.  Any pointer may be NULL.  Host-side
+ * bookkeeping only. */
 vosti_status vosti_last_schedule(const vosti_ctx* ctx, int64_t* split_items, int64_t* packed_items,
                                  int64_t* tile_items);
 

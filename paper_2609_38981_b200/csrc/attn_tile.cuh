@@ -77,7 +77,14 @@ __device__ __forceinline__ void reg_alloc() { asm volatile("setmaxnreg.inc.sync.
 template <int N>
 __device__ __forceinline__ void reg_dealloc() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
-template <int D>
+// PACKED = false: a CTA is one 128-row half of a 256-row item of one request; it walks the key
+// tiles its rows see, folds split by split and writes the output rows.
+// PACKED = true (shared-split packing): a CTA is up to 128 rows of *different* requests that name
+// the same pages for one complete split; every row sees every key of the split; the CTA walks
+// that split's eight tiles and writes each row's partial (m, z, U) where the split-parallel
+// kernel would have written it, for combine_kernel to fold.  Same tiles, same scalar rules,
+// same accumulation order per row: the partial is bit for bit the one a 16-row item produces.
+template <int D, bool PACKED = false>
 __global__ void __launch_bounds__(TileKernelCfg<D>::kThreads, 2)
 attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {
   using Cfg = TileKernelCfg<D>;
@@ -87,22 +94,40 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   constexpr int TR = Cfg::kTileRows;
   constexpr uint32_t kAbortAfterNs = 1000000000u;
 
-  // CTA -> (work item, KV head, half of the item)
-  const vosti_work_item item = P.items[(blockIdx.x >> 1) / P.Hkv];
-  const int kvh = (blockIdx.x >> 1) % P.Hkv;
-  const ReqMeta rq = P.reqs[item.req];
+  // CTA -> (work item, KV head, half of the item); packed: CTA -> (packed tile, KV head)
   const int G = P.G;
-  const int row0 = item.row_group * nc::kRowsPerGroup + (blockIdx.x & 1) * TR;  // first row of this CTA's tile
-  const int rows = rq.q_len * G;
-  if (row0 >= rows) return;  // the item's second half does not exist
-  const int n_eff = rq.start + rq.q_len;
-  const int n_tiles = (rq.start + min(rq.q_len - 1, (row0 + TR - 1) / G)) / KT + 1;  // key tiles walked
-  // Under a sliding window nothing before the first visible key of the tile's first row is
-  // needed: the walk starts at key tile T0 (rows whose own window starts later take identity
-  // steps until it does).  Stages, S buffers and barrier phases are indexed by t - T0.
-  const int p_first = rq.start + row0 / G;
-  const int T0 = nc::first_key(p_first, P.window) / KT;
-  const int lo_first = nc::window_lo(p_first, P.window);  // keys up to here are invisible to every row
+  const int unit = PACKED ? blockIdx.x : (blockIdx.x >> 1);
+  const int kvh = unit % P.Hkv;
+  ReqMeta rq;
+  int row0, rows, n_eff, n_tiles, T0, lo_first;
+  const PackedRow* prow = nullptr;  // packed: the CTA's 128 row records
+  if constexpr (PACKED) {
+    const int4 ti = P.tile_pack_items[unit / P.Hkv];  // {first page id's index in the flat table, split, rows, -}
+    prow = P.tile_rows + static_cast<size_t>(unit / P.Hkv) * TR;
+    rq = ReqMeta{};
+    rq.bt_off = ti.x - ti.y * nc::kPagesPerSplit;       // so that page index arithmetic stays absolute
+    rq.n_pages = (ti.y + 1) * nc::kPagesPerSplit;
+    row0 = 0;
+    rows = ti.z;
+    n_eff = (ti.y + 1) * nc::kSplitLen;                 // a complete split: no tail
+    n_tiles = (ti.y + 1) * TPS;
+    T0 = ti.y * TPS;
+    lo_first = nc::window_lo(0, 0);
+  } else {
+    const vosti_work_item item = P.items[unit / P.Hkv];
+    rq = P.reqs[item.req];
+    row0 = item.row_group * nc::kRowsPerGroup + (blockIdx.x & 1) * TR;  // first row of this CTA's tile
+    rows = rq.q_len * G;
+    if (row0 >= rows) return;  // the item's second half does not exist
+    n_eff = rq.start + rq.q_len;
+    n_tiles = (rq.start + min(rq.q_len - 1, (row0 + TR - 1) / G)) / KT + 1;  // key tiles walked
+    // Under a sliding window nothing before the first visible key of the tile's first row is
+    // needed: the walk starts at key tile T0 (rows whose own window starts later take identity
+    // steps until it does).  Stages, S buffers and barrier phases are indexed by t - T0.
+    const int p_first = rq.start + row0 / G;
+    T0 = nc::first_key(p_first, P.window) / KT;
+    lo_first = nc::window_lo(p_first, P.window);  // keys up to here are invisible to every row
+  }
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -151,10 +176,16 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     griddep_wait();
     const int r = tid;
     const int row = row0 + r;
-    const bool valid = row < rows;
-    const int tok = row / G;
-    const uint4* src = reinterpret_cast<const uint4*>(
-        P.q + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D);
+    bool valid = row < rows;
+    size_t q_row;  // (packed token row) * Hq + query head
+    if constexpr (PACKED) {
+      const PackedRow pr = prow[r];
+      valid = pr.p >= 0;
+      q_row = static_cast<size_t>(pr.q_row_g & 0xFFFFFF) * P.Hq + kvh * G + (static_cast<uint32_t>(pr.q_row_g) >> 24);
+    } else {
+      q_row = static_cast<size_t>(rq.q_row0 + row / G) * P.Hq + kvh * G + row % G;
+    }
+    const uint4* src = reinterpret_cast<const uint4*>(P.q + q_row * D);
 #pragma unroll
     for (int c = 0; c < D / 8; ++c) {
       const uint4 v = valid ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
@@ -285,8 +316,8 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     reg_alloc<Cfg::kRegsSoftmax>();
     const int r = tid;                          // row of the tile = tensor-memory lane
     const int row = row0 + r;
-    const bool valid = row < rows;
-    const int p = valid ? rq.start + row / G : -1;  // padding rows see nothing
+    const bool valid = PACKED ? prow[r].p >= 0 : row < rows;
+    const int p = PACKED ? prow[r].p : (valid ? rq.start + row / G : -1);  // padding rows see nothing
     const int lo = nc::window_lo(p, P.window);      // key j is visible iff lo < j <= p
     const uint32_t lane_sel = static_cast<uint32_t>(warp * 32) << 16;
     const float c = P.c;
@@ -394,9 +425,9 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     reg_alloc<Cfg::kRegsCorrection>();
     const int r = tid & (TR - 1);
     const int row = row0 + r;
-    const bool valid = row < rows;
+    const bool valid = PACKED ? prow[r].p >= 0 : row < rows;
     const int tok = row / G;
-    const int p = valid ? rq.start + tok : -1;
+    const int p = PACKED ? prow[r].p : (valid ? rq.start + tok : -1);
     // first split the row sees; before it (and in the first split the CTA walks) the
     // running result is simply taken from the split, as the fold of the split kernels does
     const int k_first = max(nc::first_key(p, P.window) / nc::kSplitLen, T0 / TPS);
@@ -405,6 +436,12 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     // and the row's place in the output
     float4* ucg = reinterpret_cast<float4*>(P.ws_uc) + static_cast<size_t>(blockIdx.x) * (D / 4) * TR + r;
     __nv_bfloat16* dst = P.out + (static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G) * D;
+    // packed: the row's partial slab, where the split-parallel kernel would have put it
+    int64_t slab = 0;
+    if constexpr (PACKED) {
+      const PackedRow pr = prow[r];
+      slab = static_cast<int64_t>(pr.slab_row) + static_cast<int64_t>(kvh) * pr.kvh_stride;
+    }
     float mc = 0.f, zc = 0.f;
     bool ok = true;
     for (int t = T0; t < n_tiles && ok; ++t) {
@@ -467,7 +504,29 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       mbar_arrive(p_full + 8 * b);
 
       // ---- end of a split: fold it into the running result (kept in global memory) -------
-      if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
+      if constexpr (PACKED) {
+        if (t + 1 == n_tiles) {  // the split is complete: its raw (m, z, U) is the row's partial
+          ok = __all_sync(kFullMask, wait(mz_full, 0));
+          if (!ok) break;
+          const float2 mz = mz_s[r];
+          ok = __all_sync(kFullMask, wait(pv_done + 8 * b, (ti >> 1) & 1));
+          if (!ok) break;
+          tc_fence_after();
+          if (valid) P.ws_mz[slab] = mz;
+          float* pu = P.ws_u + slab * D;
+#pragma unroll 1
+          for (int cb = 0; cb < D; cb += 16) {
+            uint32_t ur[16];
+            tmem_ld16(tmem + lane_sel + Cfg::kColU + cb, ur);
+            tmem_wait_ld();
+            if (valid) {
+#pragma unroll
+              for (int i = 0; i < 16; i += 4)
+                *reinterpret_cast<uint4*>(pu + cb + i) = make_uint4(ur[i], ur[i + 1], ur[i + 2], ur[i + 3]);
+            }
+          }
+        }
+      } else if ((t + 1) % TPS == 0 || t + 1 == n_tiles) {
         const int split = t / TPS;
         const int kb = (split - T0 / TPS) & 1, kuse = (split - T0 / TPS) >> 1;
         const bool resume = split > T0 / TPS;  // the CTA has stored a running result before

@@ -70,6 +70,10 @@ struct AttnParams {
   // Device-planned calls: {n_workers, n_split_tokens} written by the planning kernel earlier in
   // the stream (the two fields above are then only upper bounds for the grids); nullptr otherwise.
   const int32_t* counts;
+  // Shared-split packing through the tile kernel: per packed tile {index of the split's first page id in
+  // the flat table, split, rows in use, 0} and 128 row records; nullptr when there are none.
+  const int4* tile_pack_items;
+  const PackedRow* tile_rows;
   int32_t num_pages;         // device-planned calls: page ids are checked against it when an item is drawn
 };
 

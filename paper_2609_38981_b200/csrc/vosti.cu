@@ -17,6 +17,9 @@ namespace vosti {
 namespace {
 
 constexpr int kHostSlots = 8;        // ring of pinned staging buffers
+constexpr int kPackedTileRows = 128;  // rows of a packed tile: one CTA of the tile kernel
+constexpr int64_t kTilePackMinRowSplits = 4096;  // rows x splits of such groups from which the extra launch pays
+constexpr int kTilePackMinRows = 48;  // rows sharing a split from which packing goes through the tile kernel
 constexpr int kHostSteps = 3;        // host-buffer steps that may be in flight (vosti_step_host_async)
 constexpr size_t kAlign = 1024;
 constexpr int kTileRows = 256;       // rows of one tile-kernel work item (16 row groups)
@@ -61,7 +64,13 @@ Limits limits_of(const vosti_config& c) {
   L.part_rows_max = std::min(rows_by_batch, rows_by_total) * c.n_kv_heads * L.k_max;
   // packed rows (shared-split packing only): 16 per packed item, and packing never adds items
   const int64_t packed_rows_max = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) ? 16 * items_split : 0;
+  // packed tiles: a group that takes this route has at least kTilePackMinRows rows, so a tile of
+  // kPackedTileRows records stands for at least kTilePackMinRows / 16 sixteen-row items
+  const int64_t packed_tiles_max =
+      (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) ? items_split / (kTilePackMinRows / 16) + 1 : 0;
   const size_t attn_blob = align_up(sizeof(PackedRow) * packed_rows_max, 16) +
+                           align_up(sizeof(PackedRow) * kPackedTileRows * packed_tiles_max, 16) +
+                           align_up(sizeof(int4) * packed_tiles_max, 16) +
                            align_up(sizeof(ReqMeta) * c.max_batch, 16) +
                            align_up(sizeof(SplitItem) * items_split, 16) +
                            align_up(sizeof(vosti_work_item) * items_seq, 16) +
@@ -266,6 +275,10 @@ struct vosti_ctx {
   std::vector<int64_t> pk_off;     // per request: first entry of its complete splits in pk_mark
   std::vector<uint8_t> pk_mark;    // 1: the (request, split) pair is served by packed items
   std::vector<int32_t> pk_table, pk_next, pk_head, pk_tail;  // grouping of the candidates by key
+  std::vector<PackedRow> pk_tile_rows;   // packed tiles (groups of many rows, run by the tile kernel): 128 rows each
+  std::vector<int64_t> pk_group_stats;   // per sharing group: members, rows together, 16-row tiles apart
+  std::vector<int4> pk_tile_items;       // per packed tile {index of the split's first page id, split, rows, 0}
+  int64_t last_packed_tiles = 0;
   int64_t last_split_items = 0, last_packed_items = 0, last_tile_items = 0;  // schedule of the last attention call
   // profiling of the dominant kernel
   int profile_mode = 0;
@@ -371,7 +384,8 @@ cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, size
 
 template <int D>
 vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_split, int64_t n_seq,
-                              cudaStream_t stream, bool run_partials = true, bool run_combine = true) {
+                              cudaStream_t stream, bool run_partials = true, bool run_combine = true,
+                              int64_t n_packed_tiles = 0) {
   using Cfg = SplitKernelCfg<D>;
   const int Hkv = ctx->cfg.n_kv_heads;
   const bool prof = ctx->profile_mode != 0;
@@ -410,6 +424,16 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
                        ctx->kv_map, p);
     });
   }
+  if (n_packed_tiles > 0 && run_partials) {
+    AttnParams p = base;
+    p.n_workers = static_cast<int32_t>(n_packed_tiles * Hkv);
+    using TileCfg_ = TileKernelCfg<D>;
+    timed(2, [&] {
+      // one CTA per packed tile (up to 128 rows that share a split) and KV head
+      launch_dependent(attn_tile_kernel<D, true>, p.n_workers, TileCfg_::kThreads, TileCfg_::kSmemBytes, stream,
+                       ctx->kv_map, p);
+    });
+  }
   if (base.n_split_tokens > 0 && run_combine) {
     const int warps = base.n_split_tokens * base.Hq;
     timed(3, [&] { launch_dependent(combine_kernel<D>, (warps + 3) / 4, 128, 0, stream, base); });
@@ -438,10 +462,17 @@ vosti_status set_kernel_attributes() {
       cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
                            cudaSharedmemCarveoutMaxShared) != cudaSuccess)
     return VOSTI_ERR_CUDA;
+  if (cudaFuncSetAttribute(attn_tile_kernel<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           TileKernelCfg<D>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_tile_kernel<D, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
   // The tile kernel moves registers between its warpgroups; a request for more than the CTA
   // was given at launch would block for ever, so refuse to run a build where that could happen.
   cudaFuncAttributes attr;
   if (cudaFuncGetAttributes(&attr, attn_tile_kernel<D>) != cudaSuccess) return VOSTI_ERR_CUDA;
+  if (attr.numRegs * TileKernelCfg<D>::kThreads < TileKernelCfg<D>::kRegsAfterSplit) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  if (cudaFuncGetAttributes(&attr, attn_tile_kernel<D, true>) != cudaSuccess) return VOSTI_ERR_CUDA;
   if (attr.numRegs * TileKernelCfg<D>::kThreads < TileKernelCfg<D>::kRegsAfterSplit) return VOSTI_ERR_UNSUPPORTED_CONFIG;
   return VOSTI_OK;
 }
@@ -711,6 +742,8 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
   int64_t n_split_final = 0, n_packed_items = 0;
   std::vector<PackCand>& cands = ctx->cands;
   cands.clear();
+  ctx->pk_tile_rows.clear();
+  ctx->pk_tile_items.clear();
   pk_off.assign(static_cast<size_t>(batch) + 1, 0);
   for (int r = 0; r < batch; ++r) {
     const ReqMeta& m = reqs[r];
@@ -759,22 +792,78 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
                        bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
                        sizeof(int32_t) * nc::kPagesPerSplit) == 0;
   };
+  // What each group amounts to.  Groups of kTilePackMinRows rows or more could go through the tile
+  // kernel; that costs one more launch per call, so it is done only when the rows x splits they
+  // hold add up to enough work (or the context asks for it always).
+  struct GroupStat {
+    int members;
+    int64_t rows_together, tiles_apart;
+  };
+  std::vector<int64_t>& stats = ctx->pk_group_stats;  // three numbers per group
+  stats.assign(3 * head.size(), 0);
+  int64_t tile_row_splits = 0;
   for (size_t g = 0; g < head.size(); ++g) {
     const int lo = head[g];
     if (next[lo] < 0) continue;  // alone
-    // members: the very same split and page ids as the first (a key collision stays unpacked)
-    // and packing must save tiles: fewer 16-row tiles together than one request at a time
-    int members = 0;
-    int64_t rows_together = 0, tiles_apart = 0;
+    GroupStat gs{0, 0, 0};
     for (int i = lo; i >= 0; i = next[i])
       if (same_pages(cands[i], cands[lo])) {
         const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
-        ++members;
-        rows_together += rows;
-        tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+        ++gs.members;
+        gs.rows_together += rows;
+        gs.tiles_apart += (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
       }
-    if (members < 2 || (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup >= tiles_apart) continue;
+    stats[3 * g] = gs.members;
+    stats[3 * g + 1] = gs.rows_together;
+    stats[3 * g + 2] = gs.tiles_apart;
+    if (gs.members >= 2 && gs.rows_together >= kTilePackMinRows) tile_row_splits += gs.rows_together;
+  }
+  const bool through_tiles =
+      (ctx->cfg.flags & VOSTI_FLAG_PACK_THROUGH_TILES) || tile_row_splits >= kTilePackMinRowSplits;
+  for (size_t g = 0; g < head.size(); ++g) {
+    const int lo = head[g];
+    if (next[lo] < 0) continue;  // alone
+    // members: the very same split and page ids as the first (a key collision stays unpacked);
+    // packing must save tiles: fewer 16-row tiles together than one request at a time, or
+    // enough rows for the 128-row tiles of the tile kernel
+    const int64_t members = stats[3 * g], rows_together = stats[3 * g + 1], tiles_apart = stats[3 * g + 2];
+    if (members < 2) continue;
+    const bool to_tiles = through_tiles && rows_together >= kTilePackMinRows;
+    if (!to_tiles && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup >= tiles_apart) continue;
     const ReqMeta& first = reqs[cands[lo].req];
+    if (to_tiles) {
+      // Many rows share the split: 128 to a tile of the tensor-memory kernel, which reads the
+      // split once per 128 rows instead of once per 16.
+      std::vector<PackedRow>& trows = ctx->pk_tile_rows;
+      const int split = cands[lo].split;
+      const int64_t n_tiles = (rows_together + kPackedTileRows - 1) / kPackedTileRows;
+      const size_t first_row = trows.size();
+      trows.resize(first_row + static_cast<size_t>(n_tiles) * kPackedTileRows);
+      for (size_t i = first_row + static_cast<size_t>(rows_together); i < trows.size(); ++i)
+        trows[i] = PackedRow{0, -1, 0, 0};  // padding rows of the last tile see nothing
+      for (int64_t t = 0; t < n_tiles; ++t)
+        ctx->pk_tile_items.push_back(make_int4(
+            first.bt_off + split * nc::kPagesPerSplit, split,
+            static_cast<int>(std::min<int64_t>(kPackedTileRows, rows_together - t * kPackedTileRows)), 0));
+      PackedRow* pr = trows.data() + first_row;  // real rows are contiguous; only the last tile has padding
+      for (int i = lo; i >= 0; i = next[i]) {
+        if (!same_pages(cands[i], cands[lo])) continue;
+        const ReqMeta& m = reqs[cands[i].req];
+        pk_mark[static_cast<size_t>(pk_off[cands[i].req] + split)] = 1;
+        const int rows = m.q_len * G;
+        const int32_t slab0 = static_cast<int32_t>(m.part_base + int64_t{split} * rows);
+        const int32_t stride = m.n_splits * rows;
+        int row = 0;
+        for (int tok = 0; tok < m.q_len; ++tok)
+          for (int g = 0; g < G; ++g, ++row, ++pr) {
+            pr->q_row_g = (m.q_row0 + tok) | (g << 24);
+            pr->p = m.start + tok;
+            pr->slab_row = slab0 + row;
+            pr->kvh_stride = stride;
+          }
+      }
+      continue;
+    }
     int in_item = 0;
     auto close_item = [&]() {
       PackedRow* rows16 = packed_rows + n_packed_items * 16;
@@ -795,14 +884,17 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
       const int k = cands[i].split;
       pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
       const int rows = m.q_len * G;
-      for (int row = 0; row < rows; ++row) {
-        PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
-        pr.q_row_g = (m.q_row0 + row / G) | ((row % G) << 24);
-        pr.p = m.start + row / G;
-        pr.slab_row = static_cast<int32_t>(m.part_base + int64_t{k} * rows + row);
-        pr.kvh_stride = m.n_splits * rows;
-        if (++in_item == 16) close_item();
-      }
+      const int32_t slab0 = static_cast<int32_t>(m.part_base + int64_t{k} * rows);
+      int row = 0;
+      for (int tok = 0; tok < m.q_len; ++tok)
+        for (int g = 0; g < G; ++g, ++row) {
+          PackedRow& pr = packed_rows[n_packed_items * 16 + in_item];
+          pr.q_row_g = (m.q_row0 + tok) | (g << 24);
+          pr.p = m.start + tok;
+          pr.slab_row = slab0 + row;
+          pr.kvh_stride = m.n_splits * rows;
+          if (++in_item == 16) close_item();
+        }
     }
     if (in_item > 0) close_item();
   }
@@ -904,8 +996,8 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
 
   // ---- shared-split packing (scheduling only): packed items first in the item list (they walk a
   // whole split: the longest kind), the others follow in plan order ---------------------------
-  int64_t n_split_final = 0, n_packed_items = 0;
-  size_t off_packed = 0;
+  int64_t n_split_final = 0, n_packed_items = 0, n_packed_tiles = 0;
+  size_t off_packed = 0, off_tile_rows = 0, off_tile_items = 0;
   std::vector<int64_t>& pk_off = ctx->pk_off;
   std::vector<uint8_t>& pk_mark = ctx->pk_mark;
   const bool packing = (c.flags & VOSTI_FLAG_PACK_SHARED_SPLITS) && window == 0 && cp.phase == 0 && plan.n_split > 1 &&
@@ -916,11 +1008,18 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
                                         split_items);
     n_split_final = n_packed_items;
     at += align_up(sizeof(PackedRow) * 16 * n_packed_items, 16);
+    n_packed_tiles = static_cast<int64_t>(ctx->pk_tile_items.size());
+    off_tile_rows = at;
+    std::memcpy(blob + at, ctx->pk_tile_rows.data(), sizeof(PackedRow) * ctx->pk_tile_rows.size());
+    at += align_up(sizeof(PackedRow) * ctx->pk_tile_rows.size(), 16);
+    off_tile_items = at;
+    std::memcpy(blob + at, ctx->pk_tile_items.data(), sizeof(int4) * ctx->pk_tile_items.size());
+    at += align_up(sizeof(int4) * ctx->pk_tile_items.size(), 16);
   }
   for (int64_t i = 0; i < plan.n_split; ++i) {
     const vosti_work_item& it = plan.items[i];
     const ReqMeta& m = reqs[it.req];
-    if (n_packed_items > 0 && int64_t{it.split_begin} < pk_off[it.req + 1] - pk_off[it.req] &&
+    if ((n_packed_items > 0 || n_packed_tiles > 0) && int64_t{it.split_begin} < pk_off[it.req + 1] - pk_off[it.req] &&
         pk_mark[static_cast<size_t>(pk_off[it.req] + it.split_begin)])
       continue;  // served by packed items
     if (cp.phase == 2 || (cp.phase == 1 && it.split_begin % cp.world != cp.rank)) continue;  // not this rank's split
@@ -977,9 +1076,12 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
   p.lse = lse;
   p.counts = nullptr;
   p.num_pages = 0;
+  p.tile_pack_items = n_packed_tiles > 0 ? reinterpret_cast<const int4*>(dmeta + off_tile_items) : nullptr;
+  p.tile_rows = n_packed_tiles > 0 ? reinterpret_cast<const PackedRow*>(dmeta + off_tile_rows) : nullptr;
+  ctx->last_packed_tiles = n_packed_tiles;
   ctx->last_split_items = n_split_final;
   ctx->last_packed_items = n_packed_items;
-  ctx->last_tile_items = n_seq;
+  ctx->last_tile_items = n_seq + n_packed_tiles;
   if (cp.phase == 1) {
     // Slabs of splits other ranks own stay zero, so that a sum over ranks assembles all partials.
     if (cudaMemsetAsync(p.ws_u, 0, sizeof(float) * static_cast<size_t>(plan.n_partial_rows) * c.head_dim, stream) !=
@@ -988,8 +1090,8 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
       return VOSTI_ERR_CUDA;
   }
   st = c.head_dim == 128
-           ? launch_attention<128>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1)
-           : launch_attention<64>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1);
+           ? launch_attention<128>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1, n_packed_tiles)
+           : launch_attention<64>(ctx, p, n_split_final, n_seq, stream, cp.phase != 2, cp.phase != 1, n_packed_tiles);
   if (st != VOSTI_OK) return st;
   return release_slot(slot, stream);
 }

@@ -237,6 +237,8 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
   p.lse = nullptr;
   p.counts = nullptr;
   p.num_pages = 0;
+  p.tile_pack_items = nullptr;
+  p.tile_rows = nullptr;
   p.packed_rows = nullptr;
   return head_dim == 128 ? launch<128>(map, p, sm_count, stream) : launch<64>(map, p, sm_count, stream);
 }

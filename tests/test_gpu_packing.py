@@ -1,8 +1,9 @@
 """Shared-prefix row packing (VOSTI_FLAG_PACK_SHARED_SPLITS): rows of different
 requests that name the same physical pages for a whole 512-key split are packed
-16 to an MMA tile.  It is a scheduling decision: outputs (and the log-sum-exp)
-must be bit for bit those of the unpacked schedule, whatever mix of requests
-shares which prefix, and packing must really have happened."""
+16 to an MMA tile of the split-parallel kernel, or -- from 48 rows on -- 128 to
+a tile of the tensor-memory kernel.  It is a scheduling decision: outputs (and
+the log-sum-exp) must be bit for bit those of the unpacked schedule, whatever
+mix of requests shares which prefix, and packing must really have happened."""
 import numpy as np
 import pytest
 import torch
@@ -18,6 +19,8 @@ GEOS = {
     "d128_g8": inputs.Geometry(8, 1, 128, 16),
 }
 NUM_PAGES = 2048
+# packing, with groups of 48 rows or more always routed through the tile kernel
+TILES = vb.VOSTI_FLAG_PACK_SHARED_SPLITS | vb.VOSTI_FLAG_PACK_THROUGH_TILES
 
 
 def family(geo, seed, prefix, suffixes, first_index):
@@ -62,7 +65,7 @@ def build(geo, seed=99):
 def run(geo, reqs, tables, flags, calls, want_lse=True):
     """Upload everything, then run `calls` (lists of (request, start, q_len)) with attend only."""
     from paper_2609_38981_b200.harness import DeviceCache, bf16_bits
-    cache = DeviceCache(geo, NUM_PAGES, max_batch=32, max_total_q=4096, max_seq_len=4096, flags=flags)
+    cache = DeviceCache(geo, NUM_PAGES, max_batch=128, max_total_q=4096, max_seq_len=4096, flags=flags)
     # shared pages are written once per family member with identical content: harmless
     cache.upload(reqs, tables)
     scale = geo.head_dim ** -0.5
@@ -100,15 +103,13 @@ def test_packed_schedule_gives_the_same_bits(env, q_len):
         pytest.skip("not a split-parallel request in this geometry")
     calls = decode_calls(reqs, q_len)
     plain, plain_lse, sched0 = run(geo, reqs, tables, 0, calls)
-    packed, packed_lse, sched1 = run(geo, reqs, tables, vb.VOSTI_FLAG_PACK_SHARED_SPLITS, calls)
+    packed, packed_lse, sched1 = run(geo, reqs, tables, TILES, calls)
     for c in range(len(calls)):
         gu.assert_same_bits(packed[c], plain[c], f"call {c}")
         gu.assert_same_bits(packed_lse[c], plain_lse[c], f"call {c}, log-sum-exp")
         assert sched0[c][1] == 0
-        if (q_len * geo.group) % 16 == 0:   # every request fills its tiles: nothing to gain, nothing packed
-            assert sched1[c] == sched0[c]
-        else:
-            assert sched1[c][1] > 0 and sched1[c][0] < sched0[c][0], (sched0[c], sched1[c])
+        # packed 16 to a tile of the split-parallel kernel, or (48 rows and more) 128 to a packed tile
+        assert (sched1[c][1] > 0 or sched1[c][2] > 0) and sched1[c][0] < sched0[c][0], (sched0[c], sched1[c])
     # and both agree with the oracle
     from oracle import oracle
     scale = geo.head_dim ** -0.5
@@ -125,10 +126,19 @@ def test_expected_number_of_packed_items(env):
     brings G rows, so a family's split needs ceil(members * G / 16) packed items."""
     geo, reqs, tables = env["geo"], env["reqs"], env["tables"]
     calls = [[(i, r.n - 1, 1) for i, r in enumerate(reqs)]]
-    _, _, sched = run(geo, reqs, tables, vb.VOSTI_FLAG_PACK_SHARED_SPLITS, calls)
+    _, _, sched = run(geo, reqs, tables, TILES, calls)
     G = geo.group
-    expect = 2 * -(-6 * G // 16) + 4 * -(-5 * G // 16)
-    assert sched[0][1] == expect, (sched[0], expect)
+    small = tiles = 0
+    for members, splits in ((6, 2), (5, 4)):
+        rows = members * G
+        if rows >= 48:                      # a large group: 128 rows to a packed tile of the tile kernel
+            tiles += splits * -(-rows // 128)
+        else:
+            small += splits * -(-rows // 16)
+    assert sched[0][1] == small and sched[0][2] == tiles, (sched[0], small, tiles)
+    # without the flag that forces them, so few shared rows never pay for the tile kernel's launch
+    _, _, sched = run(geo, reqs, tables, vb.VOSTI_FLAG_PACK_SHARED_SPLITS, calls)
+    assert sched[0][2] == 0 and sched[0][1] == 2 * -(-6 * G // 16) + 4 * -(-5 * G // 16), sched[0]
 
 
 def test_a_lone_request_and_a_windowed_call_are_not_packed(env):
@@ -150,13 +160,13 @@ def test_a_lone_request_and_a_windowed_call_are_not_packed(env):
 
 def test_prefix_sharing_workload_full_size():
     """The benchmark's prefix-sharing batch (128 requests, 2048-token common prefix):
-    packed and unpacked schedules give the same bits; 4 requests share each packed tile."""
+    the unpacked schedule and both packed ones give the same bits."""
     from paper_2609_38981_b200.harness import DeviceCache, bf16_bits
     import gpu_util as gu
     w = inputs.prefix_sharing()
     geo = w.geo
     outs, sched = [], []
-    for flags in (0, vb.VOSTI_FLAG_PACK_SHARED_SPLITS):
+    for flags in (0, vb.VOSTI_FLAG_PACK_SHARED_SPLITS, TILES):
         cache = DeviceCache(geo, w.num_pages, max_batch=w.batch, max_total_q=4096,
                             max_seq_len=max(w.seq_lens) + 16, flags=flags)
         cache.upload(w.requests[:1], w.tables[:1], upto=[2048])
@@ -167,6 +177,44 @@ def test_prefix_sharing_workload_full_size():
         outs.append(bf16_bits(out))
         sched.append(vb.vosti_last_schedule(cache.ctx))
         cache.close()
-    assert torch.equal(outs[0], outs[1])
-    assert sched[1][1] == 4 * (128 * geo.group // 16), sched
-    gu.sampled_parity(w, outs[1], 64)
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+    # 512 rows share each of the 4 prefix splits: 2048 rows x splits, below the amount from which the
+    # tile kernel's launch pays, so 4 requests share each 16-row packed item ...
+    assert sched[1][1] == 4 * (128 * geo.group // 16) and sched[1][2] == 0, sched
+    # ... and, when forced, 4 packed tiles of 128 rows per split
+    assert sched[2][1] == 0 and sched[2][2] == 4 * (128 * geo.group // 128), sched
+    gu.sampled_parity(w, outs[2], 64)
+
+
+@pytest.mark.parametrize("members,q_len", [(40, 1), (23, 2), (70, 1)])
+def test_large_groups_go_through_packed_tiles(env, members, q_len):
+    """Dozens of requests on one 1100-token prefix (2 complete splits): their rows fill packed
+    tiles of 128 (the last one ragged), computed by the tensor-memory kernel in its
+    partial-output mode; bits and log-sum-exp equal the unpacked schedule's."""
+    import gpu_util as gu
+    geo = env["geo"]
+    if q_len * geo.group > 32:
+        pytest.skip("not a split-parallel request in this geometry")
+    rng = np.random.default_rng(members)
+    suffixes = [int(x) for x in rng.integers(q_len, 400, size=members)]
+    reqs = family(geo, 7, 1100, suffixes, 0)
+    P = geo.page_size
+    gen = inputs.generator(members)
+    need = [inputs.pages_needed(r.n, P) for r in reqs]
+    ids = inputs.draw_pages(gen, NUM_PAGES, 1100 // P + sum(c - 1100 // P for c in need))
+    shared, at, tables = ids[:1100 // P], 1100 // P, []
+    for c in need:
+        tables.append(shared + ids[at:at + c - 1100 // P])
+        at += c - 1100 // P
+    last = [(i, r.n - q_len, q_len) for i, r in enumerate(reqs)]
+    calls = [last, last[::-1], last[: members // 2]]
+    plain, plain_lse, sched0 = run(geo, reqs, tables, 0, calls)
+    packed, packed_lse, sched1 = run(geo, reqs, tables, TILES, calls)
+    for c, call in enumerate(calls):
+        gu.assert_same_bits(packed[c], plain[c], f"call {c}")
+        gu.assert_same_bits(packed_lse[c], plain_lse[c], f"call {c}, log-sum-exp")
+        rows = len(call) * q_len * geo.group
+        if rows >= 48:
+            assert sched1[c][2] == 2 * -(-rows // 128) and sched1[c][1] == 0, (sched1[c], rows)
+        else:
+            assert sched1[c][1] == 2 * -(-rows // 16) and sched1[c][2] == 0, (sched1[c], rows)
