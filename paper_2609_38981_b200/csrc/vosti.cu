@@ -276,6 +276,8 @@ struct vosti_ctx {
   std::vector<uint8_t> pk_mark;    // 1: the (request, split) pair is served by packed items
   std::vector<int32_t> pk_table, pk_next, pk_head, pk_tail;  // grouping of the candidates by key
   std::vector<PackedRow> pk_tile_rows;   // packed tiles (groups of many rows, run by the tile kernel): 128 rows each
+  std::vector<uint8_t> pk_member;        // per candidate: same page ids as the first of its group
+  std::vector<uint8_t> pk_keep;          // per request: some group is served from its page ids
   std::vector<int64_t> pk_group_stats;   // per sharing group: members, rows together, 16-row tiles apart
   std::vector<int4> pk_tile_items;       // per packed tile {index of the split's first page id, split, rows, 0}
   int64_t last_packed_tiles = 0;
@@ -735,8 +737,13 @@ namespace {
 // saves tiles.  Writes the packed rows at `packed_rows`, one SplitItem per packed item at the
 // front of `split_items`, marks the (request, split) pairs it has taken over in ctx->pk_mark,
 // and returns the number of packed items.
-int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, int G, const int32_t* bt_flat,
-                           PackedRow* packed_rows, SplitItem* split_items) {
+int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, int G, const int32_t* block_tables,
+                           int32_t block_table_stride, PackedRow* packed_rows, SplitItem* split_items) {
+  // page ids of split k of request r, in the caller's table (not validated here: a group is served
+  // from its first member's ids, which are validated when they are copied)
+  auto ids_of = [&](int r, int64_t k) {
+    return block_tables + static_cast<size_t>(r) * block_table_stride + k * nc::kPagesPerSplit;
+  };
   std::vector<int64_t>& pk_off = ctx->pk_off;
   std::vector<uint8_t>& pk_mark = ctx->pk_mark;
   int64_t n_split_final = 0, n_packed_items = 0;
@@ -751,7 +758,7 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
         (m.q_len > 0 && int64_t{m.q_len} * G <= nc::kSplitRowsMax) ? m.start / nc::kSplitLen : 0;
     pk_off[r + 1] = pk_off[r] + complete;
     for (int64_t k = 0; k < complete; ++k) {
-      const int32_t* ids = bt_flat + m.bt_off + k * nc::kPagesPerSplit;
+      const int32_t* ids = ids_of(r, k);
       // Grouping key: the split index with its first and last page id.  Two requests that share
       // the whole split agree on it; agreement on all 32 ids is checked when groups are formed.
       const uint64_t key = ((static_cast<uint64_t>(static_cast<uint32_t>(ids[0])) << 32) |
@@ -788,10 +795,11 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
   }
   auto same_pages = [&](const PackCand& a, const PackCand& b) {
     return a.split == b.split &&
-           std::memcmp(bt_flat + reqs[a.req].bt_off + int64_t{a.split} * nc::kPagesPerSplit,
-                       bt_flat + reqs[b.req].bt_off + int64_t{b.split} * nc::kPagesPerSplit,
-                       sizeof(int32_t) * nc::kPagesPerSplit) == 0;
+           std::memcmp(ids_of(a.req, a.split), ids_of(b.req, b.split), sizeof(int32_t) * nc::kPagesPerSplit) == 0;
   };
+  std::vector<uint8_t>& member = ctx->pk_member;  // per candidate: it has the page ids of its group's first one
+  member.assign(static_cast<size_t>(n), 0);
+  ctx->pk_keep.assign(static_cast<size_t>(batch), 0);
   // What each group amounts to.  Groups of kTilePackMinRows rows or more could go through the tile
   // kernel; that costs one more launch per call, so it is done only when the rows x splits they
   // hold add up to enough work (or the context asks for it always).
@@ -807,7 +815,8 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
     if (next[lo] < 0) continue;  // alone
     GroupStat gs{0, 0, 0};
     for (int i = lo; i >= 0; i = next[i])
-      if (same_pages(cands[i], cands[lo])) {
+      if (i == lo || same_pages(cands[i], cands[lo])) {
+        member[i] = 1;
         const int64_t rows = int64_t{reqs[cands[i].req].q_len} * G;
         ++gs.members;
         gs.rows_together += rows;
@@ -830,7 +839,8 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
     if (members < 2) continue;
     const bool to_tiles = through_tiles && rows_together >= kTilePackMinRows;
     if (!to_tiles && (rows_together + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup >= tiles_apart) continue;
-    const ReqMeta& first = reqs[cands[lo].req];
+    const int first_req = cands[lo].req;  // the group is served from this request's page ids
+    ctx->pk_keep[first_req] = 1;
     if (to_tiles) {
       // Many rows share the split: 128 to a tile of the tensor-memory kernel, which reads the
       // split once per 128 rows instead of once per 16.
@@ -843,11 +853,11 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
         trows[i] = PackedRow{0, -1, 0, 0};  // padding rows of the last tile see nothing
       for (int64_t t = 0; t < n_tiles; ++t)
         ctx->pk_tile_items.push_back(make_int4(
-            first.bt_off + split * nc::kPagesPerSplit, split,
+            first_req, split,  // .x becomes an index into the flat table once that is laid out
             static_cast<int>(std::min<int64_t>(kPackedTileRows, rows_together - t * kPackedTileRows)), 0));
       PackedRow* pr = trows.data() + first_row;  // real rows are contiguous; only the last tile has padding
       for (int i = lo; i >= 0; i = next[i]) {
-        if (!same_pages(cands[i], cands[lo])) continue;
+        if (!member[i]) continue;
         const ReqMeta& m = reqs[cands[i].req];
         pk_mark[static_cast<size_t>(pk_off[cands[i].req] + split)] = 1;
         const int rows = m.q_len * G;
@@ -871,15 +881,15 @@ int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, i
       SplitItem& si = split_items[n_split_final++];
       si = SplitItem{};
       si.q_len = in_item;  // rows in use
-      si.n_pages = first.n_pages;
-      si.bt_index = first.bt_off + cands[lo].split * nc::kPagesPerSplit;
+      si.n_pages = reqs[first_req].n_pages;
+      si.bt_index = first_req;  // becomes an index into the flat table once that is laid out
       si.split = cands[lo].split;
       si.req = static_cast<int32_t>(-1 - n_packed_items);
       ++n_packed_items;
       in_item = 0;
     };
     for (int i = lo; i >= 0; i = next[i]) {
-      if (!same_pages(cands[i], cands[lo])) continue;
+      if (!member[i]) continue;
       const ReqMeta& m = reqs[cands[i].req];
       const int k = cands[i].split;
       pk_mark[static_cast<size_t>(pk_off[cands[i].req] + k)] = 1;
@@ -941,16 +951,14 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
   const size_t off_items = at;
   std::memcpy(blob + at, plan.items.data() + plan.n_split, sizeof(vosti_work_item) * n_seq);
   at += align_up(sizeof(vosti_work_item) * n_seq, 16);
-  const size_t off_bt = at;
-  int32_t* bt_flat = reinterpret_cast<int32_t*>(blob + at);
-  int64_t bt_used = 0, row0 = 0, n_split_tokens = 0;
+  int64_t row0 = 0, n_split_tokens = 0;
   for (int r = 0; r < batch; ++r) {
     ReqMeta& m = reqs[r];
     m.q_row0 = static_cast<int32_t>(row0);
     m.q_len = q_lens[r];
     m.start = start_pos[r];
     m.n_pages = 0;
-    m.bt_off = static_cast<int32_t>(bt_used);
+    m.bt_off = 0;
     m.n_splits = 0;
     m.first_split = 0;
     m.pad = 0;
@@ -962,40 +970,16 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
     if (cp.phase != 2 && (n_pages > block_table_stride ||
                           (int64_t{seq_lens[r]} + c.page_size - 1) / c.page_size > block_table_stride))
       return VOSTI_ERR_OUT_OF_RANGE;
-    if (cp.phase == 2) {  // the fold reads no pages
-      m.n_pages = static_cast<int32_t>(n_pages);
-      m.first_split = 0;
-      m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1);
-      if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
-      continue;
-    }
-    const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
-    // Pages that lie wholly before the window of the request's first row are never
-    // visible: their table entries are not read (the caller may have freed them);
-    // page 0 stands in where a tile load still covers them.
-    const int64_t first_key = first_visible_key(start_pos[r], window);
-    const int64_t first_page = first_key / c.page_size;
-    for (int64_t b = 0; b < first_page; ++b) bt_flat[bt_used + b] = 0;
-    for (int64_t b = first_page; b < n_pages; ++b) {
-      // a context-parallel rank holds (and names) only the pages of the splits it owns
-      if (cp.phase == 1 && (b / nc::kPagesPerSplit) % cp.world != cp.rank) {
-        bt_flat[bt_used + b] = 0;
-        continue;
-      }
-      const int32_t page = row[b];
-      if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
-      bt_flat[bt_used + b] = page;
-    }
-    bt_used += n_pages;
     m.n_pages = static_cast<int32_t>(n_pages);
-    m.first_split = static_cast<int32_t>(first_key / nc::kSplitLen);
+    m.first_split = cp.phase == 2 ? 0 : static_cast<int32_t>(first_visible_key(start_pos[r], window) / nc::kSplitLen);
     m.n_splits = static_cast<int32_t>((n_eff - 1) / nc::kSplitLen + 1) - m.first_split;
     if (int64_t{q_lens[r]} * G <= nc::kSplitRowsMax) n_split_tokens += q_lens[r];
   }
-  at += align_up(sizeof(int32_t) * bt_used, 16);
 
   // ---- shared-split packing (scheduling only): packed items first in the item list (they walk a
-  // whole split: the longest kind), the others follow in plan order ---------------------------
+  // whole split: the longest kind), the others follow in plan order.  It groups on the caller's
+  // tables, before the flat table is laid out, so that pages only packed items read need not be
+  // copied for every member of a group. -------------------------------------------------------
   int64_t n_split_final = 0, n_packed_items = 0, n_packed_tiles = 0;
   size_t off_packed = 0, off_tile_rows = 0, off_tile_items = 0;
   std::vector<int64_t>& pk_off = ctx->pk_off;
@@ -1004,11 +988,56 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
                        plan.n_partial_rows < (int64_t{1} << 31) && row0 < (int64_t{1} << 24) && G <= 128;
   if (packing) {
     off_packed = at;
-    n_packed_items = pack_shared_splits(ctx, reqs, batch, G, bt_flat, reinterpret_cast<PackedRow*>(blob + at),
-                                        split_items);
+    n_packed_items = pack_shared_splits(ctx, reqs, batch, G, block_tables, block_table_stride,
+                                        reinterpret_cast<PackedRow*>(blob + at), split_items);
     n_split_final = n_packed_items;
     at += align_up(sizeof(PackedRow) * 16 * n_packed_items, 16);
     n_packed_tiles = static_cast<int64_t>(ctx->pk_tile_items.size());
+  }
+
+  // ---- the flat page-id table ------------------------------------------------------------------
+  const size_t off_bt = at;
+  int32_t* bt_flat = reinterpret_cast<int32_t*>(blob + at);
+  int64_t bt_used = 0;
+  for (int r = 0; r < batch && cp.phase != 2; ++r) {  // the fold reads no pages
+    ReqMeta& m = reqs[r];
+    if (q_lens[r] == 0) continue;
+    const int64_t n_pages = m.n_pages;
+    const int32_t* row = block_tables + static_cast<size_t>(r) * block_table_stride;
+    // Pages that lie wholly before the window of the request's first row are never
+    // visible: their table entries are not read (the caller may have freed them);
+    // page 0 stands in where a tile load still covers them.
+    const int64_t first_page = first_visible_key(start_pos[r], window) / c.page_size;
+    // The leading splits of a request that packed items serve are read from the first member of
+    // their group: this request's ids for them are not needed on the device (they equal that
+    // member's, which are copied and checked), unless it is such a first member itself.
+    int64_t skip = 0;
+    if ((n_packed_items > 0 || n_packed_tiles > 0) && !ctx->pk_keep[r]) {
+      const int64_t complete = pk_off[r + 1] - pk_off[r];
+      int64_t lead = 0;
+      while (lead < complete && pk_mark[static_cast<size_t>(pk_off[r] + lead)]) ++lead;
+      skip = lead * nc::kPagesPerSplit;
+    }
+    m.bt_off = static_cast<int32_t>(bt_used - skip);
+    for (int64_t b = skip; b < first_page; ++b) bt_flat[bt_used + b - skip] = 0;
+    for (int64_t b = std::max(skip, first_page); b < n_pages; ++b) {
+      // a context-parallel rank holds (and names) only the pages of the splits it owns
+      if (cp.phase == 1 && (b / nc::kPagesPerSplit) % cp.world != cp.rank) {
+        bt_flat[bt_used + b - skip] = 0;
+        continue;
+      }
+      const int32_t page = row[b];
+      if (page < 0 || page >= c.num_pages) return VOSTI_ERR_OUT_OF_RANGE;
+      bt_flat[bt_used + b - skip] = page;
+    }
+    bt_used += n_pages - skip;
+  }
+  at += align_up(sizeof(int32_t) * bt_used, 16);
+  if (packing) {
+    // packed items and tiles named their group's first request: now its ids have a place
+    for (int64_t i = 0; i < n_packed_items; ++i)
+      split_items[i].bt_index = reqs[split_items[i].bt_index].bt_off + split_items[i].split * nc::kPagesPerSplit;
+    for (int4& ti : ctx->pk_tile_items) ti.x = reqs[ti.x].bt_off + ti.y * nc::kPagesPerSplit;
     off_tile_rows = at;
     std::memcpy(blob + at, ctx->pk_tile_rows.data(), sizeof(PackedRow) * ctx->pk_tile_rows.size());
     at += align_up(sizeof(PackedRow) * ctx->pk_tile_rows.size(), 16);
