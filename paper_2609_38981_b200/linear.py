@@ -6,9 +6,16 @@ import ctypes
 
 import torch
 
+import os
+
 from . import binding as _vb
 
-_lib = _vb._lib
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libvosti_linear.so")
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2609_38981_b200.build` "
+        "(the linear layer has no fallback)")
+_lib = ctypes.CDLL(LIB_PATH)
 _vp = ctypes.c_void_p
 
 EXPORTS = ("vosti_linear_tile_shape", "vosti_linear_segments", "vosti_linear_workspace_bytes", "vosti_linear",
