@@ -35,6 +35,16 @@ def test_library_exports_every_declared_symbol(vb):
     assert sorted(vb.EXPORTS) == names
 
 
+def test_the_attention_library_does_not_contain_the_linear_layer(vb):
+    """Multi-GPU runs carry only the attention library: it must stand on its own."""
+    lib = ctypes.CDLL(vb.LIB_PATH)
+    assert not hasattr(lib, "vosti_linear") and not hasattr(lib, "vosti_rmsnorm")
+    assert not any("linear" in name or "rmsnorm" in name for name in vb.EXPORTS)
+    ignored = open(os.path.join(ROOT, ".gpurunignore.multi")).read().split()
+    assert "paper_2609_38981_b200/csrc/vosti_linear.cu" in ignored
+    assert "paper_2609_38981_b200/libvosti_linear.so" in ignored
+
+
 def test_linear_header_symbols_and_tile_shape(vb):
     """The linear layer's tile shape is a host-side function of (N, K) alone."""
     from paper_2609_38981_b200 import linear as vl
