@@ -17,23 +17,26 @@ namespace vosti {
 
 // Eight workers per SM (two per scheduler, so one worker's instruction latency
 // hides behind the other's); each owns kStages stages of 32 keys (K or V).
-template <int D>
+// With few items (a small batch) a CTA runs fewer workers, each with a deeper ring: a worker's
+// speed is then bound by the bytes it keeps in flight, not by its share of the SM.
+template <int D, int WARPS = 8>
 struct SplitKernelCfg {
-  static constexpr int kWarps = 8;
+  static_assert(WARPS == 8 || WARPS == 4 || WARPS == 2, "workers per CTA");
+  static constexpr int kWarps = WARPS;
   static constexpr int kStageKeys = 32;
-  static constexpr int kStages = (D == 128) ? 3 : 6;
+  static constexpr int kStages = ((D == 128) ? 24 : 48) / WARPS;
   static constexpr int kSmemBytes =
       kWarps * kStages * TileCfg<D, kStageKeys>::kStageBytes + kWarps * kStages * 8 + 1024;
 };
 
-template <int D>
-__global__ void __launch_bounds__(SplitKernelCfg<D>::kWarps * 32, 1)
+template <int D, int WARPS = 8>
+__global__ void __launch_bounds__(WARPS * 32, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {  // kv_map: the 3-D page map
   constexpr bool PM = true;  // stages are page-major: one TMA box per (page, K|V)
-  constexpr int SK = SplitKernelCfg<D>::kStageKeys;
+  constexpr int SK = SplitKernelCfg<D, WARPS>::kStageKeys;
   using C = TileCfg<D, SK>;
-  constexpr int kWarpsPerCta = SplitKernelCfg<D>::kWarps;
-  constexpr int R = SplitKernelCfg<D>::kStages;
+  constexpr int kWarpsPerCta = SplitKernelCfg<D, WARPS>::kWarps;
+  constexpr int R = SplitKernelCfg<D, WARPS>::kStages;
   constexpr int TPS = nc::kTilesPerSplit;
   constexpr int LPT = 2 * C::kParts;  // loads per tile: K parts then V parts
 

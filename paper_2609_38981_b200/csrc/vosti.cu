@@ -410,10 +410,21 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
   if (n_split > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_split * Hkv);
-    // persistent: one CTA per SM, warps draw (item, KV head) tickets
-    const int grid = std::min((p.n_workers + Cfg::kWarps - 1) / Cfg::kWarps, ctx->sm_count);
+    // persistent: one CTA per SM, warps draw (item, KV head) tickets; with few of them, fewer
+    // workers per CTA with deeper rings (scheduling only)
     timed(1, [&] {
-      launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3, p);
+      if (p.n_workers <= 2 * ctx->sm_count) {
+        using C2 = SplitKernelCfg<D, 2>;
+        launch_dependent(attn_split_kernel<D, 2>, std::min((p.n_workers + 1) / 2, ctx->sm_count), 64, C2::kSmemBytes,
+                         stream, ctx->kv_map3, p);
+      } else if (p.n_workers <= 4 * ctx->sm_count) {
+        using C4 = SplitKernelCfg<D, 4>;
+        launch_dependent(attn_split_kernel<D, 4>, std::min((p.n_workers + 3) / 4, ctx->sm_count), 128, C4::kSmemBytes,
+                         stream, ctx->kv_map3, p);
+      } else {
+        const int grid = std::min((p.n_workers + Cfg::kWarps - 1) / Cfg::kWarps, ctx->sm_count);
+        launch_dependent(attn_split_kernel<D>, grid, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3, p);
+      }
     });
   }
   if (n_seq > 0 && run_partials) {
@@ -457,7 +468,11 @@ template <int D>
 vosti_status set_kernel_attributes() {
   using Cfg = SplitKernelCfg<D>;
   if (cudaFuncSetAttribute(attn_split_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           Cfg::kSmemBytes) != cudaSuccess)
+                           Cfg::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_split_kernel<D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SplitKernelCfg<D, 4>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_split_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SplitKernelCfg<D, 2>::kSmemBytes) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            TileKernelCfg<D>::kSmemBytes) != cudaSuccess ||
