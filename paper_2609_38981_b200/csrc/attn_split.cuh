@@ -23,8 +23,10 @@ template <int D, int WARPS = 8>
 struct SplitKernelCfg {
   static_assert(WARPS == 8 || WARPS == 4 || WARPS == 2, "workers per CTA");
   static constexpr int kWarps = WARPS;
-  static constexpr int kStageKeys = 32;
-  static constexpr int kStages = ((D == 128) ? 24 : 48) / WARPS;
+  // With eight workers a ring of three 32-key stages is what the shared memory allows; with fewer,
+  // a stage is a whole 64-key tile (K or V): half as many TMA instructions and barrier probes.
+  static constexpr int kStageKeys = WARPS == 8 ? 32 : 64;
+  static constexpr int kStages = ((D == 128) ? 24 : 48) / WARPS / (kStageKeys / 32);
   static constexpr int kSmemBytes =
       kWarps * kStages * TileCfg<D, kStageKeys>::kStageBytes + kWarps * kStages * 8 + 1024;
 };
