@@ -189,8 +189,13 @@ def run_reference(args):
         return
     w = make_workload(args.workload, 0, args.pool_pages)
     step, cores = oracle_step_factory(w)
-    steps = max(1, min(args.steps, 20))
-    warm = max(0, min(args.warmup, 2))
+    # one step is the whole batch through the oracle (about 70 ms on 16 cores): K steps as asked,
+    # fewer only where K of them would take more than about two minutes
+    t0 = time.perf_counter()
+    step()
+    first = time.perf_counter() - t0
+    steps = max(1, min(args.steps, int(120.0 / max(first, 1e-3))))
+    warm = max(0, min(args.warmup, 3))
     for _ in range(warm):
         step()
     t0 = time.perf_counter()
