@@ -1319,12 +1319,23 @@ vosti_status vosti_kv_append_planned(vosti_ctx* ctx, const void* plan, const voi
 extern "C++" {
 namespace {
 template <int D>
-vosti_status launch_attention_planned(vosti_ctx* ctx, const AttnParams& p, cudaStream_t stream) {
+vosti_status launch_attention_planned(vosti_ctx* ctx, const AttnParams& p, int64_t workers_bound,
+                                      cudaStream_t stream) {
   using Cfg = SplitKernelCfg<D>;
-  // The item count is known to the device only: a full persistent grid, whose idle workers leave at once.
-  if (launch_dependent(attn_split_kernel<D>, ctx->sm_count, Cfg::kWarps * 32, Cfg::kSmemBytes, stream, ctx->kv_map3,
-                       p) != cudaSuccess)
-    return VOSTI_ERR_CUDA;
+  // The item count is known to the device only: a full persistent grid, whose idle workers leave
+  // at once.  The host's bound on it (every request at the longest context the configuration
+  // allows) still picks the few-worker variants for small batches; a loose bound costs speed only.
+  cudaError_t e;
+  if (workers_bound <= 2 * ctx->sm_count)
+    e = launch_dependent(attn_split_kernel<D, 2>, ctx->sm_count, 64, SplitKernelCfg<D, 2>::kSmemBytes, stream,
+                         ctx->kv_map3, p);
+  else if (workers_bound <= 4 * ctx->sm_count)
+    e = launch_dependent(attn_split_kernel<D, 4>, ctx->sm_count, 128, SplitKernelCfg<D, 4>::kSmemBytes, stream,
+                         ctx->kv_map3, p);
+  else
+    e = launch_dependent(attn_split_kernel<D>, ctx->sm_count, Cfg::kWarps * 32, Cfg::kSmemBytes, stream,
+                         ctx->kv_map3, p);
+  if (e != cudaSuccess) return VOSTI_ERR_CUDA;
   const int64_t warps = int64_t{p.n_split_tokens} * p.Hq;
   if (launch_dependent(combine_kernel<D>, static_cast<int>((warps + 3) / 4), 128, 0, stream, p) != cudaSuccess)
     return VOSTI_ERR_CUDA;
@@ -1373,7 +1384,10 @@ vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, con
   p.counts = reinterpret_cast<const int32_t*>(base);
   p.num_pages = static_cast<int32_t>(c.num_pages);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  return c.head_dim == 128 ? launch_attention_planned<128>(ctx, p, stream) : launch_attention_planned<64>(ctx, p, stream);
+  const int64_t groups = (int64_t{max_q_len} * p.G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+  const int64_t workers_bound = int64_t{batch} * groups * ctx->lim.k_max * c.n_kv_heads;
+  return c.head_dim == 128 ? launch_attention_planned<128>(ctx, p, workers_bound, stream)
+                           : launch_attention_planned<64>(ctx, p, workers_bound, stream);
 }
 
 vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream) {
