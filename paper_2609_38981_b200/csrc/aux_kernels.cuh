@@ -12,7 +12,7 @@ namespace vosti {
 template <int D>
 __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
   constexpr int V = D / 32;   // floats per lane
-  constexpr int BATCH = 8;    // partial rows whose loads are in flight together
+  constexpr int BATCH = 8;    // partial rows of a batch; two batches of loads are in flight
   const int lane = threadIdx.x & 31;
   const int widx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (P.counts != nullptr) griddep_wait();  // device-planned: the metadata too comes from the stream
@@ -46,16 +46,27 @@ __global__ void __launch_bounds__(128) combine_kernel(const AttnParams P) {
   };
   float uc[V];
   float mc = 0.f, zc = 0.f;
-  for (int k0 = 0; k0 < n_splits; k0 += BATCH) {
-    float uk[BATCH][V];
-    float2 mz[BATCH];
+  // Two batches of partial rows: the loads of the next one are in flight while this one is folded.
+  float uk[BATCH][V], un[BATCH][V];
+  float2 mz[BATCH], mzn[BATCH];
+  auto load_batch = [&](int k0, float (&u)[BATCH][V], float2 (&m2)[BATCH]) {
 #pragma unroll
     for (int j = 0; j < BATCH; ++j)
       if (k0 + j < n_splits) {
         const int64_t slab = slab0 + static_cast<int64_t>(k0 + j) * rows;
-        mz[j] = P.ws_mz[slab];
-        load_u(slab, uk[j]);
+        m2[j] = P.ws_mz[slab];
+        load_u(slab, u[j]);
       }
+  };
+  load_batch(0, un, mzn);
+  for (int k0 = 0; k0 < n_splits; k0 += BATCH) {
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      mz[j] = mzn[j];
+#pragma unroll
+      for (int i = 0; i < V; ++i) uk[j][i] = un[j][i];
+    }
+    if (k0 + BATCH < n_splits) load_batch(k0 + BATCH, un, mzn);
 #pragma unroll
     for (int j = 0; j < BATCH; ++j)
       if (k0 + j < n_splits) {
