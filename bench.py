@@ -333,16 +333,16 @@ def main():
     if args.device_plan:
         # The same step with its metadata in device memory, planned by a kernel, captured once in a
         # CUDA graph: the host's share of a step is one graph launch.
-        if max(w.q_lens) * (geo.n_q_heads // geo.n_kv_heads) > 32 or args.window:
-            raise SystemExit("--device-plan covers split-parallel batches (decode, speculative) without a window")
+        if max(w.q_lens) * (geo.n_q_heads // geo.n_kv_heads) > 32:
+            raise SystemExit("--device-plan covers split-parallel batches (decode, speculative)")
         plan = torch.empty(vb.vosti_device_plan_bytes(cache.ctx), dtype=torch.uint8, device=dev)
         ql_d, st_d, bt_d = (torch.from_numpy(np.ascontiguousarray(x)).to(dev) for x in (ql, st, bt))
         max_q = int(max(w.q_lens))
 
         def planned_step():
-            vb.vosti_plan_device(cache.ctx, plan, ql_d, st_d, bt_d, max_q)
+            vb.vosti_plan_device(cache.ctx, plan, ql_d, st_d, bt_d, max_q, window=args.window)
             vb.vosti_kv_append_planned(cache.ctx, plan, kn, vn, bt_d, max_q)
-            vb.vosti_paged_attention_planned(cache.ctx, plan, q, out, None, bt_d, max_q, scale)
+            vb.vosti_paged_attention_planned(cache.ctx, plan, q, out, None, bt_d, max_q, scale, window=args.window)
 
         side = torch.cuda.Stream()
         side.wait_stream(stream)

@@ -290,9 +290,13 @@ vosti_status vosti_step_host_wait(vosti_ctx* ctx, int64_t ticket);
  *
  * Only split-parallel requests: every q_len * (n_q_heads / n_kv_heads) <= 32
  * (decode, speculative queries); max_q_len bounds every q_len and must satisfy
- * the same limit (UNSUPPORTED_CONFIG otherwise).  No sliding window.  Rows of
- * q / k_new / v_new / out are packed in request order (sum of q_lens rows),
- * as in the host-planned calls; seq_len of a request is start_pos + q_len.
+ * the same limit (UNSUPPORTED_CONFIG otherwise).  Rows of q / k_new / v_new /
+ * out are packed in request order (sum of q_lens rows), as in the host-planned
+ * calls; seq_len of a request is start_pos + q_len.  `window` is the sliding
+ * window of vosti_paged_attention_ex (0 = none), a host value fixed at
+ * capture; the attention call must be given the window its plan was made
+ * with.  Block-table entries wholly before the window of a request's first row
+ * are not looked at (the caller may have given those pages back).
  *
  *   plan            device, vosti_device_plan_bytes(config) bytes, 16-byte
  *                   aligned; written by vosti_plan_device, read by the other
@@ -313,13 +317,14 @@ size_t vosti_device_plan_bytes(const vosti_config* config);
 vosti_status vosti_plan_device(vosti_ctx* ctx, void* plan, const int32_t* q_lens_dev,
                                const int32_t* start_pos_dev, const int32_t* block_tables_dev,
                                int32_t block_table_stride, int32_t batch, int32_t max_q_len,
-                               void* cuda_stream);
+                               int32_t window, void* cuda_stream);
 vosti_status vosti_kv_append_planned(vosti_ctx* ctx, const void* plan, const void* k_new,
                                      const void* v_new, const int32_t* block_tables_dev, int32_t batch,
                                      int32_t max_q_len, void* cuda_stream);
 vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, const void* q, void* out,
                                            float* lse, const int32_t* block_tables_dev, int32_t batch,
-                                           int32_t max_q_len, float softmax_scale, void* cuda_stream);
+                                           int32_t max_q_len, float softmax_scale, int32_t window,
+                                           void* cuda_stream);
 
 /* Split-parallel paged attention for callers that must not allocate.  (The
  * paper has no counterpart: this is a packaging variant of the operation

@@ -106,12 +106,13 @@ _lib.vosti_step_host_wait.argtypes = [_vp, ctypes.c_int64]
 _lib.vosti_device_plan_bytes.restype = ctypes.c_size_t
 _lib.vosti_device_plan_bytes.argtypes = [_cfgp]
 _lib.vosti_plan_device.restype = ctypes.c_int
-_lib.vosti_plan_device.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp]
+_lib.vosti_plan_device.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                   ctypes.c_int32, _vp]
 _lib.vosti_kv_append_planned.restype = ctypes.c_int
 _lib.vosti_kv_append_planned.argtypes = [_vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32, _vp]
 _lib.vosti_paged_attention_planned.restype = ctypes.c_int
 _lib.vosti_paged_attention_planned.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, ctypes.c_int32, ctypes.c_int32,
-                                               ctypes.c_float, _vp]
+                                               ctypes.c_float, ctypes.c_int32, _vp]
 _lib.vosti_poll_device_status.restype = ctypes.c_int
 _lib.vosti_poll_device_status.argtypes = [_vp, _vp]
 _lib.vosti_selftest_bounded_wait.restype = ctypes.c_int
@@ -376,11 +377,11 @@ def vosti_device_plan_bytes(ctx: Context) -> int:
 
 
 def vosti_plan_device(ctx: Context, plan, q_lens_dev, start_pos_dev, block_tables_dev, max_q_len: int,
-                      stream=None) -> None:
+                      stream=None, window: int = 0) -> None:
     """All array arguments are int32 CUDA tensors; `plan` a CUDA byte tensor of vosti_device_plan_bytes."""
     _check(_lib.vosti_plan_device(ctx.handle, _dev(plan), _dev(q_lens_dev), _dev(start_pos_dev),
                                   _dev(block_tables_dev), block_tables_dev.shape[1], q_lens_dev.shape[0],
-                                  int(max_q_len), _stream(stream)), "vosti_plan_device")
+                                  int(max_q_len), int(window), _stream(stream)), "vosti_plan_device")
 
 
 def vosti_kv_append_planned(ctx: Context, plan, k_new, v_new, block_tables_dev, max_q_len: int,
@@ -391,10 +392,10 @@ def vosti_kv_append_planned(ctx: Context, plan, k_new, v_new, block_tables_dev, 
 
 
 def vosti_paged_attention_planned(ctx: Context, plan, q, out, lse, block_tables_dev, max_q_len: int,
-                                  softmax_scale: float, stream=None) -> None:
+                                  softmax_scale: float, stream=None, window: int = 0) -> None:
     _check(_lib.vosti_paged_attention_planned(ctx.handle, _dev(plan), _dev(q), _dev(out), _dev(lse),
                                               _dev(block_tables_dev), block_tables_dev.shape[0], int(max_q_len),
-                                              float(softmax_scale), _stream(stream)),
+                                              float(softmax_scale), int(window), _stream(stream)),
            "vosti_paged_attention_planned")
 
 

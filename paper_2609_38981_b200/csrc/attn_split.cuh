@@ -111,8 +111,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
     d.n_pages = si.n_pages;
     d.ids = (si.split * nc::kPagesPerSplit + lane < si.n_pages) ? __ldg(P.bt_flat + si.bt_index + lane) : -1;
     if (P.counts != nullptr) {  // nobody has looked at these page ids yet: report strays, read page 0 instead
-      const bool stray = d.ids < -1 || d.ids >= P.num_pages ||
-                         (d.ids == -1 && si.split * nc::kPagesPerSplit + lane < si.n_pages);
+      // (entries wholly before the window of the request's first row are not looked at at all:
+      // the caller may have given those pages back; page 0 stands in where a load still covers them)
+      const int pg = si.split * nc::kPagesPerSplit + lane;
+      if (pg < nc::first_key(si.start, P.window) / nc::kPageSize) d.ids = 0;
+      const bool stray = d.ids < -1 || d.ids >= P.num_pages || (d.ids == -1 && pg < si.n_pages);
       if (__any_sync(kFullMask, stray) && lane == 0) atomicOr(P.status, kStatusBadMetadata);
       if (stray) d.ids = 0;
     }

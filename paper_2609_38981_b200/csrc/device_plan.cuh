@@ -29,8 +29,8 @@ static_assert(sizeof(DevicePlanHeader) == 64, "header is one 64-byte record");
 
 struct DevicePlanScratch {   // per request, between the two phases of the planner
   int32_t full_prefix;       // full-split items of the requests before this one
-  int32_t tail_rel[2];       // per row group: index of its last-split item within its bucket
-  int32_t pad;
+  int32_t part_rel[4];       // per row group, first and last split: index of that item within its bucket, or -1
+  int32_t pad[3];
 };
 
 struct DevicePlanLayout {
@@ -57,7 +57,7 @@ struct DevicePlanArgs {
   const int32_t* start_pos;     // device [batch]
   const int32_t* block_tables;  // device [batch][stride]
   int32_t stride, batch, max_q_len;
-  int32_t G, Hkv;
+  int32_t G, Hkv, window;
   int64_t num_pages, max_seq_len, items_max, toks_max, part_rows_max;
   DevicePlanHeader* header;
   ReqMeta* reqs;
@@ -103,16 +103,32 @@ __device__ __forceinline__ void block_exclusive_scan(const int (&v)[kPlanValues]
   __syncthreads();  // warp_totals is reused by the next chunk of requests
 }
 
-// The key tiles a 16-row group of a request walks, without a sliding window: [0, t1).
+// The key tiles a 16-row group of a request walks: [t0, t1), t0 the tile of the first key its
+// first row sees (0 without a sliding window).  Its items are the splits k0 .. k1 - 1; the first
+// and the last may hold fewer than eight of those tiles, the ones between are full.
 struct GroupSpan {
-  int k1;          // splits: [0, k1)
-  int tiles_last;  // tiles of split k1 - 1 (1..8)
+  int t0, t1, k0, k1;
+  __device__ __forceinline__ int tiles_in(int k) const {
+    return min(t1, (k + 1) * nc::kTilesPerSplit) - max(t0, k * nc::kTilesPerSplit);
+  }
+  // full-split items: [f0, f1)
+  __device__ __forceinline__ int f0() const { return k0 + (tiles_in(k0) < nc::kTilesPerSplit ? 1 : 0); }
+  __device__ __forceinline__ int f1() const {
+    return max(f0(), k1 - ((k1 - 1 > k0 || tiles_in(k0) == nc::kTilesPerSplit) && tiles_in(k1 - 1) < nc::kTilesPerSplit ? 1 : 0));
+  }
+  // partial items: the first split if it is not full; the last split if it is another one and not full
+  __device__ __forceinline__ bool first_partial() const { return tiles_in(k0) < nc::kTilesPerSplit; }
+  __device__ __forceinline__ bool last_partial() const { return k1 - 1 > k0 && tiles_in(k1 - 1) < nc::kTilesPerSplit; }
 };
-__device__ __forceinline__ GroupSpan group_span(int st, int q, int G, int x) {
+__device__ __forceinline__ GroupSpan group_span(int st, int q, int G, int x, int window) {
+  const int first_tok = (x * nc::kRowsPerGroup) / G;
   const int last_tok = min(q - 1, (x * nc::kRowsPerGroup + nc::kRowsPerGroup - 1) / G);
-  const int t1 = (st + last_tok) / nc::kKeyTile + 1;
-  const int k1 = (t1 + nc::kTilesPerSplit - 1) / nc::kTilesPerSplit;
-  return GroupSpan{k1, t1 - (k1 - 1) * nc::kTilesPerSplit};
+  GroupSpan sp;
+  sp.t0 = nc::first_key(st + first_tok, window) / nc::kKeyTile;
+  sp.t1 = (st + last_tok) / nc::kKeyTile + 1;
+  sp.k0 = sp.t0 / nc::kTilesPerSplit;
+  sp.k1 = (sp.t1 + nc::kTilesPerSplit - 1) / nc::kTilesPerSplit;
+  return sp;
 }
 
 // A request as the planner accepts it: lengths outside the premises make it empty (and set
@@ -153,27 +169,29 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
     int v[NV];
 #pragma unroll
     for (int i = 0; i < NV; ++i) v[i] = 0;
-    int tail_bucket[2] = {0, 0};
+    int part_bucket[4] = {0, 0, 0, 0};  // per group: tiles of its partial first / last split, 0 = none
+    int first_split = 0, n_splits = 0;
     if (r < A.batch) {
       if (!plan_request(A, r, q, st)) bad = 1;
       if (q > 0) {
         const int rows = q * A.G;
         const int groups = (rows + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
+        first_split = nc::first_key(st, A.window) / nc::kSplitLen;
+        n_splits = (st + q - 1) / nc::kSplitLen + 1 - first_split;
         v[0] = q;
-        v[1] = A.Hkv * ((st + q - 1) / nc::kSplitLen + 1) * rows;
+        v[1] = A.Hkv * n_splits * rows;
 #pragma unroll
         for (int x = 0; x < 2; ++x) {
           if (x >= groups) continue;
-          const GroupSpan sp = group_span(st, q, A.G, x);
-          if (sp.tiles_last == TPS) {
-            v[2] += sp.k1;
-          } else {
-            v[2] += sp.k1 - 1;
-            tail_bucket[x] = sp.tiles_last;
-#pragma unroll
-            for (int t = 1; t < TPS; ++t) v[3 + t] += sp.tiles_last == t ? 1 : 0;
-          }
+          const GroupSpan sp = group_span(st, q, A.G, x, A.window);
+          v[2] += sp.f1() - sp.f0();
+          if (sp.first_partial()) part_bucket[2 * x] = sp.tiles_in(sp.k0);
+          if (sp.last_partial()) part_bucket[2 * x + 1] = sp.tiles_in(sp.k1 - 1);
         }
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int t = 1; t < TPS; ++t) v[3 + t] += part_bucket[i] == t ? 1 : 0;
       }
     }
     int pre[NV], total[NV];
@@ -185,22 +203,27 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
       m.start = st;
       m.n_pages = q > 0 ? (st + q + nc::kPageSize - 1) / nc::kPageSize : 0;
       m.bt_off = r * A.stride;
-      m.n_splits = q > 0 ? (st + q - 1) / nc::kSplitLen + 1 : 0;
-      m.first_split = 0;
+      m.n_splits = n_splits;
+      m.first_split = first_split;
       m.pad = 0;
       m.part_base = carry[1] + pre[1];
       A.reqs[r] = m;
       DevicePlanScratch s;
       s.full_prefix = carry[2] + pre[2];
       if (prefix_in_smem) full_prefix_s[r] = s.full_prefix;
-      s.tail_rel[0] = s.tail_rel[1] = -1;
+      // a request's partial items that fall into one bucket follow one another there
 #pragma unroll
-      for (int t = 1; t < TPS; ++t) {
-        // two groups of a request in one bucket: the second follows the first
-        if (tail_bucket[0] == t) s.tail_rel[0] = carry[3 + t] + pre[3 + t];
-        if (tail_bucket[1] == t) s.tail_rel[1] = carry[3 + t] + pre[3 + t] + (tail_bucket[0] == t ? 1 : 0);
+      for (int i = 0; i < 4; ++i) {
+        s.part_rel[i] = -1;
+        if (part_bucket[i] == 0) continue;
+        int same_before = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) same_before += (j < i && part_bucket[j] == part_bucket[i]) ? 1 : 0;
+#pragma unroll
+        for (int t = 1; t < TPS; ++t)
+          if (part_bucket[i] == t) s.part_rel[i] = carry[3 + t] + pre[3 + t] + same_before;
       }
-      s.pad = 0;
+      s.pad[0] = s.pad[1] = s.pad[2] = 0;
       A.scratch[r] = s;
       for (int i = 0; i < q; ++i)
         if (m.q_row0 + i < A.toks_max) A.toks[m.q_row0 + i] = make_int2(r, i);
@@ -246,7 +269,7 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
     si.n_splits = m.n_splits;
     si.part_base = m.part_base;
     si.req = r;
-    si.first_split = 0;
+    si.first_split = m.first_split;
     return si;
   };
 
@@ -257,9 +280,11 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
     const DevicePlanScratch s = A.scratch[r];
     const int groups = (m.q_len * A.G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
     for (int x = 0; x < groups; ++x) {
-      if (s.tail_rel[x] < 0) continue;
-      const GroupSpan sp = group_span(m.start, m.q_len, A.G, x);
-      A.items[bucket_base[sp.tiles_last] + s.tail_rel[x]] = make_item(m, r, sp.k1 - 1, x);
+      const GroupSpan sp = group_span(m.start, m.q_len, A.G, x, A.window);
+      if (s.part_rel[2 * x] >= 0)
+        A.items[bucket_base[sp.tiles_in(sp.k0)] + s.part_rel[2 * x]] = make_item(m, r, sp.k0, x);
+      if (s.part_rel[2 * x + 1] >= 0)
+        A.items[bucket_base[sp.tiles_in(sp.k1 - 1)] + s.part_rel[2 * x + 1]] = make_item(m, r, sp.k1 - 1, x);
     }
   }
   // ---- phase B2: full-split items, one thread per item (request by binary search) --------------
@@ -274,20 +299,28 @@ static __global__ void __launch_bounds__(kPlanThreads) device_plan_kernel(const 
     const ReqMeta m = A.reqs[r];
     const int local = j - (prefix_in_smem ? full_prefix_s[r] : A.scratch[r].full_prefix);
     const int groups = (m.q_len * A.G + nc::kRowsPerGroup - 1) / nc::kRowsPerGroup;
-    int f[2] = {0, 0};
+    int fa[2] = {0, 0}, fb[2] = {0, 0};  // full-split items of the groups: [fa, fb)
     for (int x = 0; x < groups; ++x) {
-      const GroupSpan sp = group_span(m.start, m.q_len, A.G, x);
-      f[x] = sp.tiles_last == TPS ? sp.k1 : sp.k1 - 1;
+      const GroupSpan sp = group_span(m.start, m.q_len, A.G, x, A.window);
+      fa[x] = sp.f0();
+      fb[x] = sp.f1();
     }
-    // split outermost, row group innermost, as the host planner orders them
-    const int both = min(f[0], f[1]);
     int k, x;
-    if (local < 2 * both) {
-      k = local >> 1;
-      x = local & 1;
-    } else {
-      k = both + (local - 2 * both);
-      x = f[0] > f[1] ? 0 : 1;
+    if (groups == 2 && fa[0] == fa[1]) {
+      // split outermost, row group innermost, as the host planner orders them: the two groups
+      // that read a split get neighbouring tickets
+      const int both = min(fb[0], fb[1]) - fa[0];
+      if (local < 2 * both) {
+        k = fa[0] + (local >> 1);
+        x = local & 1;
+      } else {
+        k = fa[0] + both + (local - 2 * both);
+        x = fb[0] > fb[1] ? 0 : 1;
+      }
+    } else {  // one group, or ranges that start apart (a sliding window): group by group
+      const int n0 = fb[0] - fa[0];
+      x = local < n0 ? 0 : 1;
+      k = x == 0 ? fa[0] + local : fa[1] + (local - n0);
     }
     A.items[j] = make_item(m, r, k, x);
   }

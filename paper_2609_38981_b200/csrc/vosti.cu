@@ -1249,11 +1249,12 @@ vosti_status planned_call_ok(const vosti_ctx* ctx, const void* plan, const int32
 
 vosti_status vosti_plan_device(vosti_ctx* ctx, void* plan, const int32_t* q_lens_dev,
                                const int32_t* start_pos_dev, const int32_t* block_tables_dev,
-                               int32_t block_table_stride, int32_t batch, int32_t max_q_len,
+                               int32_t block_table_stride, int32_t batch, int32_t max_q_len, int32_t window,
                                void* cuda_stream) {
   vosti_status st = planned_call_ok(ctx, plan, block_tables_dev, batch, max_q_len);
   if (st != VOSTI_OK) return st;
-  if (block_table_stride < 0 || (batch > 0 && (!q_lens_dev || !start_pos_dev))) return VOSTI_ERR_INVALID_ARG;
+  if (block_table_stride < 0 || window < 0 || (batch > 0 && (!q_lens_dev || !start_pos_dev)))
+    return VOSTI_ERR_INVALID_ARG;
   const vosti_config& c = ctx->cfg;
   const DevicePlanLayout L = device_plan_layout(c.max_batch, c.max_total_q, c.max_seq_len);
   uint8_t* base = static_cast<uint8_t*>(plan);
@@ -1266,6 +1267,7 @@ vosti_status vosti_plan_device(vosti_ctx* ctx, void* plan, const int32_t* q_lens
   a.max_q_len = max_q_len;
   a.G = c.n_q_heads / c.n_kv_heads;
   a.Hkv = c.n_kv_heads;
+  a.window = window;
   a.num_pages = c.num_pages;
   a.max_seq_len = c.max_seq_len;
   a.items_max = std::min(L.items_max, ctx->lim.items_max);
@@ -1347,9 +1349,10 @@ vosti_status launch_attention_planned(vosti_ctx* ctx, const AttnParams& p, int64
 
 vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, const void* q, void* out, float* lse,
                                            const int32_t* block_tables_dev, int32_t batch, int32_t max_q_len,
-                                           float softmax_scale, void* cuda_stream) {
+                                           float softmax_scale, int32_t window, void* cuda_stream) {
   vosti_status st = planned_call_ok(ctx, plan, block_tables_dev, batch, max_q_len);
   if (st != VOSTI_OK) return st;
+  if (window < 0) return VOSTI_ERR_INVALID_ARG;
   if (!(softmax_scale >= 0.0f) || !std::isfinite(softmax_scale)) return VOSTI_ERR_INVALID_ARG;
   if (batch == 0) return VOSTI_OK;
   if (!q || !out) return VOSTI_ERR_INVALID_ARG;
@@ -1379,7 +1382,7 @@ vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, con
   p.Hkv = c.n_kv_heads;
   p.G = c.n_q_heads / c.n_kv_heads;
   p.c = static_cast<float>(static_cast<double>(softmax_scale) * 1.4426950408889634074);
-  p.window = 0;
+  p.window = window;  // the one the plan was made with
   p.lse = lse;
   p.counts = reinterpret_cast<const int32_t*>(base);
   p.num_pages = static_cast<int32_t>(c.num_pages);

@@ -295,3 +295,50 @@ def test_large_batches_are_planned_in_chunks(batch):
     assert vb.vosti_last_schedule(host.ctx)[0] > batch          # more items than requests: several splits and groups
     host.close()
     dev.close()
+
+
+@pytest.mark.parametrize("window", [64, 100, 513, 700, 5000])
+def test_sliding_window_steps_equal_the_host_planned_calls(env, window):
+    """Decode and speculative steps under a sliding window: items start at the split that holds
+    the first visible key, the first and last split of a row group may both be partial, and
+    block-table entries wholly before the window hold -1 (pages given back)."""
+    from paper_2609_38981_b200 import binding as vb
+    host, dev = env.new_cache(), env.new_cache()
+    env.prefill(host)
+    env.prefill(dev)
+    plan = new_plan(dev)
+    done = list(CONTEXTS)
+    rng = np.random.default_rng(window)
+    for step in range(4):
+        ql = [int(rng.integers(0, env.max_q + 1)) for _ in CONTEXTS] if step else [1] * len(CONTEXTS)
+        ql = [min(n, c + TAIL - d) for n, c, d in zip(ql, CONTEXTS, done)]
+        if sum(ql) == 0:
+            ql[0] = 1
+        call = [(i, done[i], ql[i]) for i in range(len(CONTEXTS))]
+        q, k, v = env.rows(call)
+        st = [s for _, s, _ in call]
+        # pages wholly before the window of the request's first row: freed
+        bt_w = env.bt.copy()
+        for row, s in enumerate(st):
+            bt_w[row, :max(0, s - window + 1) // env.geo.page_size] = -1
+        vb.vosti_kv_append(host.ctx, k, v, ql, st, env.bt)
+        oh = torch.empty_like(q)
+        lh = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+        vb.vosti_paged_attention_ex(host.ctx, q, oh, lh, ql, st, [s + n for s, n in zip(st, ql)], bt_w, env.scale,
+                                    window=window)
+        ql_d = torch.tensor(ql, dtype=torch.int32, device="cuda")
+        st_d = torch.tensor(st, dtype=torch.int32, device="cuda")
+        bt_d = torch.from_numpy(bt_w).cuda()
+        od = torch.empty_like(q)
+        od.view(torch.int16).fill_(0x7FC1)
+        ld = torch.full(q.shape[:2], float("nan"), dtype=torch.float32, device="cuda")
+        vb.vosti_plan_device(dev.ctx, plan, ql_d, st_d, bt_d, env.max_q, window=window)
+        vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt_d, env.max_q)
+        vb.vosti_paged_attention_planned(dev.ctx, plan, q, od, ld, bt_d, env.max_q, env.scale, window=window)
+        same(od, oh, f"window {window}, step {step}, q_lens {ql}")
+        assert torch.equal(ld.view(torch.int32), lh.view(torch.int32)), f"window {window}, step {step}: log-sum-exp"
+        assert not (od.view(torch.int16) == 0x7FC1).any()
+        done = [d + n for d, n in zip(done, ql)]
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK
+    host.close()
+    dev.close()
