@@ -748,10 +748,15 @@ namespace {
 
 // Shared-split packing (scheduling only).  Candidates: complete splits (all 512 keys below every
 // row of the request) of split-parallel requests.  Requests whose 32 page ids of a split agree
-// form a group; the rows of a group of two or more are laid out 16 to a packed item, if that
-// saves tiles.  Writes the packed rows at `packed_rows`, one SplitItem per packed item at the
-// front of `split_items`, marks the (request, split) pairs it has taken over in ctx->pk_mark,
-// and returns the number of packed items.
+// (compared in the caller's block tables) form a group, served from its first member's ids.  The
+// rows of a group of two or more are laid out 16 to a packed item of the split-parallel kernel, if
+// that saves tiles, or -- large groups, when they add up to enough work -- 128 to a packed tile of
+// the tile kernel (ctx->pk_tile_rows / pk_tile_items).  Writes the 16-row packed rows at
+// `packed_rows`, one SplitItem per packed item at the front of `split_items`, marks the (request,
+// split) pairs it has taken over in ctx->pk_mark and the first members in ctx->pk_keep, and
+// returns the number of 16-row packed items.  Items and tiles name their group's first request
+// where the index into the flat page table will go: the caller patches that in once the table is
+// laid out.
 int64_t pack_shared_splits(vosti_ctx* ctx, const ReqMeta* reqs, int32_t batch, int G, const int32_t* block_tables,
                            int32_t block_table_stride, PackedRow* packed_rows, SplitItem* split_items) {
   // page ids of split k of request r, in the caller's table (not validated here: a group is served
