@@ -154,3 +154,72 @@ def test_prefix_reuse_through_the_cache_manager(setup):
     assert mgr.check() == ""
     dev.close()
     mgr.close()
+
+
+def test_a_whole_layer_decode_step_replays_from_a_cuda_graph(setup):
+    """One capture of a decode step of the layer -- RMS norm, QKV projection, rotary embedding, device-side
+    planning, KV append, attention, output projection, MLP -- with positions and block tables in device
+    memory; every replay equals the eager, host-planned step bit for bit."""
+    from paper_2609_38981_b200 import binding as vb
+    from paper_2609_38981_b200 import linear as vl
+    from paper_2609_38981_b200.harness import DeviceCache, bf16_bits
+    layer, requests, alone = setup
+    reqs = [r for r in requests if len(r) > 12]
+    B, tail = len(reqs), 6
+    tables = inputs._assign_private_pages(inputs.generator(9), GEO, 256, [len(r) for r in reqs])
+    dev = DeviceCache(GEO, 256, max_batch=16, max_total_q=2048, max_seq_len=MAXLEN, pool_fill="nan")
+    # prefill eagerly (host-planned), all but the last `tail` positions
+    run(layer, reqs, [[(i, 0, len(r) - tail) for i, r in enumerate(reqs)]], tables=tables, cache=dev)
+    bt = torch.from_numpy(inputs.block_table_array(tables)).cuda()
+    tok = torch.zeros(B, dtype=torch.long, device="cuda")
+    pos = torch.zeros(B, dtype=torch.int32, device="cuda")
+    ones = torch.ones(B, dtype=torch.int32, device="cuda")
+    plan = torch.empty(vb.vosti_device_plan_bytes(dev.ctx), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    y = torch.zeros((B, D_MODEL), dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        x = layer.emb[tok]
+        p = pos.long()
+        h = vl.vosti_rmsnorm(x, layer.g1, EPS)
+        qkv = vl.vosti_linear(h, layer.w_qkv, workspace=ws).view(B, -1, GEO.head_dim)
+        q = layer.rope(qkv[:, :GEO.n_q_heads], p).contiguous()
+        k = layer.rope(qkv[:, GEO.n_q_heads:GEO.n_q_heads + GEO.n_kv_heads], p).contiguous()
+        v = qkv[:, GEO.n_q_heads + GEO.n_kv_heads:].contiguous()
+        att = torch.empty_like(q)
+        vb.vosti_plan_device(dev.ctx, plan, ones, pos, bt, 1)
+        vb.vosti_kv_append_planned(dev.ctx, plan, k, v, bt, 1)
+        vb.vosti_paged_attention_planned(dev.ctx, plan, q, att, None, bt, 1, GEO.head_dim ** -0.5)
+        o = vl.vosti_linear(att.view(B, -1), layer.w_o, workspace=ws)
+        x1 = (x.float() + o.float()).to(torch.bfloat16)
+        h2 = vl.vosti_rmsnorm(x1, layer.g2, EPS)
+        gu = vl.vosti_linear(h2, layer.w_gu, workspace=ws)
+        gate, up = gu[:, :D_FFN].float(), gu[:, D_FFN:].float()
+        act = (gate * torch.sigmoid(gate) * up).to(torch.bfloat16).contiguous()
+        down = vl.vosti_linear(act, layer.w_d, workspace=ws)
+        y.copy_((x1.float() + down.float()).to(torch.bfloat16))
+
+    def load(d):
+        tok.copy_(torch.tensor([r[len(r) - tail + d] for r in reqs]))
+        pos.copy_(torch.tensor([len(r) - tail + d for r in reqs], dtype=torch.int32))
+
+    load(0)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                                  # warm-up outside capture (writes position len - tail, as replay 0 will)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    index = {id(r): i for i, r in enumerate(requests)}
+    for d in range(tail):
+        load(d)
+        graph.replay()
+        got = bf16_bits(y)
+        for j, r in enumerate(reqs):
+            want = alone[index[id(r)]][len(r) - tail + d]
+            assert torch.equal(got[j], want), f"replay {d}, request {j}: differs from its run alone"
+    assert vb.vosti_poll_device_status(dev.ctx) == vb.VOSTI_OK and vl.vosti_linear_poll_status() == 0
+    dev.close()
