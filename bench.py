@@ -497,7 +497,7 @@ def main():
                     "useful_flops_per_launch": flops, "kernel_us": k_ms * 1e3,
                     "launches_timed": int(kernels_timed), "traffic": None}
         else:
-            roof = {"bound": "hbm", "kernel": "attn_split_kernel<128>",
+            roof = {"bound": "hbm", "kernel": "attn_split_kernel<128, 8>",
                     "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": (achieved / peak) if achieved else None,
                     "frac_of_8TBs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
