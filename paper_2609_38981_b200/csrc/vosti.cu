@@ -1058,12 +1058,14 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
     for (int64_t i = 0; i < n_packed_items; ++i)
       split_items[i].bt_index = reqs[split_items[i].bt_index].bt_off + split_items[i].split * nc::kPagesPerSplit;
     for (int4& ti : ctx->pk_tile_items) ti.x = reqs[ti.x].bt_off + ti.y * nc::kPagesPerSplit;
-    off_tile_rows = at;
-    std::memcpy(blob + at, ctx->pk_tile_rows.data(), sizeof(PackedRow) * ctx->pk_tile_rows.size());
-    at += align_up(sizeof(PackedRow) * ctx->pk_tile_rows.size(), 16);
-    off_tile_items = at;
-    std::memcpy(blob + at, ctx->pk_tile_items.data(), sizeof(int4) * ctx->pk_tile_items.size());
-    at += align_up(sizeof(int4) * ctx->pk_tile_items.size(), 16);
+    if (n_packed_tiles > 0) {
+      off_tile_rows = at;
+      std::memcpy(blob + at, ctx->pk_tile_rows.data(), sizeof(PackedRow) * ctx->pk_tile_rows.size());
+      at += align_up(sizeof(PackedRow) * ctx->pk_tile_rows.size(), 16);
+      off_tile_items = at;
+      std::memcpy(blob + at, ctx->pk_tile_items.data(), sizeof(int4) * ctx->pk_tile_items.size());
+      at += align_up(sizeof(int4) * ctx->pk_tile_items.size(), 16);
+    }
   }
   for (int64_t i = 0; i < plan.n_split; ++i) {
     const vosti_work_item& it = plan.items[i];
