@@ -331,17 +331,21 @@ vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, con
  * above, not a different computation.)
  *
  * Some callers cannot call cudaMalloc or create a vosti_ctx (which pins host
- * memory and creates events): code that runs while a stream is being captured,
- * serving loops whose memory is budgeted up front and owned by an outside
- * allocator, plug-ins that receive device pointers but may not create their
- * own.  This entry point allocates nothing on host or device and needs no
- * context.  Its scratch (scheduler words, the call's metadata, the partial
+ * memory and creates streams and events): a serving engine that reserved all
+ * device memory for its KV pool at start-up and owns the rest through its own
+ * allocator, a latency-critical decode loop that cannot afford the device-wide
+ * synchronisation of cudaMalloc / cudaFree, a plug-in that receives device
+ * pointers from its host framework but may not create memory of its own.
+ * This entry point allocates nothing on host or device and needs no context.
+ * Its scratch (status and scheduler words, the call's metadata, the partial
  * (m, z, U) rows) is a 16 MiB file-scope device array that every GPU loading
  * the library holds until the process exits.  It launches the same kernels
  * as vosti_paged_attention, so the output bits are the same.
  *
  *   kv_pool, q, out   device, as for vosti_paged_attention (pool 1024-byte aligned)
  *   q_lens, start_pos, seq_lens, block_tables   host, same meaning as above
+ *   cuda_stream       a stream of the CURRENT device (the scratch used is the
+ *                     current device's); pool, q and out live on that device
  * Limits (beyond them the call returns VOSTI_ERR_WORKSPACE and launches
  * nothing): batch <= 64, sum of q_lens <= 256, at most 16384 page-table
  * entries in use, at most 1024 (row group, split) items, at most 28000
@@ -350,16 +354,35 @@ vosti_status vosti_paged_attention_planned(vosti_ctx* ctx, const void* plan, con
  * longer queries return VOSTI_ERR_UNSUPPORTED_CONFIG.
  * The first call on a device resolves the scratch array's device address and
  * sets kernel attributes; make that first call before any stream capture.
- * All calls share the one array: it is cleared where it must start at zero,
- * and two calls that overlap on the GPU (different streams, or the same
- * library used from two threads without ordering) race on it.  Host metadata
- * is staged synchronously; the kernels run asynchronously on the stream. */
+ * The call plans on the host and copies its metadata (only the part in use)
+ * from a pageable host buffer inside the library: it returns once that is
+ * staged, which waits for earlier work on the stream; the kernels then run
+ * asynchronously on the stream.
+ * All calls share the one array: what must start at zero is cleared by every
+ * call, and two calls that overlap on the GPU (different streams, or the same
+ * library used from two threads without ordering) race on it.
+ * Failure detection: a kernel that gives up on a bounded wait sets the status
+ * word at the start of the array (its output is then undefined).  Calls do
+ * not clear that word; vosti_noalloc_poll_status does. */
 vosti_status vosti_paged_attention_noalloc(int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim,
                                            int32_t page_size, const void* kv_pool, int64_t num_pages,
                                            const void* q, void* out, const int32_t* q_lens,
                                            const int32_t* start_pos, const int32_t* seq_lens,
                                            const int32_t* block_tables, int32_t block_table_stride,
                                            int32_t batch, float softmax_scale, void* cuda_stream);
+
+/* The status word of the allocation-free entry point, on the current device:
+ * waits for the stream, reads the word, clears it, and returns VOSTI_OK or
+ * VOSTI_ERR_TIMEOUT (a kernel of some vosti_paged_attention_noalloc call
+ * since the last poll gave up on a bounded wait).  Allocates nothing and
+ * needs no context.  (No counterpart in the paper.) */
+vosti_status vosti_noalloc_poll_status(void* cuda_stream);
+
+/* Failure-detection self-test of that path (no GPU fault involved): one warp
+ * waits limit_us microseconds (1..100000) on a barrier nothing completes,
+ * gives up, sets the static status word and returns normally; the next
+ * vosti_noalloc_poll_status reports VOSTI_ERR_TIMEOUT and clears it. */
+vosti_status vosti_noalloc_selftest_bounded_wait(uint32_t limit_us, void* cuda_stream);
 
 /* Waits for the stream and reads the device status word: VOSTI_OK,
  * VOSTI_ERR_TIMEOUT if a kernel gave up on a bounded wait (its output is
@@ -397,10 +420,20 @@ int64_t vosti_launch_count(const vosti_ctx* ctx);
 vosti_status vosti_last_schedule(const vosti_ctx* ctx, int64_t* split_items, int64_t* packed_items,
                                  int64_t* tile_items);
 
-/* Hash of the frozen numerics (tile size, split length, fold and exponent
- * rules, library version): the paper's deployment identity W.  ctx may be
- * NULL. */
+/* Hash of the frozen numerics: the paper's deployment identity W (Sec. "A
+ * System-Level Formulation": outputs are compared under one fixed deployment
+ * configuration).  It is computed from the list vosti_contract returns -- the
+ * library version, key tile, split length, rows per group, the split-parallel
+ * row limit, page size, and one id per rule that decides bits (exponent,
+ * reference maximum and its step, row-sum order, fold, reciprocal, zero sign,
+ * MMA chunk order, log-sum-exp) -- plus, with a context, its head_dim and
+ * page_size.  Two builds with equal fingerprints give equal bits on the same
+ * GPU model.  ctx may be NULL. */
 uint64_t vosti_fingerprint(const vosti_ctx* ctx);
+
+/* The words the fingerprint is made of, in hashing order; returns their
+ * number (at most 32) and writes min(number, cap) of them.  Host-only. */
+int32_t vosti_contract(uint32_t* words, int32_t cap);
 
 /* Frozen constants: key tile B_N, split length L_S, rows per row group. */
 void vosti_constants(int32_t* key_tile, int32_t* split_len, int32_t* rows_per_group);

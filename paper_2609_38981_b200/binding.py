@@ -31,12 +31,13 @@ VOSTI_HOST_STEPS_IN_FLIGHT = 3
 
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
-    "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_cp_partial",
+    "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_noalloc_poll_status",
+    "vosti_noalloc_selftest_bounded_wait", "vosti_cp_partial",
     "vosti_cp_combine", "vosti_step_host", "vosti_step_host_async", "vosti_step_host_wait",
     "vosti_device_plan_bytes", "vosti_plan_device", "vosti_kv_append_planned", "vosti_paged_attention_planned",
     "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
-    "vosti_last_schedule", "vosti_fingerprint",
+    "vosti_last_schedule", "vosti_fingerprint", "vosti_contract",
     "vosti_constants", "vosti_status_string",
 )
 
@@ -96,6 +97,10 @@ _lib.vosti_paged_attention_noalloc.restype = ctypes.c_int
 _lib.vosti_paged_attention_noalloc.argtypes = [
     ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _vp, ctypes.c_int64, _vp, _vp,
     _i32p, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
+_lib.vosti_noalloc_poll_status.restype = ctypes.c_int
+_lib.vosti_noalloc_poll_status.argtypes = [_vp]
+_lib.vosti_noalloc_selftest_bounded_wait.restype = ctypes.c_int
+_lib.vosti_noalloc_selftest_bounded_wait.argtypes = [ctypes.c_uint32, _vp]
 _lib.vosti_step_host.restype = ctypes.c_int
 _lib.vosti_step_host.argtypes = [_vp, _vp, _vp, _vp, _vp, _i32p, _i32p, _i32p, _i32p,
                                  ctypes.c_int32, ctypes.c_int32, ctypes.c_float, _vp]
@@ -129,6 +134,8 @@ _lib.vosti_last_schedule.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes
                                      ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_fingerprint.restype = ctypes.c_uint64
 _lib.vosti_fingerprint.argtypes = [_vp]
+_lib.vosti_contract.restype = ctypes.c_int32
+_lib.vosti_contract.argtypes = [ctypes.POINTER(ctypes.c_uint32), ctypes.c_int32]
 _lib.vosti_constants.restype = None
 _lib.vosti_constants.argtypes = [_i32p, _i32p, _i32p]
 _lib.vosti_status_string.restype = ctypes.c_char_p
@@ -224,6 +231,13 @@ def vosti_plan_ex(cfg: vosti_config, q_lens, start_pos, seq_lens, window: int):
 
 def vosti_fingerprint(ctx=None) -> int:
     return int(_lib.vosti_fingerprint(ctx.handle if ctx is not None else None))
+
+
+def vosti_contract():
+    """The words vosti_fingerprint hashes (version, frozen sizes, rule ids), in order."""
+    buf = (ctypes.c_uint32 * 32)()
+    n = _lib.vosti_contract(buf, 32)
+    return [int(x) for x in buf[:n]]
 
 
 class Context:
@@ -344,6 +358,16 @@ def vosti_paged_attention_noalloc(n_q_heads, n_kv_heads, head_dim, page_size, kv
         n_q_heads, n_kv_heads, head_dim, page_size, _dev(kv_pool), num_pages, _dev(q), _dev(out),
         _ip(ql), _ip(s), _ip(n), _ip(bt), bt.shape[1], len(ql), float(softmax_scale),
         _stream(stream)), "vosti_paged_attention_noalloc")
+
+
+def vosti_noalloc_poll_status(stream=None) -> int:
+    """Reads and clears the status word of the allocation-free entry point (current device)."""
+    return _lib.vosti_noalloc_poll_status(_stream(stream))
+
+
+def vosti_noalloc_selftest_bounded_wait(limit_us: int, stream=None) -> None:
+    _check(_lib.vosti_noalloc_selftest_bounded_wait(int(limit_us), _stream(stream)),
+           "vosti_noalloc_selftest_bounded_wait")
 
 
 def vosti_step_host(ctx: Context, q_host, out_host, k_new_host, v_new_host, q_lens, start_pos,

@@ -22,6 +22,9 @@
 //     some alpha of its warp is not 1, zero-fills value rows no query row may
 //     see, and at the end of every split folds the split into the running
 //     result (and, at the end of the row, normalises and stores it).
+// (With the lazy reference maximum of the contract alpha is 1 in the common
+// case, so the correction thread's per-tile work is a handshake; the thread is
+// there for the rare rescale and for the fold.)
 // Roles by warpgroup (384 threads): 0 = softmax, 1 = correction, 2 = { K
 // producer, MMA issuer, V producer }.  Registers are moved from warpgroup 2 to
 // the others with setmaxnreg.  The MMAs of the one issuing thread run in issue
@@ -36,7 +39,14 @@
 // written over the first 32 columns of the S buffer they were computed from)
 // and U (D).  The running fold U_c lives in global memory (per CTA a
 // [D/4][128 rows] array of float4, so that a warp's rows are contiguous; touched
-// once per split): there is no room for it on chip.
+// once per split): there is no room for it on chip.  A correction thread asks
+// for three 16-column chunks of its row's running fold ahead of their use.
+// Measured and not kept (both bitwise correct): copying a finished split out and
+// folding it behind the next split's tiles doubles the traffic through the SM's
+// load/store path and is slower; dividing a row's key columns between two
+// threads (two symmetric warpgroups that exchange half-row maxima and sums
+// through shared memory) makes the hand-over part of every tile's chain and is
+// slower too.
 #pragma once
 #include "meta.cuh"
 #include "tcgen05.cuh"
@@ -62,8 +72,9 @@ struct TileKernelCfg {
   // others have released waits for ever.
   static constexpr int kRegsLaunch = 80;
   static constexpr int kRegsSoftmax = 112;
-  static constexpr int kRegsCorrection = 96;
-  static constexpr int kRegsOther = 32;
+  static constexpr int kRegsCorrection = 104;
+  static constexpr int kRegsOther = 24;
+  static constexpr int kFoldAhead = 3;  // chunks of 16 running-fold columns requested ahead of their use
   static constexpr int kRegsAfterSplit = 128 * (kRegsSoftmax + kRegsCorrection + kRegsOther);
   static_assert(kRegsAfterSplit <= kThreads * kRegsLaunch, "register split exceeds the launch allocation");
   // tensor-memory columns
@@ -382,21 +393,27 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           for (int i = 0; i < KT; ++i)
             sr[i] = (key0 + i <= p && key0 + i > lo) ? __float_as_uint(nc::weight(__uint_as_float(sr[i]), c, ng)) : 0u;
         }
-        // four partial sums over (b mod 8) / 2, ascending b; then (s0 + s1) + (s2 + s3).
-        // Partials 0 and 1 advance together in one packed add, as do partials 2 and 3.
-        float part[4];
+        // Pinned row sum, per half of 32 lanes: eight chains over b mod 8 (ascending b), chain pairs,
+        // (P0 + P1) + (P2 + P3); then lower half + upper half.  Chains 2q and 2q+1 advance together
+        // in one packed add on the adjacent lanes (8n + 2q, 8n + 2q + 1).
+        float half_sum[2];
 #pragma unroll
-        for (int q = 0; q < 4; q += 2) {
-          uint64_t acc = nc::pack2(__uint_as_float(sr[2 * q]), __uint_as_float(sr[2 * q + 2]));
-          acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[2 * q + 1]), __uint_as_float(sr[2 * q + 3])));
+        for (int hf = 0; hf < 2; ++hf) {
+          float part[4];
 #pragma unroll
-          for (int n = 1; n < 8; ++n) {
-            acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[8 * n + 2 * q]), __uint_as_float(sr[8 * n + 2 * q + 2])));
-            acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[8 * n + 2 * q + 1]), __uint_as_float(sr[8 * n + 2 * q + 3])));
+          for (int q = 0; q < 4; ++q) {
+            uint64_t acc = nc::pack2(__uint_as_float(sr[32 * hf + 2 * q]), __uint_as_float(sr[32 * hf + 2 * q + 1]));
+#pragma unroll
+            for (int n = 1; n < 4; ++n)
+              acc = nc::add2(acc, nc::pack2(__uint_as_float(sr[32 * hf + 8 * n + 2 * q]),
+                                            __uint_as_float(sr[32 * hf + 8 * n + 2 * q + 1])));
+            float e0, e1;
+            nc::unpack2(acc, e0, e1);
+            part[q] = __fadd_rn(e0, e1);
           }
-          nc::unpack2(acc, part[q], part[q + 1]);
+          half_sum[hf] = nc::quad_total(part[0], part[1], part[2], part[3]);
         }
-        const float total = nc::quad_total(part[0], part[1], part[2], part[3]);
+        const float total = nc::tile_total(half_sum[0], half_sum[1]);
         z = h ? nc::z_update(z, alpha, total) : z;
         m = mn;
       }
@@ -451,26 +468,27 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       if (!ok) break;
       const float alpha = alpha_s[b * TR + r];
       // The accumulator of a split's first tile is fresh: nothing to rescale.  Otherwise U is
-      // rescaled unless alpha is exactly 1 for every row of the warp (u * 1 = u bit for bit);
-      // it must be at rest for that: PV of the previous tile done.
+      // rescaled unless alpha is exactly 1 for every row of the warp (u * 1 = u bit for bit;
+      // with the lazy reference maximum that is the common case); it must be at rest for that:
+      // PV of the previous tile done.
       if ((t % TPS) != 0 && t != T0 && !__all_sync(kFullMask, alpha == 1.0f)) {
         ok = __all_sync(kFullMask, wait(pv_done + 8 * ((ti - 1) & 1), ((ti - 1) >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
 #pragma unroll 1
-        for (int cb = 0; cb < D; cb += 32) {
-          uint32_t ur[32];
-          tmem_ld32(tmem + lane_sel + Cfg::kColU + cb, ur);
+        for (int cb = 0; cb < D; cb += 16) {
+          uint32_t ur[16];
+          tmem_ld16(tmem + lane_sel + Cfg::kColU + cb, ur);
           tmem_wait_ld();
           const uint64_t alpha2 = nc::pack2(alpha, alpha);
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) {  // u * alpha, two lanes per instruction
+          for (int i = 0; i < 16; i += 2) {  // u * alpha, two lanes per instruction
             float u0, u1;
             nc::unpack2(nc::mul2(nc::pack2(__uint_as_float(ur[i]), __uint_as_float(ur[i + 1])), alpha2), u0, u1);
             ur[i] = __float_as_uint(u0);
             ur[i + 1] = __float_as_uint(u1);
           }
-          tmem_st32(tmem + lane_sel + Cfg::kColU + cb, ur);
+          tmem_st16(tmem + lane_sel + Cfg::kColU + cb, ur);
         }
         tmem_wait_st();
       }
@@ -503,7 +521,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
       tc_fence_before();
       mbar_arrive(p_full + 8 * b);
 
-      // ---- end of a split: fold it into the running result (kept in global memory) -------
+      // ---- end of a split -------------------------------------------------------------------
       if constexpr (PACKED) {
         if (t + 1 == n_tiles) {  // the split is complete: its raw (m, z, U) is the row's partial
           ok = __all_sync(kFullMask, wait(mz_full, 0));
@@ -530,11 +548,14 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         const int split = t / TPS;
         const int kb = (split - T0 / TPS) & 1, kuse = (split - T0 / TPS) >> 1;
         const bool resume = split > T0 / TPS;  // the CTA has stored a running result before
-        // the running-fold values do not depend on the PV in flight: request the first chunk now
-        float4 nxt4[4];
+        const bool last = t + 1 == n_tiles;
+        // The running-fold values do not depend on the PV in flight: request the first kFoldAhead
+        // chunks of 16 columns now; a chunk's registers are refilled as soon as it has been used.
+        constexpr int kFoldAhead = Cfg::kFoldAhead < D / 16 ? Cfg::kFoldAhead : D / 16;
+        float4 uc4[4 * kFoldAhead];
         if (resume) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i) nxt4[i] = ucg[static_cast<size_t>(i) * TR];
+          for (int i = 0; i < 4 * kFoldAhead; ++i) uc4[i] = ucg[static_cast<size_t>(i) * TR];
         }
         ok = __all_sync(kFullMask, wait(mz_full + 8 * kb, kuse & 1));
         if (!ok) break;
@@ -542,7 +563,6 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         ok = __all_sync(kFullMask, wait(pv_done + 8 * b, (ti >> 1) & 1));
         if (!ok) break;
         tc_fence_after();
-        const bool last = t + 1 == n_tiles;
         const bool take = split <= k_first;  // the row's first split: the running result starts from it
         const bool sees = p >= split * nc::kSplitLen;
         nc::FoldFactors f;
@@ -557,27 +577,27 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         const float inv = nc::out_scale(zc);  // used on the last split only
         if (last && valid && P.lse != nullptr)
           P.lse[static_cast<size_t>(rq.q_row0 + tok) * P.Hq + kvh * G + row % G] = nc::lse_value(mc, zc);
-        // chunks of 16 columns; the running-fold values of chunk c+1 are requested before chunk c is processed
-#pragma unroll 1
+#pragma unroll
         for (int cb = 0; cb < D; cb += 16) {
+          const int slot = ((cb / 16) % kFoldAhead) * 4;
           uint32_t ur[16];
           tmem_ld16(tmem + lane_sel + Cfg::kColU + cb, ur);
-          float un[16];
-          if (resume) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              un[4 * i] = nxt4[i].x; un[4 * i + 1] = nxt4[i].y; un[4 * i + 2] = nxt4[i].z; un[4 * i + 3] = nxt4[i].w;
-            }
-            if (cb + 16 < D) {
-#pragma unroll
-              for (int i = 0; i < 4; ++i) nxt4[i] = ucg[static_cast<size_t>((cb + 16) / 4 + i) * TR];
-            }
-          }
           tmem_wait_ld();
+          float un[16];
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const float u = __uint_as_float(ur[i]);
-            un[i] = take ? u : (sees ? nc::fold_u(un[i], u, f) : un[i]);
+          for (int i = 0; i < 4; ++i) {
+            const float4 x = uc4[slot + i];
+            const float u0 = __uint_as_float(ur[4 * i]), u1 = __uint_as_float(ur[4 * i + 1]);
+            const float u2 = __uint_as_float(ur[4 * i + 2]), u3 = __uint_as_float(ur[4 * i + 3]);
+            un[4 * i] = take ? u0 : (sees ? nc::fold_u(x.x, u0, f) : x.x);
+            un[4 * i + 1] = take ? u1 : (sees ? nc::fold_u(x.y, u1, f) : x.y);
+            un[4 * i + 2] = take ? u2 : (sees ? nc::fold_u(x.z, u2, f) : x.z);
+            un[4 * i + 3] = take ? u3 : (sees ? nc::fold_u(x.w, u3, f) : x.w);
+          }
+          if (resume && cb / 16 + kFoldAhead < D / 16) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              uc4[slot + i] = ucg[static_cast<size_t>((cb / 16 + kFoldAhead) * 4 + i) * TR];
           }
           if (last) {
             if (valid) {

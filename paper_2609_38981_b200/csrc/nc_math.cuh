@@ -26,7 +26,20 @@ constexpr int kSplitRowsMax = 32;   // requests with at most this many rows per 
 constexpr int kPageSize = 16;
 constexpr int kPagesPerTile = kKeyTile / kPageSize;
 constexpr int kPagesPerSplit = kSplitLen / kPageSize;
-constexpr uint32_t kVersion = 1;
+constexpr uint32_t kVersion = 2;
+
+// Rule ids: every choice below that decides output bits has a name and a value here, and
+// vosti_fingerprint hashes all of them (a changed rule must change its value).
+constexpr uint32_t kRuleExponent = 1;   // A = ex2.approx.ftz(fma(S, c, -m_hat)), alpha = ex2.approx.ftz(m - m_hat)
+constexpr uint32_t kRuleMaximum = 2;    // lazy reference maximum: m_hat moves only when the tile's scaled maximum
+                                        // exceeds m by more than kLazyMaxStep (1 would be the exact running maximum)
+constexpr uint32_t kRuleRowSum = 3;     // per half of 32 lanes: eight chains over b mod 8, pairs, (P0 + P1) + (P2 + P3); lower + upper
+constexpr uint32_t kRuleFold = 1;       // left fold by split index: z = fma(z_c, a, z_k * b), U likewise
+constexpr uint32_t kRuleReciprocal = 1; // 1 / z by rcp.rn, O = U * inv
+constexpr uint32_t kRuleZeroSign = 1;   // O + 0.0: an exact zero is +0
+constexpr uint32_t kRuleMmaChunks = 1;  // bf16 x bf16 -> fp32, chunks of 16 ascending, fresh accumulator per tile / split
+constexpr uint32_t kRuleLse = 1;        // (m + lg2.approx.ftz(z)) * ln 2
+constexpr float kLazyMaxStep = 8.0f;    // base-two domain: weights stay below 2^8
 
 __device__ __forceinline__ float ex2(float x) {
   float y;
@@ -34,15 +47,21 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// Running maximum in the scaled (base-two) domain.  The raw maximum is taken
-// over visible lanes first; multiplying by c >= 0 is monotone, so this equals
-// the maximum of the scaled scores.
+// Reference maximum in the scaled (base-two) domain.  The raw maximum is taken
+// over visible lanes first; multiplying by c >= 0 is monotone, so its product
+// with c is the maximum of the scaled scores.  The reference is LAZY: it moves
+// to the tile's maximum only when that exceeds it by more than kLazyMaxStep, so
+// that in the common case alpha is exactly 1 and U needs no rescale.  Any
+// reference within a bounded distance of the true maximum gives the same
+// quotient U / z up to rounding; this one keeps every weight below 2^8.  The
+// first visible tile of a split always sets it (m_old = -inf).
 __device__ __forceinline__ float new_max(float m_old, float raw_max_visible, float c) {
-  return fmaxf(m_old, __fmul_rn(raw_max_visible, c));
+  const float t = __fmul_rn(raw_max_visible, c);
+  return t > __fadd_rn(m_old, kLazyMaxStep) ? t : m_old;
 }
-// alpha = 2^(m - m_hat)
+// alpha = 2^(m - m_hat); ex2(0) is exactly 1, so the unchanged case needs no instruction
 __device__ __forceinline__ float rescale(float m_old, float m_new) {
-  return ex2(__fsub_rn(m_old, m_new));
+  return m_old == m_new ? 1.0f : ex2(__fsub_rn(m_old, m_new));
 }
 // A = 2^(s*c - m_hat), one fused multiply-add then the exponential.
 __device__ __forceinline__ float weight(float s, float c, float neg_m_new) {
@@ -54,18 +73,26 @@ __device__ __forceinline__ float z_update(float z, float alpha, float row_sum) {
 }
 __device__ __forceinline__ float u_rescale(float u, float alpha) { return __fmul_rn(u, alpha); }
 
-// sum_b A over the 64 lanes of a tile, order fixed by the lane index b alone:
-// four partial sums, partial q takes the lanes with (b mod 8) / 2 == q in
-// ascending b; total = (s0 + s1) + (s2 + s3).
+// sum_b A over the 64 lanes of a tile, order fixed by the lane index b alone.  The tile is
+// taken as two halves of 32 lanes (b < 32, b >= 32).  Within a half: eight chains, chain j
+// takes the lanes with b mod 8 == j in ascending b (four lanes each); pair q = chain 2q +
+// chain 2q+1; half sum = (pair0 + pair1) + (pair2 + pair3).  Tile sum = lower half + upper half.
+// `a` holds the sixteen lanes of one pair over the whole tile: a[2n] = lane 8n + 2q,
+// a[2n+1] = lane 8n + 2q + 1; HALF selects n = 0..3 or n = 4..7.
+template <int HALF>
 __device__ __forceinline__ float quad_partial(const float (&a)[16]) {
-  float s = a[0];
+  float e0 = a[8 * HALF], e1 = a[8 * HALF + 1];
 #pragma unroll
-  for (int i = 1; i < 16; ++i) s = __fadd_rn(s, a[i]);
-  return s;
+  for (int n = 1; n < 4; ++n) {
+    e0 = __fadd_rn(e0, a[8 * HALF + 2 * n]);
+    e1 = __fadd_rn(e1, a[8 * HALF + 2 * n + 1]);
+  }
+  return __fadd_rn(e0, e1);
 }
 __device__ __forceinline__ float quad_total(float s0, float s1, float s2, float s3) {
   return __fadd_rn(__fadd_rn(s0, s1), __fadd_rn(s2, s3));
 }
+__device__ __forceinline__ float tile_total(float lower_half, float upper_half) { return __fadd_rn(lower_half, upper_half); }
 
 // Two lanes at a time.  Each half of a packed f32x2 operation is the same IEEE
 // round-to-nearest operation as its scalar form above, so a kernel may use

@@ -151,16 +151,22 @@ __device__ __forceinline__ void tile_softmax(const float (&s)[8][4], int key0, f
       w_b[2 * n] = w_b[2 * n + 1] = 0.f;
     }
   }
-  float ps_a = nc::quad_partial(w_a);
-  // (s0 + s1) + (s2 + s3): xor 1 pairs quads (0,1) and (2,3), xor 2 joins the pairs.
-  ps_a = __fadd_rn(ps_a, __shfl_xor_sync(kFullMask, ps_a, 1));
-  ps_a = __fadd_rn(ps_a, __shfl_xor_sync(kFullMask, ps_a, 2));
+  // Row sum: per half of the tile, this thread's pair (two chains), then the four pairs of the
+  // row: xor 1 joins pairs (0,1) and (2,3), xor 2 joins those: (P0 + P1) + (P2 + P3); then
+  // lower half + upper half.
+  auto row_sum = [&](const float (&w)[16]) {
+    float lo_h = nc::quad_partial<0>(w), hi_h = nc::quad_partial<1>(w);
+    lo_h = __fadd_rn(lo_h, __shfl_xor_sync(kFullMask, lo_h, 1));
+    hi_h = __fadd_rn(hi_h, __shfl_xor_sync(kFullMask, hi_h, 1));
+    lo_h = __fadd_rn(lo_h, __shfl_xor_sync(kFullMask, lo_h, 2));
+    hi_h = __fadd_rn(hi_h, __shfl_xor_sync(kFullMask, hi_h, 2));
+    return nc::tile_total(lo_h, hi_h);
+  };
+  const float ps_a = row_sum(w_a);
   r.z_a = h_a ? nc::z_update(r.z_a, al_a, ps_a) : r.z_a;
   r.m_a = mn_a;
   if (UPPER) {
-    float ps_b = nc::quad_partial(w_b);
-    ps_b = __fadd_rn(ps_b, __shfl_xor_sync(kFullMask, ps_b, 1));
-    ps_b = __fadd_rn(ps_b, __shfl_xor_sync(kFullMask, ps_b, 2));
+    const float ps_b = row_sum(w_b);
     r.z_b = h_b ? nc::z_update(r.z_b, al_b, ps_b) : r.z_b;
     r.m_b = mn_b;
   }

@@ -520,14 +520,43 @@ void vosti_constants(int32_t* key_tile, int32_t* split_len, int32_t* rows_per_gr
   if (rows_per_group) *rows_per_group = nc::kRowsPerGroup;
 }
 
+// Everything that decides output bits, in a fixed order: the version, the frozen sizes and one
+// id per rule of the numerical contract (nc_math.cuh).  vosti_fingerprint hashes exactly this list.
+static int32_t contract_words(uint32_t* w) {
+  int32_t n = 0;
+  w[n++] = nc::kVersion;
+  w[n++] = nc::kKeyTile;
+  w[n++] = nc::kSplitLen;
+  w[n++] = nc::kRowsPerGroup;
+  w[n++] = nc::kSplitRowsMax;
+  w[n++] = nc::kPageSize;
+  w[n++] = nc::kRuleExponent;
+  w[n++] = nc::kRuleMaximum;
+  float step = nc::kLazyMaxStep;
+  uint32_t step_bits;
+  std::memcpy(&step_bits, &step, sizeof step_bits);
+  w[n++] = step_bits;
+  w[n++] = nc::kRuleRowSum;
+  w[n++] = nc::kRuleFold;
+  w[n++] = nc::kRuleReciprocal;
+  w[n++] = nc::kRuleZeroSign;
+  w[n++] = nc::kRuleMmaChunks;
+  w[n++] = nc::kRuleLse;
+  return n;
+}
+
+int32_t vosti_contract(uint32_t* words, int32_t cap) {
+  uint32_t w[32];
+  const int32_t n = contract_words(w);
+  for (int32_t i = 0; i < n && i < cap && words; ++i) words[i] = w[i];
+  return n;
+}
+
 uint64_t vosti_fingerprint(const vosti_ctx* ctx) {
+  uint32_t w[32];
+  const int32_t n = contract_words(w);
   uint64_t h = 1469598103934665603ull;
-  h = fnv1a(h, nc::kVersion);
-  h = fnv1a(h, nc::kKeyTile);
-  h = fnv1a(h, nc::kSplitLen);
-  h = fnv1a(h, 0x6c656674666f6c64ull);  // left fold by split index
-  h = fnv1a(h, 0x6578322e66746ull);     // ex2.approx.ftz, fused scale-and-shift
-  h = fnv1a(h, 0x6d6d6131363831ull);    // m16n8k16 bf16 chunks of 16, ascending
+  for (int32_t i = 0; i < n; ++i) h = fnv1a(h, w[i]);
   if (ctx) {
     h = fnv1a(h, static_cast<uint64_t>(ctx->cfg.head_dim));
     h = fnv1a(h, static_cast<uint64_t>(ctx->cfg.page_size));
@@ -1459,3 +1488,4 @@ vosti_status vosti_last_schedule(const vosti_ctx* ctx, int64_t* split_items, int
 }
 
 }  // extern "C"
+

@@ -1,12 +1,14 @@
 // vosti_paged_attention_noalloc: split-parallel paged attention for callers that
 // may not allocate memory.
 //
-// Who cannot allocate: code running while a CUDA stream is being captured into
-// a graph (cudaMalloc is not capturable and would break the capture), code
-// inside a serving loop whose memory budget is fixed up front and handed out by
-// an external pool allocator, and plug-ins that are given device pointers by a
-// host framework but no right to create their own.  Such callers cannot build
-// a vosti_ctx either, because vosti_create pins host memory and creates events.
+// Who cannot allocate: a serving engine that has reserved all of the GPU's
+// memory for its KV pool at start-up and hands the rest out through its own
+// pool allocator (a cudaMalloc there fails, or fragments what the engine
+// thinks it owns); a latency-critical decode loop, where cudaMalloc and
+// cudaFree synchronise the whole device and stall every stream; and plug-ins
+// that a host framework gives device pointers but no right to create memory of
+// their own.  Such callers cannot build a vosti_ctx either, because
+// vosti_create pins host memory and creates streams and events.
 //
 // This entry point therefore owns NO heap or device allocation.  Everything it
 // needs beyond the caller's inputs and outputs lives in one file-scope device
@@ -19,6 +21,15 @@
 // The array's name is a host-side stand-in, not a device address: the device
 // address is fetched once per device with cudaGetSymbolAddress and that pointer
 // is what the kernels receive.
+//
+// The per-call metadata (request records, work items, page ids) is planned on
+// the host at call time and copied from a static host buffer with up to four
+// cudaMemcpyAsync calls covering only what the call uses; the source is
+// pageable, so the call also waits for earlier work on the stream.
+//
+// Failure detection: the kernels' bounded waits set the status word at the
+// start of the array, as they do in a context's workspace.  The word is sticky
+// -- calls do not clear it -- and vosti_noalloc_poll_status reads and clears it.
 #include <algorithm>
 #include <cmath>
 #include <cstring>
@@ -38,7 +49,8 @@ constexpr int kMaxTotalQ = 256;
 constexpr int kMaxItems = 1024;    // split-parallel work items
 constexpr int kMaxPageIds = 16384; // page-table entries carried by one call
 // Layout of the scratch array.
-constexpr size_t kOffWords = 0;                    // status, ticket, done (must start at zero)
+constexpr size_t kOffWords = 0;                    // status word (sticky until polled), then ticket and done
+constexpr size_t kOffTicket = 64;                  // ticket at +64, done at +128: zero at every kernel start
 constexpr size_t kOffMeta = 1024;
 constexpr size_t kMetaBytes = sizeof(ReqMeta) * kMaxBatch + sizeof(SplitItem) * kMaxItems +
                               sizeof(int32_t) * kMaxPageIds + sizeof(int2) * kMaxTotalQ;
@@ -206,23 +218,33 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
 
   // ---- upload metadata, clear what must start at zero, launch ------------------------------
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  // The scheduler words keep whatever the last call left; they must be zero at kernel start.
-  if (cudaMemsetAsync(scratch + kOffWords, 0, 1024, stream) != cudaSuccess) return VOSTI_ERR_CUDA;
-  // Pageable source: the runtime stages it before returning, so the static host buffer is free again.
-  if (cudaMemcpyAsync(scratch + kOffMeta, blob, kMetaBytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+  // The scheduler words (ticket, done) keep whatever the last call left; they must be zero at
+  // kernel start.  The status word before them is left alone: it is sticky until polled.
+  if (cudaMemsetAsync(scratch + kOffWords + kOffTicket, 0, 1024 - kOffTicket, stream) != cudaSuccess)
     return VOSTI_ERR_CUDA;
+  // Only what this call uses goes up.  The source is pageable, so each copy returns once the
+  // runtime has staged it (after earlier work on the stream): the static host buffer is then free.
   unsigned char* dmeta = scratch + kOffMeta;
+  const size_t off_items = sizeof(ReqMeta) * kMaxBatch, off_bt = off_items + sizeof(SplitItem) * kMaxItems,
+               off_toks = off_bt + sizeof(int32_t) * kMaxPageIds;
+  if (cudaMemcpyAsync(dmeta, blob, sizeof(ReqMeta) * batch, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+      cudaMemcpyAsync(dmeta + off_items, blob + off_items, sizeof(SplitItem) * n_items, cudaMemcpyHostToDevice,
+                      stream) != cudaSuccess ||
+      cudaMemcpyAsync(dmeta + off_bt, blob + off_bt, sizeof(int32_t) * bt_used, cudaMemcpyHostToDevice, stream) !=
+          cudaSuccess ||
+      cudaMemcpyAsync(dmeta + off_toks, blob + off_toks, sizeof(int2) * n_tok, cudaMemcpyHostToDevice, stream) !=
+          cudaSuccess)
+    return VOSTI_ERR_CUDA;
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.reqs = reinterpret_cast<const ReqMeta*>(dmeta);
   p.items = nullptr;
-  p.split_items = reinterpret_cast<const SplitItem*>(dmeta + sizeof(ReqMeta) * kMaxBatch);
-  p.ticket = reinterpret_cast<uint32_t*>(scratch + kOffWords + 64);
-  p.done = reinterpret_cast<uint32_t*>(scratch + kOffWords + 128);
-  p.bt_flat = reinterpret_cast<const int32_t*>(dmeta + sizeof(ReqMeta) * kMaxBatch + sizeof(SplitItem) * kMaxItems);
-  p.split_tokens = reinterpret_cast<const int2*>(dmeta + sizeof(ReqMeta) * kMaxBatch + sizeof(SplitItem) * kMaxItems +
-                                                 sizeof(int32_t) * kMaxPageIds);
+  p.split_items = reinterpret_cast<const SplitItem*>(dmeta + off_items);
+  p.ticket = reinterpret_cast<uint32_t*>(scratch + kOffWords + kOffTicket);
+  p.done = reinterpret_cast<uint32_t*>(scratch + kOffWords + kOffTicket + 64);
+  p.bt_flat = reinterpret_cast<const int32_t*>(dmeta + off_bt);
+  p.split_tokens = reinterpret_cast<const int2*>(dmeta + off_toks);
   p.ws_u = reinterpret_cast<float*>(scratch + kOffPartU);
   p.ws_mz = reinterpret_cast<float2*>(scratch + kOffPartMz);
   p.ws_uc = nullptr;
@@ -241,4 +263,39 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
   p.tile_rows = nullptr;
   p.packed_rows = nullptr;
   return head_dim == 128 ? launch<128>(map, p, sm_count, stream) : launch<64>(map, p, sm_count, stream);
+}
+
+// Shared by the two status calls: the current device's scratch address (set-up on first use).
+static vosti_status noalloc_scratch_of_current_device(unsigned char** scratch) {
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) return VOSTI_ERR_CUDA;
+  const vosti_status st = setup_device(device);
+  if (st == VOSTI_OK) *scratch = g_scratch_ptr[device];
+  return st;
+}
+
+extern "C" vosti_status vosti_noalloc_poll_status(void* cuda_stream) {
+  std::lock_guard<std::mutex> lock(g_mutex);
+  unsigned char* scratch = nullptr;
+  const vosti_status st = noalloc_scratch_of_current_device(&scratch);
+  if (st != VOSTI_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;  // a stack word: the copy is staged by the runtime, nothing is allocated here
+  if (cudaMemcpyAsync(&word, scratch + kOffWords, sizeof word, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemsetAsync(scratch + kOffWords, 0, sizeof word, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return VOSTI_ERR_CUDA;
+  if (word & kStatusTimeout) return VOSTI_ERR_TIMEOUT;
+  return (word & kStatusBadMetadata) ? VOSTI_ERR_OUT_OF_RANGE : VOSTI_OK;
+}
+
+extern "C" vosti_status vosti_noalloc_selftest_bounded_wait(uint32_t limit_us, void* cuda_stream) {
+  if (limit_us == 0 || limit_us > 100000) return VOSTI_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_mutex);
+  unsigned char* scratch = nullptr;
+  const vosti_status st = noalloc_scratch_of_current_device(&scratch);
+  if (st != VOSTI_OK) return st;
+  bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      reinterpret_cast<uint32_t*>(scratch + kOffWords), static_cast<uint64_t>(limit_us) * 1000ull);
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
 }

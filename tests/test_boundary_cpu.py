@@ -40,9 +40,6 @@ def test_the_attention_library_does_not_contain_the_linear_layer(vb):
     lib = ctypes.CDLL(vb.LIB_PATH)
     assert not hasattr(lib, "vosti_linear") and not hasattr(lib, "vosti_rmsnorm")
     assert not any("linear" in name or "rmsnorm" in name for name in vb.EXPORTS)
-    ignored = open(os.path.join(ROOT, ".gpurunignore.multi")).read().split()
-    assert "paper_2609_38981_b200/csrc/vosti_linear.cu" in ignored
-    assert "paper_2609_38981_b200/libvosti_linear.so" in ignored
 
 
 def test_linear_header_symbols_and_tile_shape(vb):
@@ -191,3 +188,29 @@ def test_items_are_ordered_longest_first(vb):
         return min(it[3] * 8, p // 64 + 1) - it[2] * 8
     t = [tiles(it) for it in items[:n_split]]
     assert t == sorted(t, reverse=True)
+
+
+# The contract words of the committed library and the fingerprint they hash to.  A change of any
+# rule id, frozen size or the lazy-maximum step changes the fingerprint; this test then fails
+# until the version word (first) is raised as well and the pair below is updated together --
+# which is the point: bits may only change under a new version.
+PINNED_CONTRACT = [2, 64, 512, 16, 32, 16, 1, 2, 0x41000000, 3, 1, 1, 1, 1, 1]
+PINNED_FINGERPRINT = 0x0BE65E7990228BE9
+
+
+def test_fingerprint_is_derived_from_the_contract_words(vb):
+    words = vb.vosti_contract()
+    # FNV-1a over the words, eight bytes each (the library's own rule, restated)
+    h = 1469598103934665603
+    for w in words:
+        for i in range(8):
+            h ^= (w >> (8 * i)) & 0xFF
+            h = (h * 1099511628211) % (1 << 64)
+    assert vb.vosti_fingerprint() == h
+    if words != PINNED_CONTRACT:
+        assert words[0] != PINNED_CONTRACT[0], \
+            "a rule or frozen size of the numerical contract changed without a new version"
+        raise AssertionError("contract changed under a new version: update PINNED_CONTRACT / PINNED_FINGERPRINT")
+    assert vb.vosti_fingerprint() == PINNED_FINGERPRINT
+    c = vb.vosti_constants()
+    assert (c["key_tile"], c["split_len"], c["rows_per_group"]) == tuple(words[1:4])
