@@ -215,10 +215,13 @@ vosti_status vosti_paged_attention_ex(vosti_ctx* ctx, const void* q, void* out, 
  *                         own pool and block table (entries of other ranks'
  *                         splits are not read); the slabs of all other splits
  *                         are set to zero;
- *   a sum over ranks   -- of the two workspace ranges this call reports
- *                         (fp32; an all-reduce), which assembles every split's
- *                         partial exactly (x + 0 = x; zeros may change sign,
- *                         which the output rule absorbs);
+ *   an exchange        -- that gives every rank every split's partial rows in
+ *                         the two workspace ranges this call reports: an
+ *                         all-gather of the rows each rank owns (listed by
+ *                         vosti_cp_segments; half the volume of the
+ *                         alternative), or a sum over ranks of the whole
+ *                         ranges (fp32 all-reduce: x + 0 = x; zeros may change
+ *                         sign, which the output rule absorbs);
  *   vosti_cp_combine   -- the left fold over all splits and the output, on any
  *                         rank that wants the result.
  * The fold sees the same partials in the same order as a single-GPU call, so
@@ -236,6 +239,19 @@ vosti_status vosti_cp_partial(vosti_ctx* ctx, const void* q, const int32_t* q_le
 vosti_status vosti_cp_combine(vosti_ctx* ctx, void* out, float* lse, const int32_t* q_lens,
                               const int32_t* start_pos, const int32_t* seq_lens, int32_t batch,
                               void* cuda_stream);
+
+/* The exchange plan of a context-parallel call (host-only, needs no GPU): the
+ * partial rows that rank cp_rank of cp_world writes, as segments (first row,
+ * number of rows) in ascending order; rows index both ranges vosti_cp_partial
+ * reports ([row][head_dim] fp32 and [row] (m, z)).  The segments of all ranks
+ * are disjoint and together cover rows 0 .. *n_partial_rows - 1.  Writes
+ * min(*n_segments, cap) segments as pairs of int64; a first call with cap = 0
+ * sizes the array.  Same premises and errors as vosti_plan; requests with long
+ * queries give UNSUPPORTED_CONFIG. */
+vosti_status vosti_cp_segments(const vosti_config* config, const int32_t* q_lens,
+                               const int32_t* start_pos, const int32_t* seq_lens, int32_t batch,
+                               int32_t cp_rank, int32_t cp_world, int64_t* segments, int64_t cap,
+                               int64_t* n_segments, int64_t* n_partial_rows);
 
 /* One serving step from HOST buffers: copies q, k_new, v_new to the device,
  * runs vosti_kv_append then vosti_paged_attention, copies the output back

@@ -32,7 +32,7 @@ VOSTI_HOST_STEPS_IN_FLIGHT = 3
 EXPORTS = (
     "vosti_workspace_bytes", "vosti_plan", "vosti_plan_ex", "vosti_create", "vosti_destroy", "vosti_kv_append",
     "vosti_paged_attention", "vosti_paged_attention_ex", "vosti_paged_attention_noalloc", "vosti_noalloc_poll_status",
-    "vosti_noalloc_selftest_bounded_wait", "vosti_cp_partial",
+    "vosti_noalloc_selftest_bounded_wait", "vosti_cp_partial", "vosti_cp_segments",
     "vosti_cp_combine", "vosti_step_host", "vosti_step_host_async", "vosti_step_host_wait",
     "vosti_device_plan_bytes", "vosti_plan_device", "vosti_kv_append_planned", "vosti_paged_attention_planned",
     "vosti_poll_device_status",
@@ -91,6 +91,10 @@ _szp = ctypes.POINTER(ctypes.c_size_t)
 _lib.vosti_cp_partial.restype = ctypes.c_int
 _lib.vosti_cp_partial.argtypes = [_vp, _vp, _i32p, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32,
                                   ctypes.c_float, ctypes.c_int32, ctypes.c_int32, _szp, _szp, _szp, _szp, _vp]
+_lib.vosti_cp_segments.restype = ctypes.c_int
+_lib.vosti_cp_segments.argtypes = [_cfgp, _i32p, _i32p, _i32p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                   ctypes.c_void_p, ctypes.c_int64, ctypes.POINTER(ctypes.c_int64),
+                                   ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_cp_combine.restype = ctypes.c_int
 _lib.vosti_cp_combine.argtypes = [_vp, _vp, _vp, _i32p, _i32p, _i32p, ctypes.c_int32, _vp]
 _lib.vosti_paged_attention_noalloc.restype = ctypes.c_int
@@ -246,6 +250,7 @@ class Context:
     def __init__(self, cfg: vosti_config, keep=()):
         self.cfg = cfg
         self._keep = tuple(keep)
+        self.workspace = keep[1] if len(keep) > 1 else None   # the torch tensor behind cfg.workspace
         h = _vp()
         _check(_lib.vosti_create(ctypes.byref(h), ctypes.byref(cfg)), "vosti_create")
         self.handle = h
@@ -335,6 +340,20 @@ def vosti_cp_partial(ctx: Context, q, q_lens, start_pos, seq_lens, block_tables,
     u = ws[v[0].value:v[0].value + v[1].value].view(torch.float32)
     mz = ws[v[2].value:v[2].value + v[3].value].view(torch.float32)
     return u, mz
+
+
+def vosti_cp_segments(cfg: vosti_config, q_lens, start_pos, seq_lens, cp_rank: int, cp_world: int):
+    """Host-only: the partial rows rank cp_rank owns, as an int64 array [n, 2] of (first row,
+    rows), and the total number of partial rows of the call."""
+    ql, s, n = _host_i32(q_lens), _host_i32(start_pos), _host_i32(seq_lens)
+    cnt, rows = ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.vosti_cp_segments(ctypes.byref(cfg), _ip(ql), _ip(s), _ip(n), len(ql), cp_rank, cp_world,
+                                  None, 0, ctypes.byref(cnt), ctypes.byref(rows)), "vosti_cp_segments")
+    seg = np.zeros((max(cnt.value, 1), 2), dtype=np.int64)
+    _check(_lib.vosti_cp_segments(ctypes.byref(cfg), _ip(ql), _ip(s), _ip(n), len(ql), cp_rank, cp_world,
+                                  seg.ctypes.data, cnt.value, ctypes.byref(cnt), ctypes.byref(rows)),
+           "vosti_cp_segments")
+    return seg[:cnt.value], rows.value
 
 
 def vosti_cp_combine(ctx: Context, out, lse, q_lens, start_pos, seq_lens, stream=None) -> None:

@@ -766,6 +766,39 @@ vosti_status vosti_cp_partial(vosti_ctx* ctx, const void* q, const int32_t* q_le
   return VOSTI_OK;
 }
 
+vosti_status vosti_cp_segments(const vosti_config* config, const int32_t* q_lens, const int32_t* start_pos,
+                               const int32_t* seq_lens, int32_t batch, int32_t cp_rank, int32_t cp_world,
+                               int64_t* segments, int64_t cap, int64_t* n_segments, int64_t* n_partial_rows) {
+  if (!config || cap < 0 || (cap > 0 && !segments)) return VOSTI_ERR_INVALID_ARG;
+  if (cp_world < 1 || cp_rank < 0 || cp_rank >= cp_world) return VOSTI_ERR_INVALID_ARG;
+  if (!geometry_ok(*config)) return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  Plan plan;
+  std::vector<int64_t> part_base(static_cast<size_t>(std::max(batch, 0)));
+  const vosti_status st = plan_requests(*config, q_lens, start_pos, seq_lens, batch, 0, &plan, part_base.data());
+  if (st != VOSTI_OK) return st;
+  if (static_cast<int64_t>(plan.items.size()) != plan.n_split) return VOSTI_ERR_UNSUPPORTED_CONFIG;  // long queries
+  const int64_t G = config->n_q_heads / config->n_kv_heads;
+  int64_t n = 0;
+  // The partial rows of request r, KV head h, split k are rows [base, base + rows) with
+  // base = part_base[r] + (h * n_splits + k) * rows; split k belongs to rank k mod world.
+  for (int r = 0; r < batch; ++r) {
+    if (q_lens[r] == 0) continue;
+    const int64_t rows = int64_t{q_lens[r]} * G;
+    const int64_t n_splits = (int64_t{start_pos[r]} + q_lens[r] - 1) / nc::kSplitLen + 1;
+    for (int64_t h = 0; h < config->n_kv_heads; ++h)
+      for (int64_t k = cp_rank; k < n_splits; k += cp_world) {
+        if (n < cap) {
+          segments[2 * n] = part_base[r] + (h * n_splits + k) * rows;
+          segments[2 * n + 1] = rows;
+        }
+        ++n;
+      }
+  }
+  if (n_segments) *n_segments = n;
+  if (n_partial_rows) *n_partial_rows = plan.n_partial_rows;
+  return VOSTI_OK;
+}
+
 vosti_status vosti_cp_combine(vosti_ctx* ctx, void* out, float* lse, const int32_t* q_lens,
                               const int32_t* start_pos, const int32_t* seq_lens, int32_t batch, void* cuda_stream) {
   CpMode cp;

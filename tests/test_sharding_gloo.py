@@ -1,6 +1,6 @@
 """The N > 1 path on CPU: ranks take their own seeded batch (no data-path
 collective), and the only exchange is the max / sum of scalars after the timed
-region.  Run as two gloo ranks."""
+region, through the function bench.py uses for it.  Run as two gloo ranks."""
 import os
 import socket
 
@@ -26,14 +26,13 @@ def _rank_main(rank, world, port, ret):
     sig = torch.tensor([float(sum(w.seq_lens)), float(w.kv_bytes()), float(w.total_q)], dtype=torch.float64)
     gathered = [torch.zeros_like(sig) for _ in range(world)]
     dist.all_gather(gathered, sig)
-    elapsed = torch.tensor([1.0 + rank, 2.0 + rank], dtype=torch.float64)      # stand-in timings
-    dist.all_reduce(elapsed, op=dist.ReduceOp.MAX)
-    total = sig[1:].clone()
-    dist.all_reduce(total, op=dist.ReduceOp.SUM)
+    # the reductions bench.py itself runs after its timed region (same function, gloo instead of NCCL)
+    elapsed = bench.reduce_over_ranks(dist, [1.0 + rank, 2.0 + rank], "max")      # stand-in timings
+    total = bench.reduce_over_ranks(dist, sig[1:].tolist(), "sum")
     if rank == 0:
         ret["gathered"] = [g.tolist() for g in gathered]
-        ret["elapsed"] = elapsed.tolist()
-        ret["total"] = total.tolist()
+        ret["elapsed"] = elapsed
+        ret["total"] = total
     dist.barrier()
     dist.destroy_process_group()
 
