@@ -484,6 +484,7 @@ def run_workload(env, args, name, headline, pack=False, cold_regions=0, min_seco
 
     # host cost of enqueuing a step, measured on an idle queue (nothing to wait for)
     h_us = []
+    vb.vosti_host_time(cache.ctx, reset=True)
     for _ in range(5):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -491,6 +492,7 @@ def run_workload(env, args, name, headline, pack=False, cold_regions=0, min_seco
         step()
         h_us.append((time.perf_counter() - t0) * 1e6 / 2)
     torch.cuda.synchronize()
+    host_ns, _ = vb.vosti_host_time(cache.ctx, reset=True)   # the library's own share (C, without the binding)
 
     tile_bound = name == "mixed_chunked_prefill"     # dominant kernel: the tcgen05 tile kernel
     sampler = ClockSampler(env.local)
@@ -533,7 +535,8 @@ def run_workload(env, args, name, headline, pack=False, cold_regions=0, min_seco
         "pass_ms": {"median": median(pass_ms), "min": min(pass_ms), "max": max(pass_ms)},
         "timed_seconds": sum(pass_ms) / 1e3,
         "ms_per_step_with_kernel_events": median(roof_ms) / args.steps,
-        "host_enqueue_us_per_step": min(h_us), "launches_per_step": launches_per_step,
+        "host_enqueue_us_per_step": min(h_us), "host_library_us_per_step": host_ns / 1e3 / 10,
+        "launches_per_step": launches_per_step,
         "clocks": clocks,
         "schedule": dict(zip(("split_items", "packed_items", "tile_items"), vb.vosti_last_schedule(cache.ctx))),
     }
@@ -847,6 +850,7 @@ def main():
             "tokens_per_s": tok_all / (ms_per_step * 1e-3),
             "pct_of_8TBs": 100.0 * value / env.world / NOMINAL_HBM_GBS,
             "host_enqueue_us_per_step": rec["host_enqueue_us_per_step"],
+            "host_library_us_per_step": rec["host_library_us_per_step"],
             "gpu_launches": int(round(rec["launches_per_step"] * args.steps)),
             "clocks": rec["clocks"],
             "e2e": {"value": bytes_all / (e2e_max * 1e-3) / 1e9, "unit": UNIT,

@@ -427,6 +427,13 @@ vosti_status vosti_profile_read(vosti_ctx* ctx, double* kernel_ms_sum, int64_t* 
 /* Kernels launched through this context since creation. */
 int64_t vosti_launch_count(const vosti_ctx* ctx);
 
+/* Host time (steady clock, nanoseconds) spent inside vosti_kv_append and the
+ * host-planned attention entry points of this context -- validation, planning,
+ * metadata upload, launches -- and the number of such calls, since creation
+ * or the last call with reset != 0.  Measures the library's own host cost
+ * without the binding's.  Either pointer may be NULL. */
+vosti_status vosti_host_time(vosti_ctx* ctx, int64_t* nanoseconds, int64_t* calls, int32_t reset);
+
 /* The schedule of the last attention call of this context: split-parallel work
  * items (16-row packed ones included), how many of them are packed items
  * (shared-split packing, VOSTI_FLAG_PACK_SHARED_SPLITS), and tile items: the

@@ -37,7 +37,7 @@ EXPORTS = (
     "vosti_device_plan_bytes", "vosti_plan_device", "vosti_kv_append_planned", "vosti_paged_attention_planned",
     "vosti_poll_device_status",
     "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
-    "vosti_last_schedule", "vosti_fingerprint", "vosti_contract",
+    "vosti_last_schedule", "vosti_fingerprint", "vosti_contract", "vosti_host_time",
     "vosti_constants", "vosti_status_string",
 )
 
@@ -138,6 +138,8 @@ _lib.vosti_last_schedule.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes
                                      ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_fingerprint.restype = ctypes.c_uint64
 _lib.vosti_fingerprint.argtypes = [_vp]
+_lib.vosti_host_time.restype = ctypes.c_int
+_lib.vosti_host_time.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
 _lib.vosti_contract.restype = ctypes.c_int32
 _lib.vosti_contract.argtypes = [ctypes.POINTER(ctypes.c_uint32), ctypes.c_int32]
 _lib.vosti_constants.restype = None
@@ -158,6 +160,8 @@ def _check(status: int, where: str) -> None:
 
 
 def _host_i32(a) -> np.ndarray:
+    if type(a) is np.ndarray and a.dtype == np.int32 and a.flags.c_contiguous:
+        return a                      # the common case of a serving loop: nothing to convert
     return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
 
 
@@ -235,6 +239,13 @@ def vosti_plan_ex(cfg: vosti_config, q_lens, start_pos, seq_lens, window: int):
 
 def vosti_fingerprint(ctx=None) -> int:
     return int(_lib.vosti_fingerprint(ctx.handle if ctx is not None else None))
+
+
+def vosti_host_time(ctx: "Context", reset: bool = False):
+    """(nanoseconds, calls) the library spent on the host in append / attention calls of ctx."""
+    ns, calls = ctypes.c_int64(), ctypes.c_int64()
+    _check(_lib.vosti_host_time(ctx.handle, ctypes.byref(ns), ctypes.byref(calls), int(reset)), "vosti_host_time")
+    return ns.value, calls.value
 
 
 def vosti_contract():
