@@ -135,3 +135,15 @@ def sampled_parity(w, out_bits, n_samples, seed=0, window=0):
     assert np.isfinite(got).all()
     assert err.max() <= 1e-2 and err.mean() <= 1e-3, (err.max(), err.mean())
     return float(err.max()), float(err.mean())
+
+
+def full_parity(w, out_bits):
+    """Every (request, token, head) output of a workload's call against the oracle's paged
+    front-end (feasible where the query rows are few: decode and speculative batches)."""
+    from oracle import oracle
+    geo = w.geo
+    pool, bt = compact_host_pool(w)
+    ref = oracle.paged_attention(inputs.bits(w.packed_q()), pool, w.q_lens, w.start_pos, w.seq_lens,
+                                 bt, n_kv_heads=geo.n_kv_heads, page_size=geo.page_size,
+                                 scale=geo.head_dim ** -0.5)
+    return assert_parity(out_bits, ref, f"{w.name}: all {out_bits.shape[0] * out_bits.shape[1]} rows vs oracle")

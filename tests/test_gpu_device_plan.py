@@ -111,6 +111,12 @@ def test_decode_and_speculative_steps_equal_the_host_planned_calls(env):
         od, ld = device_step(env, dev, plan, call, env.max_q)
         same(od, oh, f"step {step}, q_lens {ql}")
         assert torch.equal(ld.view(torch.int32), lh.view(torch.int32)), f"step {step}: log-sum-exp differs bitwise"
+        if step < 2:   # and directly against the fp64 oracle (not only against the host-planned GPU path)
+            import gpu_util as gu
+            if not hasattr(env, "oracle"):
+                env.oracle = gu.oracle_rows(env.reqs, env.scale)
+            ref = np.concatenate([env.oracle[i][s:s + n] for i, s, n in call if n > 0])
+            gu.assert_parity(od.cpu().view(torch.int16), ref, f"device-planned step {step} vs oracle")
         assert not (od.view(torch.int16) == 0x7FC1).any()
         done = [d + n for d, n in zip(done, ql)]
     used = sorted({p for t in env.tables for p in t})

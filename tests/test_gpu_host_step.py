@@ -40,6 +40,10 @@ def env():
     c.close()
     for i in want:
         assert (want[i] != 0x7FC2).all()
+    # the device-tensor result every host-buffer variant is compared with is itself within the
+    # stated tolerance of the fp64 oracle
+    for i, ref in enumerate(gu.oracle_rows(reqs, SCALE)):
+        gu.assert_parity(want[i], ref, f"device calls vs oracle, request {i}")
     return dict(reqs=reqs, tables=tables, cache=cache, want=want, gu=gu)
 
 

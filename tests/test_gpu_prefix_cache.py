@@ -111,6 +111,13 @@ def test_reuse_equals_cold_and_shared_pages_are_not_rewritten():
     A = stem
     B = stem[:100] + rng.integers(0, VOCAB, size=70).tolist()
     cold_a, cold_b = cold(A), cold(B)
+    # the cold run everything else is compared with is within the stated tolerance of the fp64 oracle
+    import gpu_util as gu
+    from oracle import oracle
+    rows = model()
+    ref = oracle.attention_dense(inputs.bits(rows("q", A, 0)), inputs.bits(rows("k", A, 0)),
+                                 inputs.bits(rows("v", A, 0)), 0, GEO.head_dim ** -0.5)
+    gu.assert_parity(torch.stack([cold_a[p] for p in range(len(A))]), ref, "cold run vs oracle")
     e = Engine(64)
     assert e.admit(1, A) == 0
     out_a = e.run_to_end(1, 64)
