@@ -414,6 +414,23 @@ vosti_status vosti_poll_device_status(vosti_ctx* ctx, void* cuda_stream);
  * the context stays usable. */
 vosti_status vosti_selftest_bounded_wait(vosti_ctx* ctx, uint32_t limit_us, void* cuda_stream);
 
+/* Self-test of the hardware premises of the numerical contract (the paper's
+ * trusted tile-operation rules, Sec. "Value-Aware Regional Analysis", and the
+ * dot rule of App. A "Backward Regional Dependencies"): computes one small
+ * product twice -- with tcgen05.mma and with mma.sync.m16n8k16, both in
+ * chunks of 16 ascending from a zero accumulator -- and writes both results.
+ *   mode 0 (score form): D[128][64] = A[128][64] . B[64][64]^T
+ *   mode 1 (value form): D[128][64] = W[128][64] . V[64][64], W from tensor memory
+ *   a, b     device bf16, row-major, 16-byte aligned
+ *   d_tc, d_warp   device fp32 [128][64]: the tcgen05 and the warp-MMA result
+ * The caller compares bits (the two kernels of the library agree bit for bit
+ * only if these do), permutes rows of a to check that an output row depends on
+ * its own operand row alone, and zeroes weights to check that a zero weight
+ * contributes exactly nothing.  A bounded wait inside reports through the
+ * device status word. */
+vosti_status vosti_selftest_mma(vosti_ctx* ctx, const void* a, const void* b, int32_t mode, float* d_tc,
+                                float* d_warp, void* cuda_stream);
+
 /* Timing of one kernel of the path with CUDA events recorded on the caller's
  * stream around each of its launches.  mode: 0 stops recording; 1 times the
  * split-parallel attention kernel (the decode hot loop, a3-a7), 2 the

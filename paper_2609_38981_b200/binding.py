@@ -36,7 +36,7 @@ EXPORTS = (
     "vosti_cp_combine", "vosti_step_host", "vosti_step_host_async", "vosti_step_host_wait",
     "vosti_device_plan_bytes", "vosti_plan_device", "vosti_kv_append_planned", "vosti_paged_attention_planned",
     "vosti_poll_device_status",
-    "vosti_selftest_bounded_wait", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
+    "vosti_selftest_bounded_wait", "vosti_selftest_mma", "vosti_profile_enable", "vosti_profile_read", "vosti_launch_count",
     "vosti_last_schedule", "vosti_fingerprint", "vosti_contract", "vosti_host_time",
     "vosti_constants", "vosti_status_string",
 )
@@ -138,6 +138,8 @@ _lib.vosti_last_schedule.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes
                                      ctypes.POINTER(ctypes.c_int64)]
 _lib.vosti_fingerprint.restype = ctypes.c_uint64
 _lib.vosti_fingerprint.argtypes = [_vp]
+_lib.vosti_selftest_mma.restype = ctypes.c_int
+_lib.vosti_selftest_mma.argtypes = [_vp, _vp, _vp, ctypes.c_int32, _vp, _vp, _vp]
 _lib.vosti_host_time.restype = ctypes.c_int
 _lib.vosti_host_time.argtypes = [_vp, ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_int64), ctypes.c_int32]
 _lib.vosti_contract.restype = ctypes.c_int32
@@ -239,6 +241,12 @@ def vosti_plan_ex(cfg: vosti_config, q_lens, start_pos, seq_lens, window: int):
 
 def vosti_fingerprint(ctx=None) -> int:
     return int(_lib.vosti_fingerprint(ctx.handle if ctx is not None else None))
+
+
+def vosti_selftest_mma(ctx: "Context", a, b, mode: int, d_tc, d_warp, stream=None) -> None:
+    """One [128 x 64] product by tcgen05.mma (d_tc) and by mma.sync (d_warp); see include/vosti.h."""
+    _check(_lib.vosti_selftest_mma(ctx.handle, _dev(a), _dev(b), int(mode), _dev(d_tc), _dev(d_warp),
+                                   _stream(stream)), "vosti_selftest_mma")
 
 
 def vosti_host_time(ctx: "Context", reset: bool = False):

@@ -15,7 +15,7 @@ _INC = os.path.join("..", "..", "include")
 TARGETS = {
     LIB: (["vosti.cu", "vosti_noalloc.cu", "prefix_cache.cpp"],
           ["attn_split.cuh", "attn_tile.cuh", "aux_kernels.cuh", "device_plan.cuh", "tile_math.cuh", "meta.cuh",
-           "nc_math.cuh", "ptx.cuh", "tcgen05.cuh", os.path.join(_INC, "vosti.h"), os.path.join(_INC, "vosti_cache.h")]),
+           "nc_math.cuh", "ptx.cuh", "tcgen05.cuh", "selftest_mma.cuh", os.path.join(_INC, "vosti.h"), os.path.join(_INC, "vosti_cache.h")]),
     LIB_LINEAR: (["vosti_linear.cu"],
                  ["ptx.cuh", "tcgen05.cuh", os.path.join(_INC, "vosti.h"), os.path.join(_INC, "vosti_linear.h")]),
 }

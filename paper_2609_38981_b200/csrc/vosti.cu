@@ -13,6 +13,7 @@
 #include "attn_tile.cuh"
 #include "aux_kernels.cuh"
 #include "device_plan.cuh"
+#include "selftest_mma.cuh"
 
 namespace vosti {
 namespace {
@@ -1513,6 +1514,18 @@ vosti_status vosti_selftest_bounded_wait(vosti_ctx* ctx, uint32_t limit_us, void
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status),
                                                    static_cast<uint64_t>(limit_us) * 1000ull);
+  ++ctx->launches;
+  return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
+}
+
+vosti_status vosti_selftest_mma(vosti_ctx* ctx, const void* a, const void* b, int32_t mode, float* d_tc,
+                                float* d_warp, void* cuda_stream) {
+  if (!ctx || !a || !b || !d_tc || !d_warp || (mode != 0 && mode != 1)) return VOSTI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) % 16) return VOSTI_ERR_INVALID_ARG;
+  constexpr int kSmem = 128 * 128 + 64 * 128 + 64 + 1024;
+  mma_selftest_kernel<<<1, 128, kSmem, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const __nv_bfloat16*>(a), static_cast<const __nv_bfloat16*>(b), mode, d_tc, d_warp,
+      reinterpret_cast<uint32_t*>(ctx->ws + ctx->lim.off_status));
   ++ctx->launches;
   return cudaGetLastError() == cudaSuccess ? VOSTI_OK : VOSTI_ERR_CUDA;
 }
