@@ -70,6 +70,15 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
 vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,
                            void* cuda_stream);
 
+/* Hash of everything that decides the bits of vosti_linear and vosti_rmsnorm
+ * (Sec. "A System-Level Formulation": the deployment configuration): the
+ * version, the tile sizes, the segment rule's two constants -- the wave of 148
+ * units is a frozen number, not the SM count of the device in use -- and one
+ * id per reduction rule.  vosti_linear_contract returns those words (their
+ * number; writes min(number, cap)).  Host-only. */
+uint64_t vosti_linear_fingerprint(void);
+int32_t vosti_linear_contract(uint32_t* words, int32_t cap);
+
 /* Waits for `cuda_stream` and reports whether a linear kernel gave up on a
  * bounded wait since the last poll (VOSTI_ERR_TIMEOUT), clearing the word. */
 vosti_status vosti_linear_poll_status(void* cuda_stream);

@@ -28,6 +28,15 @@ struct LinearCfg {
   static constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators: the epilogue of a segment overlaps the next one's MMAs
 };
 
+// Frozen constants of the linear layer's numerics (hashed by vosti_linear_fingerprint).  The
+// wave size is the SM count of a B200 taken as a NUMBER: it decides where segment sums are cut and
+// must not follow the device the library happens to run on.
+constexpr uint32_t kLinearVersion = 1;
+constexpr int kSegmentWaveUnits = 148;      // (column tile, segment) units of one wave
+constexpr int kSegmentMinBlocks = 16;       // a segment holds at least this many 64-wide K blocks (1024 elements)
+constexpr uint32_t kRuleSegmentSum = 1;     // per segment: zero fp32 accumulator, chunks of 16 ascending; sums added left to right
+constexpr uint32_t kRuleRmsNorm = 1;        // lane l adds its 16-byte vectors l, l+32, ... ascending with fma; butterfly; rsqrt.rn
+
 // The K range of a weight is cut into `n_seg` segments of whole 64-wide blocks, a function of
 // (N, K) alone; segment j covers blocks [j * B / n_seg, (j + 1) * B / n_seg).
 struct Segments {
@@ -40,8 +49,8 @@ __host__ __device__ inline Segments segments_of(int64_t N, int64_t K) {
   // as many (column tile, segment) units as fit one wave over the 148 SMs of a B200 when the batch
   // is a single row tile, but segments of at least 1024 elements: every segment costs the
   // large-batch schedule a pass over the accumulator
-  int64_t want = 148 / col_tiles;
-  const int64_t cap = k_blocks / 16 > 0 ? k_blocks / 16 : 1;
+  int64_t want = kSegmentWaveUnits / col_tiles;
+  const int64_t cap = k_blocks / kSegmentMinBlocks > 0 ? k_blocks / kSegmentMinBlocks : 1;
   if (want > cap) want = cap;
   if (want < 1) want = 1;
   return Segments{static_cast<int>(want), k_blocks};
@@ -700,6 +709,27 @@ vosti_status vosti_linear_tile_shape(int64_t N, int64_t K, int32_t* b_m, int32_t
   if (b_n) *b_n = N % 256 == 0 ? 256 : 128;
   if (b_k) *b_k = 64;
   return VOSTI_OK;
+}
+
+int32_t vosti_linear_contract(uint32_t* words, int32_t cap) {
+  const uint32_t w[] = {kLinearVersion, 128u /* B_M */, 256u /* widest B_N */, 128u /* B_N otherwise */, 64u /* B_K */,
+                        static_cast<uint32_t>(kSegmentWaveUnits), static_cast<uint32_t>(kSegmentMinBlocks),
+                        kRuleSegmentSum, kRuleRmsNorm};
+  const int32_t n = static_cast<int32_t>(sizeof w / sizeof w[0]);
+  for (int32_t i = 0; i < n && i < cap && words; ++i) words[i] = w[i];
+  return n;
+}
+
+uint64_t vosti_linear_fingerprint(void) {
+  uint32_t w[16];
+  const int32_t n = vosti_linear_contract(w, 16);
+  uint64_t h = 1469598103934665603ull;
+  for (int32_t i = 0; i < n; ++i)
+    for (int b = 0; b < 8; ++b) {
+      h ^= (static_cast<uint64_t>(w[i]) >> (8 * b)) & 0xff;
+      h *= 1099511628211ull;
+    }
+  return h;
 }
 
 vosti_status vosti_linear_segments(int64_t N, int64_t K, int32_t* n_segments) {

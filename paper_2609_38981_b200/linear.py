@@ -19,7 +19,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 _vp = ctypes.c_void_p
 
 EXPORTS = ("vosti_linear_tile_shape", "vosti_linear_segments", "vosti_linear_workspace_bytes", "vosti_linear",
-           "vosti_rmsnorm", "vosti_linear_poll_status")
+           "vosti_rmsnorm", "vosti_linear_poll_status", "vosti_linear_fingerprint", "vosti_linear_contract")
 
 _lib.vosti_linear_tile_shape.restype = ctypes.c_int
 _lib.vosti_linear_tile_shape.argtypes = [ctypes.c_int64, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -31,6 +31,10 @@ _lib.vosti_linear_workspace_bytes.restype = ctypes.c_size_t
 _lib.vosti_linear_workspace_bytes.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_int64]
 _lib.vosti_rmsnorm.restype = ctypes.c_int
 _lib.vosti_rmsnorm.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_float, _vp]
+_lib.vosti_linear_fingerprint.restype = ctypes.c_uint64
+_lib.vosti_linear_fingerprint.argtypes = []
+_lib.vosti_linear_contract.restype = ctypes.c_int32
+_lib.vosti_linear_contract.argtypes = [ctypes.POINTER(ctypes.c_uint32), ctypes.c_int32]
 _lib.vosti_linear_poll_status.restype = ctypes.c_int
 _lib.vosti_linear_poll_status.argtypes = [_vp]
 
@@ -90,3 +94,13 @@ def vosti_rmsnorm(x: torch.Tensor, weight: torch.Tensor, eps: float, y: torch.Te
 
 def vosti_linear_poll_status(stream=None) -> int:
     return int(_lib.vosti_linear_poll_status(_vb._stream(stream)))
+
+
+def vosti_linear_fingerprint() -> int:
+    return int(_lib.vosti_linear_fingerprint())
+
+
+def vosti_linear_contract():
+    buf = (ctypes.c_uint32 * 16)()
+    n = _lib.vosti_linear_contract(buf, 16)
+    return [int(x) for x in buf[:n]]

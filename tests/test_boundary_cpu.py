@@ -214,3 +214,28 @@ def test_fingerprint_is_derived_from_the_contract_words(vb):
     assert vb.vosti_fingerprint() == PINNED_FINGERPRINT
     c = vb.vosti_constants()
     assert (c["key_tile"], c["split_len"], c["rows_per_group"]) == tuple(words[1:4])
+
+
+PINNED_LINEAR_CONTRACT = [1, 128, 256, 128, 64, 148, 16, 1, 1]
+PINNED_LINEAR_FINGERPRINT = 0xB054C1B6905B3D79
+
+
+def test_linear_fingerprint_is_derived_from_its_contract_words(vb):
+    """The linear layer's identity: tile sizes, the segment rule's constants (the wave of 148 units
+    is a frozen number), one id per reduction rule.  Same discipline as the attention library."""
+    from paper_2609_38981_b200 import linear as vl
+    words = vl.vosti_linear_contract()
+    h = 1469598103934665603
+    for w in words:
+        for i in range(8):
+            h ^= (w >> (8 * i)) & 0xFF
+            h = (h * 1099511628211) % (1 << 64)
+    assert vl.vosti_linear_fingerprint() == h
+    if words != PINNED_LINEAR_CONTRACT:
+        assert words[0] != PINNED_LINEAR_CONTRACT[0], "a linear-layer rule changed without a new version"
+        raise AssertionError("linear contract changed under a new version: update the pinned pair")
+    assert h == PINNED_LINEAR_FINGERPRINT
+    # the segment rule is what the words say: floor(148 / column tiles), segments of >= 16 blocks
+    assert vl.vosti_linear_segments(4096, 4096) == min(148 // (4096 // 256), 4096 // 64 // 16)
+    assert vl.vosti_linear_segments(28672, 4096) == 1
+    assert vl.vosti_linear_segments(4096, 14336) == min(148 // 16, 14336 // 64 // 16)
