@@ -147,3 +147,17 @@ def full_parity(w, out_bits):
                                  bt, n_kv_heads=geo.n_kv_heads, page_size=geo.page_size,
                                  scale=geo.head_dim ** -0.5)
     return assert_parity(out_bits, ref, f"{w.name}: all {out_bits.shape[0] * out_bits.shape[1]} rows vs oracle")
+
+
+def drifting_request(geo, seed, index, n, step=37, jump=0.5, gain=64.0):
+    """A request whose scores climb with the key position: every `step` keys the component of K
+    along a fixed direction grows by `jump`, and every query carries `gain` along that direction,
+    so the scaled score rises by several units of the lazy reference maximum's step inside one
+    split and the reference has to move (alpha != 1, U rescaled) again and again."""
+    r = inputs.make_request(geo, seed, index, n)
+    ramp = (torch.arange(n) // step).to(torch.float32) * jump
+    k = r.k.to(torch.float32)
+    k[:, :, 0] += ramp[:, None]
+    q = r.q.to(torch.float32)
+    q[:, :, 0] += gain
+    return inputs.RequestContent(n=n, q0=0, k=k.to(torch.bfloat16), v=r.v, q=q.to(torch.bfloat16))

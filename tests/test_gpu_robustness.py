@@ -106,3 +106,34 @@ def test_random_schedules_give_the_canonical_bits(seed):
         gu.assert_same_bits(outs[i], canon[i], f"seed {seed} request {i} (context {contexts[i]}, window {window})")
     assert vb.vosti_poll_device_status(c.ctx) == vb.VOSTI_OK
     c.close()
+
+
+@pytest.mark.parametrize("geo", [inputs.Geometry(8, 2, 128, 16), inputs.TINY], ids=["d128_g4", "d64_g2"])
+def test_a_moving_reference_maximum_is_the_same_in_every_schedule(geo):
+    """Scores that climb by more than the lazy reference's step many times inside a split: the
+    reference moves, alpha != 1, U is rescaled -- in the split-parallel kernel's registers and in
+    the tile kernel's tensor memory alike.  Prefill in one call, chunks of 100, and token-by-token
+    decode of the tail must agree bit for bit, and match the oracle."""
+    import gpu_util as gu
+    from paper_2609_38981_b200.harness import DeviceCache
+    scale = geo.head_dim ** -0.5
+    contexts = (700, 1300)
+    reqs = [gu.drifting_request(geo, 31, i, n) for i, n in enumerate(contexts)]
+    tables = inputs._assign_private_pages(inputs.generator(31), geo, 300, contexts)
+
+    def cache():
+        return DeviceCache(geo, 300, max_batch=4, max_total_q=4096, max_seq_len=2048, pool_fill="random")
+    c = cache()
+    full = gu.run_schedule(c, reqs, tables, [[(i, 0, n) for i, n in enumerate(contexts)]], scale)
+    c.close()
+    for i, ref in enumerate(gu.oracle_rows(reqs, scale)):
+        gu.assert_parity(full[i], ref, f"drifting scores, request {i}")
+    c = cache()
+    sched = [[(i, s, min(100, n - s)) for i, n in enumerate(contexts) if s < n - 40] for s in range(0, max(contexts), 100)]
+    sched = [[(i, s, min(q, contexts[i] - 40 - s)) for i, s, q in call if contexts[i] - 40 - s > 0] for call in sched]
+    sched = [call for call in sched if call]
+    sched += [[(i, n - 40 + k, 1) for i, n in enumerate(contexts)] for k in range(40)]     # decode the last 40 tokens
+    mixed = gu.run_schedule(c, reqs, tables, sched, scale)
+    c.close()
+    for i in full:
+        gu.assert_same_bits(mixed[i], full[i], f"drifting scores, request {i}: chunks + decode vs one call")
