@@ -432,9 +432,11 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
         launch_dependent(attn_split_kernel<D, 2>, std::min((p.n_workers + 1) / 2, ctx->sm_count), 64, C2::kSmemBytes,
                          stream, ctx->kv_map3, p);
       } else if (p.n_workers <= 4 * ctx->sm_count ||
-                 (p.n_workers > 8 * ctx->sm_count && p.n_workers <= 14 * ctx->sm_count)) {
-        // (also between one and two rounds of eight workers per SM, where the second round would be
-        // mostly empty: four faster workers per SM balance better -- measured 2-5 % on 32-48 requests)
+                 (p.n_workers > 8 * ctx->sm_count && p.n_workers <= 13 * ctx->sm_count)) {
+        // (also between one and one and a half rounds of eight workers per SM, where the second round
+        // would be mostly empty: four faster workers per SM balance better -- measured 2-5 % on decode
+        // batches of 32-48 requests; beyond 13 tickets per SM -- the packed prefix-sharing batch has
+        // 13.8 -- eight workers are faster again, 59 against 68 us on that batch)
         using C4 = SplitKernelCfg<D, 4>;
         launch_dependent(attn_split_kernel<D, 4>, std::min((p.n_workers + 3) / 4, ctx->sm_count), 128, C4::kSmemBytes,
                          stream, ctx->kv_map3, p);
