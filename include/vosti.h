@@ -78,7 +78,13 @@ enum {
   /* With PACK_SHARED_SPLITS: groups of 48 rows or more always go through the
    * tensor-memory kernel, however little they hold (tests; callers that know
    * their steps are bound by the GPU and not by the host). */
-  VOSTI_FLAG_PACK_THROUGH_TILES = 4
+  VOSTI_FLAG_PACK_THROUGH_TILES = 4,
+  /* A call that launches both the split-parallel kernel (decode and other short
+   * queries) and the tensor-memory tile kernel (prefill chunks, packed tiles)
+   * runs the two side by side on every SM: they read nothing of each other and
+   * are bound by different units.  This flag runs them one after the other
+   * instead (tests compare the two schedules bit for bit; measurements). */
+  VOSTI_FLAG_NO_OVERLAP = 8
 };
 
 /* The fixed deployment configuration (Sec. "Fixed kernel choices": tile

@@ -27,6 +27,7 @@ VOSTI_OK, VOSTI_ERR_INVALID_ARG, VOSTI_ERR_UNSUPPORTED_CONFIG, VOSTI_ERR_OUT_OF_
 VOSTI_FLAG_CHECK_WRITE_SLOTS = 1
 VOSTI_FLAG_PACK_SHARED_SPLITS = 2
 VOSTI_FLAG_PACK_THROUGH_TILES = 4
+VOSTI_FLAG_NO_OVERLAP = 8
 VOSTI_HOST_STEPS_IN_FLIGHT = 3
 
 EXPORTS = (

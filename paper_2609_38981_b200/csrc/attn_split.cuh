@@ -19,26 +19,32 @@ namespace vosti {
 // hides behind the other's); each owns kStages stages of 32 keys (K or V).
 // With few items (a small batch) a CTA runs fewer workers, each with a deeper ring: a worker's
 // speed is then bound by the bytes it keeps in flight, not by its share of the SM.
-template <int D, int WARPS = 8>
+//
+// NARROW (four workers, each with the eight-worker ring): the CTA takes half of an SM's shared
+// memory and registers, so that a CTA of the tensor-memory tile kernel fits beside it.  Used when a
+// tile kernel follows in the same call: the two then run side by side (the split-parallel rows are
+// bound by HBM, the tiles by the tensor pipe and the SFU), see launch_attention().
+template <int D, int WARPS = 8, bool NARROW = false>
 struct SplitKernelCfg {
   static_assert(WARPS == 8 || WARPS == 4 || WARPS == 2, "workers per CTA");
+  static_assert(!NARROW || WARPS == 4, "the narrow variant has four workers");
   static constexpr int kWarps = WARPS;
   // With eight workers a ring of three 32-key stages is what the shared memory allows; with fewer,
   // a stage is a whole 64-key tile (K or V): half as many TMA instructions and barrier probes.
-  static constexpr int kStageKeys = WARPS == 8 ? 32 : 64;
-  static constexpr int kStages = ((D == 128) ? 24 : 48) / WARPS / (kStageKeys / 32);
+  static constexpr int kStageKeys = (WARPS == 8 || NARROW) ? 32 : 64;
+  static constexpr int kStages = NARROW ? 3 : ((D == 128) ? 24 : 48) / WARPS / (kStageKeys / 32);
   static constexpr int kSmemBytes =
       kWarps * kStages * TileCfg<D, kStageKeys>::kStageBytes + kWarps * kStages * 8 + 1024;
 };
 
-template <int D, int WARPS = 8>
+template <int D, int WARPS = 8, bool NARROW = false>
 __global__ void __launch_bounds__(WARPS * 32, 1)
 attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P) {  // kv_map: the 3-D page map
   constexpr bool PM = true;  // stages are page-major: one TMA box per (page, K|V)
-  constexpr int SK = SplitKernelCfg<D, WARPS>::kStageKeys;
+  constexpr int SK = SplitKernelCfg<D, WARPS, NARROW>::kStageKeys;
   using C = TileCfg<D, SK>;
-  constexpr int kWarpsPerCta = SplitKernelCfg<D, WARPS>::kWarps;
-  constexpr int R = SplitKernelCfg<D, WARPS>::kStages;
+  constexpr int kWarpsPerCta = SplitKernelCfg<D, WARPS, NARROW>::kWarps;
+  constexpr int R = SplitKernelCfg<D, WARPS, NARROW>::kStages;
   constexpr int TPS = nc::kTilesPerSplit;
   constexpr int LPT = 2 * C::kParts;  // loads per tile: K parts then V parts
 
@@ -49,7 +55,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t stage0 = base + warp * R * C::kStageBytes;
   const uint32_t bar0 = base + kWarpsPerCta * R * C::kStageBytes + warp * R * 8;
-
   if (lane == 0) {
     tma_prefetch_desc(&kv_map);
 #pragma unroll
@@ -142,6 +147,11 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
   bool has_nxt = true;      // assumed until the second draw says otherwise
   bool drew_second = false;
   griddep_wait();           // the pool (appended tokens) and Q come from earlier work in the stream
+  // The kernel after this one may be scheduled from here on (where an SM has room, or as this
+  // grid's CTAs retire).  What it reads of this kernel's results it reads after its own
+  // griddep_wait(); a tile kernel that reads none of them starts at once, and everything before
+  // this kernel in the stream is complete by then, because every worker has waited for it above.
+  griddep_launch();
 
   // ---- load stream -------------------------------------------------------------
   uint32_t g_issue = 0, g_cons = 0;  // loads issued / consumed since kernel start
@@ -301,7 +311,6 @@ attn_split_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P
       for (int e = 0; e < C::NE; ++e) *reinterpret_cast<float2*>(dst + 8 * e) = make_float2(u[e][2], u[e][3]);
       if (quad == 0) P.ws_mz[out_b] = make_float2(r.m_b, r.z_b);
     }
-
     if (!has_nxt) break;
     cur = nxt;
     --ahead;

@@ -53,7 +53,6 @@
 #include "tile_math.cuh"
 
 namespace vosti {
-
 template <int D>
 struct TileKernelCfg {
   static constexpr int kItemRows = 256;                      // rows of a work item: two CTAs
@@ -184,7 +183,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   }
   // Q tile -> shared memory, [half][row][128 B] with the 128-byte swizzle; padding rows are zero.
   if (warp < 4) {
-    griddep_wait();
+    if (!P.beside_split) griddep_wait();
     const int r = tid;
     const int row = row0 + r;
     bool valid = row < rows;
@@ -254,7 +253,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
     // V producer and issuer on warps 8, 9 and 11 measured 3 % faster than on 8, 10 and 9.
     if (warp == 8 || warp == 9) {
       // ================= TMA producers: warp 8 loads the K tiles, warp 9 the V tiles ========
-      griddep_wait();
+      if (!P.beside_split) griddep_wait();
       const int is_v = warp == 9;
       const int32_t* bt = P.bt_flat + rq.bt_off;
       auto fetch_pages = [&](int split) -> int {
@@ -558,7 +557,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
         float4 uc4[4 * kFoldAhead];
         if (resume) {
 #pragma unroll
-          for (int i = 0; i < 4 * kFoldAhead; ++i) uc4[i] = ucg[static_cast<size_t>(i) * TR];
+          for (int i = 0; i < 4 * kFoldAhead; ++i) uc4[i] = __ldcg(ucg + static_cast<size_t>(i) * TR);
         }
         ok = __all_sync(kFullMask, wait(mz_full + 8 * kb, kuse & 1));
         if (!ok) break;
@@ -600,7 +599,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           if (resume && cb / 16 + kFoldAhead < D / 16) {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              uc4[slot + i] = ucg[static_cast<size_t>((cb / 16 + kFoldAhead) * 4 + i) * TR];
+              uc4[slot + i] = __ldcg(ucg + static_cast<size_t>((cb / 16 + kFoldAhead) * 4 + i) * TR);
           }
           if (last) {
             if (valid) {
@@ -619,7 +618,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
           } else {
 #pragma unroll
             for (int i = 0; i < 4; ++i)
-              ucg[static_cast<size_t>(cb / 4 + i) * TR] = make_float4(un[4 * i], un[4 * i + 1], un[4 * i + 2], un[4 * i + 3]);
+              __stcg(ucg + static_cast<size_t>(cb / 4 + i) * TR, make_float4(un[4 * i], un[4 * i + 1], un[4 * i + 2], un[4 * i + 3]));
           }
         }
       }
@@ -629,6 +628,7 @@ attn_tile_kernel(const __grid_constant__ CUtensorMap kv_map, const AttnParams P)
   // Common exit: every role ends here, also after a timeout, so tensor memory is always released.
   tc_fence_before();
   __syncthreads();
+  if (P.beside_split && tid == 0) griddep_wait();  // this grid is not complete before the one beside it is
   if (warp == 0)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(Cfg::kTmemCols));
 }

@@ -75,6 +75,10 @@ struct AttnParams {
   const int4* tile_pack_items;
   const PackedRow* tile_rows;
   int32_t num_pages;         // device-planned calls: page ids are checked against it when an item is drawn
+  // Tile kernel launched right behind a split-parallel kernel of the same call, whose results it does
+  // not read: it does not wait for that kernel before it starts (the two run side by side) but before
+  // it ends, so that the kernel after it, which waits for this one, has waited for both.
+  int32_t beside_split;
 };
 
 struct AppendParams {

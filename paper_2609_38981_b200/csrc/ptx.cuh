@@ -15,6 +15,9 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 // Blocks until every kernel this grid depends on has completed and its writes
 // are visible.  A no-op when the grid was launched without the attribute.
 __device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel in the stream (launched with programmatic serialization) be scheduled as this
+// grid's CTAs retire; it still waits in its own griddep_wait() until this grid has completed.
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 // ---- mbarrier -------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {

@@ -20,7 +20,7 @@ namespace {
 
 constexpr int kHostSlots = 8;        // ring of pinned staging buffers
 constexpr int kPackedTileRows = 128;  // rows of a packed tile: one CTA of the tile kernel
-constexpr int64_t kTilePackMinRowSplits = 4096;  // rows x splits of such groups from which the extra launch pays
+constexpr int64_t kTilePackMinRowSplits = 2048;  // rows x splits of such groups from which the extra launch pays
 constexpr int kTilePackMinRows = 48;  // rows sharing a split from which packing goes through the tile kernel
 constexpr int kHostSteps = 3;        // host-buffer steps that may be in flight (vosti_step_host_async)
 constexpr size_t kAlign = 1024;
@@ -421,13 +421,31 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
     if (rec) cudaEventRecord(ctx->ev_stop[ctx->ev_used++], stream);
     ++ctx->launches;
   };
+  // A tile kernel that follows a split-parallel kernel reads nothing that kernel writes, and the two
+  // are bound by different things (HBM; tensor pipe and SFU).  They run side by side: the split
+  // kernel in its narrow form, which leaves half of every SM to one CTA of the tile kernel, releases
+  // its successor as soon as its own inputs are complete; the tile kernel starts without waiting
+  // and waits before it ends (AttnParams::beside_split).  Scheduling only: no bits depend on it.
+  // (With event pairs around the kernels they run one after the other, in their usual forms.)
+  const int64_t tile_ctas = (n_seq > 0 ? 2 * n_seq : n_packed_tiles) * Hkv;
+  const bool side_by_side = n_split > 0 && run_partials && !prof && tile_ctas >= ctx->sm_count / 2 &&
+                            !(ctx->cfg.flags & VOSTI_FLAG_NO_OVERLAP);
+  // The narrow form pays when the tile kernel has CTAs for the place beside it for as long as the
+  // split kernel runs (measured: mixed chunked-prefill step 501 -> 485 us narrow, 493 us not); a short
+  // tile kernel rather fills the SMs that the split kernel's CTAs leave (packed prefix-sharing step
+  // 56.8 us narrow, 55.2 us not).
+  const bool narrow = tile_ctas >= 2 * ctx->sm_count;
   if (n_split > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_split * Hkv);
     // persistent: one CTA per SM, warps draw (item, KV head) tickets; with few of them, fewer
     // workers per CTA with deeper rings (scheduling only)
     timed(1, [&] {
-      if (p.n_workers <= 2 * ctx->sm_count) {
+      if (side_by_side && narrow) {
+        using CN = SplitKernelCfg<D, 4, true>;
+        launch_dependent(attn_split_kernel<D, 4, true>, std::min((p.n_workers + 3) / 4, ctx->sm_count), 128,
+                         CN::kSmemBytes, stream, ctx->kv_map3, p);
+      } else if (p.n_workers <= 2 * ctx->sm_count) {
         using C2 = SplitKernelCfg<D, 2>;
         launch_dependent(attn_split_kernel<D, 2>, std::min((p.n_workers + 1) / 2, ctx->sm_count), 64, C2::kSmemBytes,
                          stream, ctx->kv_map3, p);
@@ -449,6 +467,7 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
   if (n_seq > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_seq * Hkv);
+    p.beside_split = side_by_side ? 1 : 0;
     using TileCfg_ = TileKernelCfg<D>;
     timed(2, [&] {
       // two CTAs (128 rows each) per item and KV head
@@ -459,6 +478,7 @@ vosti_status launch_attention(vosti_ctx* ctx, const AttnParams& base, int64_t n_
   if (n_packed_tiles > 0 && run_partials) {
     AttnParams p = base;
     p.n_workers = static_cast<int32_t>(n_packed_tiles * Hkv);
+    p.beside_split = (side_by_side && n_seq == 0) ? 1 : 0;  // behind another tile kernel: the usual wait
     using TileCfg_ = TileKernelCfg<D>;
     timed(2, [&] {
       // one CTA per packed tile (up to 128 rows that share a split) and KV head
@@ -491,7 +511,12 @@ vosti_status set_kernel_attributes() {
       cudaFuncSetAttribute(attn_split_kernel<D, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            SplitKernelCfg<D, 4>::kSmemBytes) != cudaSuccess ||
       cudaFuncSetAttribute(attn_split_kernel<D, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           SplitKernelCfg<D, 2>::kSmemBytes) != cudaSuccess)
+                           SplitKernelCfg<D, 2>::kSmemBytes) != cudaSuccess ||
+      cudaFuncSetAttribute(attn_split_kernel<D, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           SplitKernelCfg<D, 4, true>::kSmemBytes) != cudaSuccess ||
+      // the SM keeps its largest shared-memory partition, so that a tile CTA fits beside this kernel's
+      cudaFuncSetAttribute(attn_split_kernel<D, 4, true>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                           cudaSharedmemCarveoutMaxShared) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_tile_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            TileKernelCfg<D>::kSmemBytes) != cudaSuccess ||
@@ -1201,6 +1226,7 @@ vosti_status attention_impl(vosti_ctx* ctx, const void* q, void* out, float* lse
 
   uint8_t* dmeta = slot->device;
   AttnParams p;
+  p.beside_split = 0;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.reqs = reinterpret_cast<const ReqMeta*>(dmeta + off_reqs);

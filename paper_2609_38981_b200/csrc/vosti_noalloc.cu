@@ -236,6 +236,7 @@ extern "C" vosti_status vosti_paged_attention_noalloc(
           cudaSuccess)
     return VOSTI_ERR_CUDA;
   AttnParams p;
+  p.beside_split = 0;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.reqs = reinterpret_cast<const ReqMeta*>(dmeta);

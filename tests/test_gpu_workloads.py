@@ -11,10 +11,10 @@ from paper_2609_38981_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 
-def make_cache(w, max_total_q=8192, fill="zeros"):
+def make_cache(w, max_total_q=8192, fill="zeros", flags=0):
     from paper_2609_38981_b200.harness import DeviceCache
     return DeviceCache(w.geo, w.num_pages, max_batch=max(w.batch, 8), max_total_q=max_total_q,
-                       max_seq_len=max(w.seq_lens), pool_fill=fill)
+                       max_seq_len=max(w.seq_lens), pool_fill=fill, flags=flags)
 
 
 def run_step(cache, w):
@@ -135,4 +135,11 @@ def test_mixed_chunked_prefill_equals_requests_alone_with_chunk_128():
         q = w.requests[r].q_rows(w.start_pos[r], 1)
         alone = gu.bf16_bits(cache.attend(q, [1], [w.start_pos[r]], [w.seq_lens[r]], bt[r:r + 1], scale))
         assert torch.equal(alone[0], out[row0[r]])
+    cache.close()
+    # The call above ran its two attention kernels side by side (the decodes' split-parallel kernel in
+    # its narrow form beside the chunks' tile kernel); one after the other they give the same bits.
+    from paper_2609_38981_b200 import binding as vb
+    cache = make_cache(w, flags=vb.VOSTI_FLAG_NO_OVERLAP)
+    cache.upload(w.requests, w.tables, upto=w.start_pos)
+    assert torch.equal(run_step(cache, w), out)
     cache.close()
