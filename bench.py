@@ -105,6 +105,30 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+def live_copy_gbs(dev):
+    """This GPU's own device-to-device copy bandwidth (read + write bytes over time, 1 GiB, best of 5),
+    reported beside the roofline's denominator: boxes of the pool differ by a few per cent."""
+    import torch
+    try:
+        n = 1 << 30
+        src = torch.empty(n, dtype=torch.uint8, device=dev)
+        dst = torch.empty_like(src)
+        src.fill_(1)
+        best = None
+        for _ in range(6):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            dst.copy_(src)
+            b.record()
+            b.synchronize()
+            ms = a.elapsed_time(b)
+            best = ms if best is None else min(best, ms)
+        del src, dst
+        return 2.0 * n / (best * 1e-3) / 1e9
+    except Exception:
+        return None
+
+
 def ncu_traffic_per_launch(kernel: str, workload: str):
     """dram bytes per launch of the dominant kernel from the committed ncu summary, if any."""
     path = os.path.join(ROOT, "profiles", f"{kernel}_{workload}.md")
@@ -121,6 +145,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.index, self.samples, self.reasons, self.max_mhz = index, [], set(), None
+        self.mem_samples = []
         self._halt = threading.Event()
         self.ok = False
         try:
@@ -147,6 +172,7 @@ class ClockSampler(threading.Thread):
         while not self._halt.is_set():
             try:
                 self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                self.mem_samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_MEM))
                 try:
                     mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
                 except Exception:
@@ -162,7 +188,8 @@ class ClockSampler(threading.Thread):
         self._halt.set()
         self.join(timeout=2)
         med = sorted(self.samples)[len(self.samples) // 2] if self.samples else None
-        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+        mem = sorted(self.mem_samples)[len(self.mem_samples) // 2] if self.mem_samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "mem_mhz": mem, "reasons": sorted(self.reasons),
                 "samples": len(self.samples)}
 
 
@@ -879,6 +906,12 @@ def main():
                     "output_equals_device_path": out_match},
             "roofline": rec["roofline"],
         }
+        # context for the fraction: what a plain copy reaches on this very GPU, now (not the denominator)
+        live = live_copy_gbs(env.dev)
+        if live is not None and isinstance(line["roofline"], dict):
+            line["roofline"]["this_gpu_copy_gbs_now"] = live
+            if line["roofline"].get("achieved"):
+                line["roofline"]["frac_of_this_gpu_copy"] = line["roofline"]["achieved"] / live
         if not args.no_cpu_baseline:
             # the oracle as it stands on this machine's host cores (rank 0 only, also when N > 1)
             ostep, cores = oracle_step_factory(w)
