@@ -40,13 +40,19 @@
 // and U (D).  The running fold U_c lives in global memory (per CTA a
 // [D/4][128 rows] array of float4, so that a warp's rows are contiguous; touched
 // once per split): there is no room for it on chip.  A correction thread asks
-// for three 16-column chunks of its row's running fold ahead of their use.
-// Measured and not kept (both bitwise correct): copying a finished split out and
+// for three 16-column chunks of its row's running fold ahead of their use, with
+// cache-global loads and stores (the array is streamed; L1 would only be churned).
+// When this kernel is launched right behind a split-parallel kernel of the same
+// call it starts without waiting for it and waits before it ends instead
+// (AttnParams::beside_split): the two kernels then share the SMs.
+// Measured and not kept (all bitwise correct): copying a finished split out and
 // folding it behind the next split's tiles doubles the traffic through the SM's
 // load/store path and is slower; dividing a row's key columns between two
 // threads (two symmetric warpgroups that exchange half-row maxima and sums
 // through shared memory) makes the hand-over part of every tile's chain and is
-// slower too.
+// slower too; so is keeping the first 16 to 48 columns of the running fold in the
+// correction thread's registers (it has none to spare: the spills cost more than
+// the traffic saved).
 #pragma once
 #include "meta.cuh"
 #include "tcgen05.cuh"
