@@ -1,5 +1,6 @@
 // Split-parallel attention (decode, speculative and other short queries): a
-// persistent kernel, one CTA per SM, four independent warp workers per CTA.
+// persistent kernel, one CTA per SM, eight (or four, or two) independent warp
+// workers per CTA.
 //
 // A worker draws (item, KV head) tickets from a global counter.  An item is one
 // KV split (512 keys) of one 16-row group of a request; the worker walks its
