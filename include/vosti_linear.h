@@ -54,13 +54,32 @@ size_t vosti_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
 /* y [M, N] = x [M, K] * w [N, K]^T (one weight row per output feature, as a
  * linear layer stores it).  M >= 0 is free; M = 0 does nothing.
  * workspace: device memory, 16-byte aligned, or NULL.  With at least
- * vosti_linear_workspace_bytes(M, N, K) bytes the call may use the split
- * schedule; without, it always walks whole tiles.  The output bits are the same
- * either way.
+ * vosti_linear_workspace_bytes(M, N, K) bytes the call may spread the K
+ * segments of a tile over CTAs also where a tile has more than eight segments
+ * (see vosti_linear_ex).  The output bits are the same whichever schedule runs.
  * Errors: INVALID_ARG (null or misaligned pointers, negative M),
  * UNSUPPORTED_CONFIG (see vosti_linear_tile_shape), CUDA. */
 vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
                           void* workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* The same with the schedule named by the caller (tests compare them bit for
+ * bit; measurements).  vosti_linear picks one by itself, VOSTI_LINEAR_AUTO:
+ * with few row tiles the K segments of a tile are spread over CTAs -- in
+ * clusters that add the segment sums out of each other's shared memory when a
+ * tile has two to eight segments, else through the workspace if one is given;
+ * with many row tiles CTA pairs (B_N = 256, large M) or single CTAs walk whole
+ * tiles.  A schedule that does not apply to the shape (SPLIT_CLUSTER with one
+ * or more than eight segments, SPLIT_WORKSPACE with one segment or without the
+ * workspace, PAIRS with B_N = 128) returns UNSUPPORTED_CONFIG. */
+enum {
+  VOSTI_LINEAR_AUTO = 0,
+  VOSTI_LINEAR_WHOLE_TILES = 1,
+  VOSTI_LINEAR_SPLIT_WORKSPACE = 2,
+  VOSTI_LINEAR_SPLIT_CLUSTER = 3,
+  VOSTI_LINEAR_PAIRS = 4
+};
+vosti_status vosti_linear_ex(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
+                             void* workspace, size_t workspace_bytes, int32_t schedule, void* cuda_stream);
 
 /* y [M, K] = x * rsqrt(mean_k(x^2) + eps) * weight [K], per row: the sum of
  * squares is taken in a fixed order that depends on K only (each lane of the

@@ -73,6 +73,32 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int m_tiles, int n_cols) 
   return TileCoord{(first_m + in_band % rows) * BM, (in_band / rows) * BN};
 }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// The address, in the cluster's shared window, of `addr` in the CTA of rank `rank`.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t cluster_addr) {
+  float4 v;
+  // (ordered against the cluster barriers around its use by their own memory clobbers)
+  asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+               : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+               : "r"(cluster_addr));
+  return v;
+}
+
 // The numerical contract of an output element: for each segment of K a sum s_j that starts from
 // a zero fp32 accumulator and takes the products in ascending K order (tcgen05.mma, K = 16 per
 // instruction); then t = s_0, t = t + s_j for j = 1, 2, ... in fp32, round to nearest; then
@@ -83,14 +109,23 @@ __device__ __forceinline__ TileCoord tile_coord(int t, int m_tiles, int n_cols) 
 //   SPLIT = true (few row tiles, e.g. a decode batch): the unit of work is a (tile, segment)
 //     pair, so that every SM streams a slice of the weight; s_j goes to a workspace and
 //     linear_fold_kernel adds the segments in the same order.
+//   SPLIT and CLUSTER (the same units, when a tile's segments number at most eight): the CTAs that
+//     hold the segments of one tile form a cluster; each leaves its s_j in its own shared memory,
+//     and after a cluster barrier CTA j adds, for its share of the tile's columns, s_0, s_1, ... in
+//     that order out of the peers' shared memory and writes the bf16 result.  No workspace, no
+//     second kernel, and the segment sums never travel through L2.
 // Which one runs is a scheduling decision that may depend on M; the bits do not.
-template <int BN, bool SPLIT>
+template <int BN, bool SPLIT, bool CLUSTER = false>
 __global__ void __launch_bounds__(LinearCfg<BN>::kThreads, 1)
 linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap w_map,
               __nv_bfloat16* __restrict__ y, float* __restrict__ seg_ws, int M, int N, int K) {
   using Cfg = LinearCfg<BN>;
   constexpr int NS = Cfg::kStages;
   constexpr uint32_t kAbortAfterNs = 1000000000u;
+  // CLUSTER: a row of the CTA's segment sum in shared memory; the 16 bytes beyond BN floats keep
+  // 16-byte accesses of consecutive rows on different banks
+  constexpr uint32_t kPartRow = BN * 4 + 16;
+  static_assert(!CLUSTER || 128 * kPartRow <= static_cast<uint32_t>(NS * Cfg::kStageBytes), "segment sum fits the stages");
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
@@ -232,7 +267,22 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         const bool in_range = tc.m0 + r < M;
-        if (SPLIT) {
+        if constexpr (SPLIT && CLUSTER) {
+          // s_j of this unit -> this CTA's shared memory, [row][BN] fp32 with rows kPartRow bytes apart
+          // (the pipeline stages are idle: the unit's MMAs are done, and the CTA has no other unit)
+          const uint32_t dst = base + r * kPartRow + c0 * 4;
+#pragma unroll 1
+          for (int cb = 0; cb < 128; cb += 32) {
+            uint32_t v[32];
+            tmem_ld32(tmem + lane_sel + buf * BN + c0 + cb, v);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+              asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst + (cb + i) * 4), "r"(v[i]), "r"(v[i + 1]),
+                           "r"(v[i + 2]), "r"(v[i + 3])
+                           : "memory");
+          }
+        } else if (SPLIT) {
           // s_j of this unit -> workspace [column tile][segment][row][BN]
           float* dst = seg_ws + ((static_cast<size_t>(tc.n0 / BN) * seg.n_seg + sj) * M + (tc.m0 + r)) * BN + c0;
 #pragma unroll 1
@@ -286,6 +336,57 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
     }
   }
 
+  if constexpr (SPLIT && CLUSTER) {
+    // Every thread of the cluster gets here, also after a wait has given up.  First barrier: the
+    // segment sums of the tile are in the shared memory of the CTAs that computed them.
+    cluster_sync_all();
+    if (warp >= 2) {
+      const int n = seg.n_seg;                       // = CTAs of the cluster; this CTA's rank = its segment
+      const int j = static_cast<int>(cluster_ctarank());
+      const int g_lo = j * (BN / 8) / n, g_hi = (j + 1) * (BN / 8) / n;  // this CTA's groups of eight columns
+      const int cpr = 2 * (g_hi - g_lo);             // 16-byte chunks (four columns) per row of its share
+      int tile, sj;
+      step_of(blockIdx.x, 0, tile, sj);
+      const TileCoord tc = tile_coord<Cfg::kBM, BN>(tile, m_tiles, n_cols);
+      // Consecutive threads take consecutive chunks of a row: a warp's request to a peer's shared
+      // memory is one contiguous piece (scattered 16-byte requests crawl), and so is its store.
+      constexpr int kStride = 32 * Cfg::kEpiWarps, kBatch = 1;  // (more chunks in flight per thread measured slower)
+      for (int idx0 = tid - 64; idx0 < Cfg::kBM * cpr; idx0 += kBatch * kStride) {
+        float4 a[kBatch][8];  // every value is requested before the first is used
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int idx = idx0 + u * kStride;
+          if (idx < Cfg::kBM * cpr) {
+            const int row = idx / cpr, ch = idx - row * cpr;
+            const uint32_t local = base + row * kPartRow + g_lo * 32 + ch * 16;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              if (q < n) a[u][q] = ld_cluster_f4(map_to_cta(local, static_cast<uint32_t>(q)));
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+          const int idx = idx0 + u * kStride;
+          if (idx < Cfg::kBM * cpr) {
+            const int row = idx / cpr, ch = idx - row * cpr;
+            float4 t = a[u][0];
+#pragma unroll
+            for (int q = 1; q < 8; ++q)  // t = s_0, then t + s_1, ... : the contract's order
+              if (q < n) {
+                t.x = __fadd_rn(t.x, a[u][q].x); t.y = __fadd_rn(t.y, a[u][q].y);
+                t.z = __fadd_rn(t.z, a[u][q].z); t.w = __fadd_rn(t.w, a[u][q].w);
+              }
+            if (tc.m0 + row < M) {
+              __nv_bfloat162 lo2 = __floats2bfloat162_rn(t.x, t.y), hi2 = __floats2bfloat162_rn(t.z, t.w);
+              *reinterpret_cast<uint2*>(y + static_cast<size_t>(tc.m0 + row) * N + tc.n0 + g_lo * 8 + ch * 4) =
+                  make_uint2(*reinterpret_cast<uint32_t*>(&lo2), *reinterpret_cast<uint32_t*>(&hi2));
+            }
+          }
+        }
+      }
+    }
+    cluster_sync_all();  // nobody reads this CTA's shared memory any more
+  }
   tc_fence_before();
   __syncthreads();
   if (warp == 1)
@@ -312,23 +413,6 @@ struct PairCfg {
   static constexpr uint32_t kTmemCols = 2 * kBN;
 };
 
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// The address, in the cluster's shared window, of `addr` in the CTA of rank `rank`.
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
 // TMA load into this CTA's shared memory whose bytes are counted on the leader CTA's mbarrier.
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int32_t x, int32_t y,
                                                  uint32_t leader_bar) {
@@ -623,10 +707,24 @@ size_t split_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   return sizeof(float) * static_cast<size_t>(segments_of(N, K).n_seg) * M * N;
 }
 
+// Whether spreading the segments over CTAs through the workspace is expected to beat whole tiles:
+// rounds of K blocks on the busiest SM, plus what the segment sums cost on their way through the
+// workspace and back, in units of the time of one 64-wide K block of a tile (about 0.4 us; the sums
+// cost about one block time per 190,000 of their elements, fitted to the measurements below).  Measured on the Llama-3.1-8B
+// shapes: 6144 x 4096 at 384 rows 32 us split, 29 us whole; 4096 x 14336 at 256 rows 46 us split,
+// 93 us whole.  Scheduling only.
+inline bool split_pays(int64_t M, int64_t N, int64_t tiles, const Segments& seg, int sm_count) {
+  auto rounds = [&](int64_t units) { return (units + sm_count - 1) / sm_count; };
+  const int64_t per_seg = (seg.k_blocks + seg.n_seg - 1) / seg.n_seg;
+  const int64_t whole = rounds(tiles) * seg.k_blocks;
+  const int64_t split = rounds(tiles * seg.n_seg) * per_seg + M * N * seg.n_seg / 190000;
+  return split < whole;
+}
+
 template <int BN>
 vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K,
                            void* workspace, size_t workspace_bytes, int sm_count, cudaStream_t stream,
-                           bool use_pairs = false) {
+                           int schedule, bool use_pairs = false) {
   using Cfg = LinearCfg<BN>;
   static bool attr_set[64] = {};
   int dev = 0;
@@ -635,6 +733,8 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
     if (cudaFuncSetAttribute(linear_kernel<BN, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(linear_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(linear_kernel<BN, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg::kSmemBytes) != cudaSuccess)
       return VOSTI_ERR_CUDA;
     attr_set[dev] = true;
@@ -643,16 +743,54 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
   if (!make_map(fn, &x_map, x, M, K, Cfg::kBM) || !make_map(fn, &w_map, w, N, K, BN)) return VOSTI_ERR_CUDA;
   const int64_t tiles = ((M + Cfg::kBM - 1) / Cfg::kBM) * (N / BN);
   const Segments seg = segments_of(N, K);
-  // Scheduling only: split the segments over CTAs when whole tiles would leave most SMs idle
-  // and the caller has provided room for the segment sums.
-  const bool split = seg.n_seg > 1 && tiles * 2 <= sm_count && workspace != nullptr &&
-                     workspace_bytes >= split_workspace_bytes(M, N, K) &&
-                     reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
   __nv_bfloat16* yb = static_cast<__nv_bfloat16*>(y);
+  // Scheduling only.  Few row tiles (whole tiles would leave most SMs idle): the segments of a tile
+  // are spread over CTAs -- in clusters that add the segment sums themselves when a tile has at most
+  // eight segments (the portable cluster size), else through the caller's workspace if there is one.
+  // Many row tiles: CTA pairs when the caller's estimate favours them, else single CTAs.
+  const bool few = tiles * 2 <= sm_count;
+  const bool ws_ok = workspace != nullptr && workspace_bytes >= split_workspace_bytes(M, N, K) &&
+                     reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
+  const bool cluster_ok = seg.n_seg > 1 && seg.n_seg <= 8;
+  const bool pairs_ok = BN == 256 && sm_count >= 2;
+  int sched = schedule;
+  if (sched == VOSTI_LINEAR_AUTO) {
+    // (clusters only when all of them fit the SMs at once: a second round of one-unit CTAs costs
+    // more than the persistent workspace route's second round)
+    if (few && cluster_ok && tiles * seg.n_seg <= (sm_count / seg.n_seg) * seg.n_seg) sched = VOSTI_LINEAR_SPLIT_CLUSTER;
+    else if (seg.n_seg > 1 && ws_ok && split_pays(M, N, tiles, seg, sm_count)) sched = VOSTI_LINEAR_SPLIT_WORKSPACE;
+    else if (pairs_ok && use_pairs) sched = VOSTI_LINEAR_PAIRS;
+    else sched = VOSTI_LINEAR_WHOLE_TILES;
+  } else if ((sched == VOSTI_LINEAR_SPLIT_CLUSTER && !cluster_ok) ||
+             (sched == VOSTI_LINEAR_SPLIT_WORKSPACE && !(seg.n_seg > 1 && ws_ok)) ||
+             (sched == VOSTI_LINEAR_PAIRS && !pairs_ok)) {
+    return VOSTI_ERR_UNSUPPORTED_CONFIG;
+  }
+  if (sched == VOSTI_LINEAR_SPLIT_CLUSTER) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(tiles * seg.n_seg));  // one cluster per tile, one CTA per segment
+    cfg.blockDim = dim3(Cfg::kThreads);
+    cfg.dynamicSmemBytes = Cfg::kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(seg.n_seg);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, linear_kernel<BN, true, true>, x_map, w_map, yb, static_cast<float*>(nullptr),
+                           static_cast<int>(M), static_cast<int>(N), static_cast<int>(K)) == cudaSuccess)
+      return VOSTI_OK;
+    (void)cudaGetLastError();
+    if (schedule != VOSTI_LINEAR_AUTO) return VOSTI_ERR_CUDA;
+    // such clusters cannot be placed on this device: the other routes remain
+    sched = (seg.n_seg > 1 && ws_ok) ? VOSTI_LINEAR_SPLIT_WORKSPACE : VOSTI_LINEAR_WHOLE_TILES;
+  }
+  const bool split = sched == VOSTI_LINEAR_SPLIT_WORKSPACE;
   if constexpr (BN == 256) {
-    // CTA pairs (less operand traffic per SM, deeper pipeline) when the caller's estimate favours them.
     const int n_pairs = sm_count / 2;
-    if (!split && n_pairs > 0 && use_pairs) {
+    if (sched == VOSTI_LINEAR_PAIRS) {
       static bool pair_attr_set[64] = {};
       if (!pair_attr_set[dev]) {
         if (cudaFuncSetAttribute(linear_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -748,6 +886,12 @@ size_t vosti_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
 
 vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* workspace,
                           size_t workspace_bytes, void* cuda_stream) {
+  return vosti_linear_ex(x, w, y, M, N, K, workspace, workspace_bytes, VOSTI_LINEAR_AUTO, cuda_stream);
+}
+
+vosti_status vosti_linear_ex(const void* x, const void* w, void* y, int64_t M, int64_t N, int64_t K, void* workspace,
+                             size_t workspace_bytes, int32_t schedule, void* cuda_stream) {
+  if (schedule < VOSTI_LINEAR_AUTO || schedule > VOSTI_LINEAR_PAIRS) return VOSTI_ERR_INVALID_ARG;
   int32_t bn = 0;
   const vosti_status shape = vosti_linear_tile_shape(N, K, nullptr, &bn, nullptr);
   if (shape != VOSTI_OK) return shape;
@@ -770,7 +914,8 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
       cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
     return VOSTI_ERR_CUDA;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (bn != 256) return launch_linear<128>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream);
+  if (bn != 256)
+    return launch_linear<128>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream, schedule);
   // Scheduling only (the bits are the same either way): CTA pairs when there is more than one
   // row tile, the pairs have at least three rounds of 256 x 256 tiles (below that a round of
   // single CTAs is measured to be as fast or faster), and their rounds, a little cheaper each,
@@ -780,7 +925,7 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
   const int64_t r_single = rounds(m128 * (N / 256), sm_count);
   const int64_t r_pair = sm_count >= 2 ? rounds(m256 * (N / 256), sm_count / 2) : 0;
   const bool use_pairs = M > 128 && r_pair >= 3 && 0.93 * static_cast<double>(r_pair) <= static_cast<double>(r_single);
-  return launch_linear<256>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream, use_pairs);
+  return launch_linear<256>(fn, x, w, y, M, N, K, workspace, workspace_bytes, sm_count, stream, schedule, use_pairs);
 }
 
 vosti_status vosti_rmsnorm(const void* x, const void* weight, void* y, int64_t M, int64_t K, float eps,

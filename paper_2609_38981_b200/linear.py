@@ -19,12 +19,15 @@ _lib = ctypes.CDLL(LIB_PATH)
 _vp = ctypes.c_void_p
 
 EXPORTS = ("vosti_linear_tile_shape", "vosti_linear_segments", "vosti_linear_workspace_bytes", "vosti_linear",
-           "vosti_rmsnorm", "vosti_linear_poll_status", "vosti_linear_fingerprint", "vosti_linear_contract")
+           "vosti_linear_ex", "vosti_rmsnorm", "vosti_linear_poll_status", "vosti_linear_fingerprint", "vosti_linear_contract")
 
 _lib.vosti_linear_tile_shape.restype = ctypes.c_int
 _lib.vosti_linear_tile_shape.argtypes = [ctypes.c_int64, ctypes.c_int64] + [ctypes.POINTER(ctypes.c_int32)] * 3
 _lib.vosti_linear.restype = ctypes.c_int
 _lib.vosti_linear.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp, ctypes.c_size_t, _vp]
+_lib.vosti_linear_ex.restype = ctypes.c_int
+_lib.vosti_linear_ex.argtypes = [_vp, _vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64, _vp, ctypes.c_size_t,
+                                 ctypes.c_int32, _vp]
 _lib.vosti_linear_segments.restype = ctypes.c_int
 _lib.vosti_linear_segments.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.POINTER(ctypes.c_int32)]
 _lib.vosti_linear_workspace_bytes.restype = ctypes.c_size_t
@@ -62,10 +65,18 @@ def _bf16_cuda(t: torch.Tensor, ndim: int) -> torch.Tensor:
     return t
 
 
+VOSTI_LINEAR_AUTO = 0
+VOSTI_LINEAR_WHOLE_TILES = 1
+VOSTI_LINEAR_SPLIT_WORKSPACE = 2
+VOSTI_LINEAR_SPLIT_CLUSTER = 3
+VOSTI_LINEAR_PAIRS = 4
+
+
 def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, workspace: torch.Tensor = None,
-                 stream=None) -> torch.Tensor:
+                 stream=None, schedule: int = VOSTI_LINEAR_AUTO) -> torch.Tensor:
     """y [M, N] = x [M, K] @ w [N, K]^T; tensors are CUDA bf16, contiguous.  workspace: an optional
-    CUDA byte tensor (see vosti_linear_workspace_bytes) that allows the split schedule for small M."""
+    CUDA byte tensor (see vosti_linear_workspace_bytes) for the split schedule that needs one.
+    schedule: VOSTI_LINEAR_AUTO, or one of the schedules by name (vosti_linear_ex)."""
     x, w = _bf16_cuda(x, 2), _bf16_cuda(w, 2)
     M, K = x.shape
     N = w.shape[0]
@@ -75,8 +86,12 @@ def vosti_linear(x: torch.Tensor, w: torch.Tensor, y: torch.Tensor = None, works
     _bf16_cuda(y, 2)
     assert y.shape == (M, N)
     ws_ptr, ws_bytes = (0, 0) if workspace is None else (workspace.data_ptr(), workspace.numel() * workspace.element_size())
-    _vb._check(_lib.vosti_linear(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, ws_ptr, ws_bytes,
-                                 _vb._stream(stream)), "vosti_linear")
+    if schedule == VOSTI_LINEAR_AUTO:
+        _vb._check(_lib.vosti_linear(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, ws_ptr, ws_bytes,
+                                     _vb._stream(stream)), "vosti_linear")
+    else:
+        _vb._check(_lib.vosti_linear_ex(_vb._dev(x), _vb._dev(w), _vb._dev(y), M, N, K, ws_ptr, ws_bytes,
+                                        int(schedule), _vb._stream(stream)), "vosti_linear_ex")
     return y
 
 

@@ -79,6 +79,38 @@ def test_row_level_contract(N, K):
         assert torch.equal(y[inv[i]], single[j]), (N, K, "permuted", i)
 
 
+@pytest.mark.parametrize("N,K,n_seg", [(1024, 4096, 4), (512, 2048, 2), (256, 8192, 8), (256, 6144, 6),
+                                       (128, 3072, 3), (256, 9216, 9), (768, 1024, 1)])
+def test_every_schedule_gives_the_same_bits(N, K, n_seg):
+    """The K segments of a tile computed by one CTA in turn (whole tiles), by one CTA each with the
+    sums added from a workspace by a second kernel, or by the CTAs of a cluster that add the sums out
+    of each other's shared memory (2 to 8 segments: a power of two, 6 and 3, whose column shares are
+    uneven): same bits, for a single row, ragged and several row tiles.  A schedule that does not apply
+    is refused."""
+    from paper_2609_38981_b200 import binding as vb
+    from paper_2609_38981_b200 import linear as vl
+    from paper_2609_38981_b200.harness import bf16_bits
+    assert vl.vosti_linear_segments(N, K) == n_seg
+    x, w = data(N, K, 300, 21)
+    xd, wd = x.cuda(), w.cuda()
+    for M in (1, 5, 128, 200, 300):
+        xm = xd[:M].contiguous()
+        whole = bf16_bits(vl.vosti_linear(xm, wd, schedule=vl.VOSTI_LINEAR_WHOLE_TILES))
+        assert torch.equal(bf16_bits(vl.vosti_linear(xm, wd, workspace=workspace(M, N, K))), whole), (M, "auto")
+        assert torch.equal(bf16_bits(vl.vosti_linear(xm, wd)), whole), (M, "auto, no workspace")
+        if n_seg > 1:
+            y = vl.vosti_linear(xm, wd, workspace=workspace(M, N, K), schedule=vl.VOSTI_LINEAR_SPLIT_WORKSPACE)
+            assert torch.equal(bf16_bits(y), whole), (M, "workspace")
+        if 2 <= n_seg <= 8:
+            y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+            vl.vosti_linear(xm, wd, y, schedule=vl.VOSTI_LINEAR_SPLIT_CLUSTER)
+            assert torch.equal(bf16_bits(y), whole), (M, "cluster")
+        else:
+            with pytest.raises(vb.VostiError):
+                vl.vosti_linear(xm, wd, schedule=vl.VOSTI_LINEAR_SPLIT_CLUSTER)
+    assert vl.vosti_linear_poll_status() == 0
+
+
 def test_tile_shape_and_segments_are_functions_of_the_weight_only():
     from paper_2609_38981_b200 import linear as vl
     assert vl.vosti_linear_tile_shape(4096, 4096) == (128, 256, 64)
