@@ -66,10 +66,11 @@ vosti_status vosti_linear(const void* x, const void* w, void* y, int64_t M, int6
  * bit; measurements).  vosti_linear picks one by itself, VOSTI_LINEAR_AUTO:
  * with few row tiles the K segments of a tile are spread over CTAs -- in
  * clusters that add the segment sums out of each other's shared memory when a
- * tile has two to eight segments, else through the workspace if one is given;
+ * tile has two to eight segments (by name: up to sixteen, clusters beyond the
+ * portable size), else through the workspace if one is given;
  * with many row tiles CTA pairs (B_N = 256, large M) or single CTAs walk whole
  * tiles.  A schedule that does not apply to the shape (SPLIT_CLUSTER with one
- * or more than eight segments, SPLIT_WORKSPACE with one segment or without the
+ * or more than sixteen segments, SPLIT_WORKSPACE with one segment or without the
  * workspace, PAIRS with B_N = 128) returns UNSUPPORTED_CONFIG. */
 enum {
   VOSTI_LINEAR_AUTO = 0,

@@ -35,6 +35,7 @@ constexpr uint32_t kLinearVersion = 1;
 constexpr int kSegmentWaveUnits = 148;      // (column tile, segment) units of one wave
 constexpr int kSegmentMinBlocks = 16;       // a segment holds at least this many 64-wide K blocks (1024 elements)
 constexpr uint32_t kRuleSegmentSum = 1;     // per segment: zero fp32 accumulator, chunks of 16 ascending; sums added left to right
+constexpr int kMaxClusterSegments = 16;      // segments of a tile that a cluster can add (scheduling only)
 constexpr uint32_t kRuleRmsNorm = 1;        // lane l adds its 16-byte vectors l, l+32, ... ascending with fma; butterfly; rsqrt.rn
 
 // The K range of a weight is cut into `n_seg` segments of whole 64-wide blocks, a function of
@@ -352,7 +353,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
       // memory is one contiguous piece (scattered 16-byte requests crawl), and so is its store.
       constexpr int kStride = 32 * Cfg::kEpiWarps, kBatch = 1;  // (more chunks in flight per thread measured slower)
       for (int idx0 = tid - 64; idx0 < Cfg::kBM * cpr; idx0 += kBatch * kStride) {
-        float4 a[kBatch][8];  // every value is requested before the first is used
+        float4 a[kBatch][kMaxClusterSegments];  // every value is requested before the first is used
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
           const int idx = idx0 + u * kStride;
@@ -360,7 +361,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
             const int row = idx / cpr, ch = idx - row * cpr;
             const uint32_t local = base + row * kPartRow + g_lo * 32 + ch * 16;
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
+            for (int q = 0; q < kMaxClusterSegments; ++q)
               if (q < n) a[u][q] = ld_cluster_f4(map_to_cta(local, static_cast<uint32_t>(q)));
           }
         }
@@ -371,7 +372,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
             const int row = idx / cpr, ch = idx - row * cpr;
             float4 t = a[u][0];
 #pragma unroll
-            for (int q = 1; q < 8; ++q)  // t = s_0, then t + s_1, ... : the contract's order
+            for (int q = 1; q < kMaxClusterSegments; ++q)  // t = s_0, then t + s_1, ... : the contract's order
               if (q < n) {
                 t.x = __fadd_rn(t.x, a[u][q].x); t.y = __fadd_rn(t.y, a[u][q].y);
                 t.z = __fadd_rn(t.z, a[u][q].z); t.w = __fadd_rn(t.w, a[u][q].w);
@@ -735,7 +736,10 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
         cudaFuncSetAttribute(linear_kernel<BN, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(linear_kernel<BN, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             Cfg::kSmemBytes) != cudaSuccess)
+                             Cfg::kSmemBytes) != cudaSuccess ||
+        // clusters of nine to sixteen CTAs (a tile with as many segments) are beyond the portable size
+        cudaFuncSetAttribute(linear_kernel<BN, true, true>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) !=
+            cudaSuccess)
       return VOSTI_ERR_CUDA;
     attr_set[dev] = true;
   }
@@ -751,14 +755,19 @@ vosti_status launch_linear(EncodeTiledFn fn, const void* x, const void* w, void*
   const bool few = tiles * 2 <= sm_count;
   const bool ws_ok = workspace != nullptr && workspace_bytes >= split_workspace_bytes(M, N, K) &&
                      reinterpret_cast<uintptr_t>(workspace) % 16 == 0;
-  const bool cluster_ok = seg.n_seg > 1 && seg.n_seg <= 8;
+  const bool cluster_ok = seg.n_seg > 1 && seg.n_seg <= kMaxClusterSegments;
   const bool pairs_ok = BN == 256 && sm_count >= 2;
   int sched = schedule;
   if (sched == VOSTI_LINEAR_AUTO) {
     // (clusters only when all of them fit the SMs at once: a second round of one-unit CTAs costs
     // more than the persistent workspace route's second round)
-    if (few && cluster_ok && tiles * seg.n_seg <= (sm_count / seg.n_seg) * seg.n_seg) sched = VOSTI_LINEAR_SPLIT_CLUSTER;
+    // (and of the portable size: nine CTAs to a cluster were placed eight clusters at a time and took
+    // 45 us where the workspace route takes 26-36, 4096 x 14336 at 1-128 rows)
+    if (few && cluster_ok && seg.n_seg <= 8 && tiles * seg.n_seg <= (sm_count / seg.n_seg) * seg.n_seg)
+      sched = VOSTI_LINEAR_SPLIT_CLUSTER;
     else if (seg.n_seg > 1 && ws_ok && split_pays(M, N, tiles, seg, sm_count)) sched = VOSTI_LINEAR_SPLIT_WORKSPACE;
+    // (without a workspace the large clusters still halve the time of whole tiles at those sizes)
+    else if (few && cluster_ok && tiles * seg.n_seg <= sm_count) sched = VOSTI_LINEAR_SPLIT_CLUSTER;
     else if (pairs_ok && use_pairs) sched = VOSTI_LINEAR_PAIRS;
     else sched = VOSTI_LINEAR_WHOLE_TILES;
   } else if ((sched == VOSTI_LINEAR_SPLIT_CLUSTER && !cluster_ok) ||

@@ -84,8 +84,8 @@ def test_row_level_contract(N, K):
 def test_every_schedule_gives_the_same_bits(N, K, n_seg):
     """The K segments of a tile computed by one CTA in turn (whole tiles), by one CTA each with the
     sums added from a workspace by a second kernel, or by the CTAs of a cluster that add the sums out
-    of each other's shared memory (2 to 8 segments: a power of two, 6 and 3, whose column shares are
-    uneven): same bits, for a single row, ragged and several row tiles.  A schedule that does not apply
+    of each other's shared memory (a power of two; 6, 3 and 9 segments, whose column shares are uneven;
+    9 is a cluster beyond the portable size): same bits, for a single row, ragged and several row tiles.  A schedule that does not apply
     is refused."""
     from paper_2609_38981_b200 import binding as vb
     from paper_2609_38981_b200 import linear as vl
@@ -101,7 +101,7 @@ def test_every_schedule_gives_the_same_bits(N, K, n_seg):
         if n_seg > 1:
             y = vl.vosti_linear(xm, wd, workspace=workspace(M, N, K), schedule=vl.VOSTI_LINEAR_SPLIT_WORKSPACE)
             assert torch.equal(bf16_bits(y), whole), (M, "workspace")
-        if 2 <= n_seg <= 8:
+        if 2 <= n_seg <= 16:
             y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
             vl.vosti_linear(xm, wd, y, schedule=vl.VOSTI_LINEAR_SPLIT_CLUSTER)
             assert torch.equal(bf16_bits(y), whole), (M, "cluster")
