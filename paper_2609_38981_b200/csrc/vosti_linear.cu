@@ -272,8 +272,9 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
           // s_j of this unit -> this CTA's shared memory, [row][BN] fp32 with rows kPartRow bytes apart
           // (the pipeline stages are idle: the unit's MMAs are done, and the CTA has no other unit)
           const uint32_t dst = base + r * kPartRow + c0 * 4;
+          const bool warp_live = tc.m0 + (warp & 3) * 32 < M;  // else: rows beyond M, never read
 #pragma unroll 1
-          for (int cb = 0; cb < 128; cb += 32) {
+          for (int cb = 0; cb < 128 && warp_live; cb += 32) {
             uint32_t v[32];
             tmem_ld32(tmem + lane_sel + buf * BN + c0 + cb, v);
             tmem_wait_ld();
@@ -352,12 +353,13 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
       // Consecutive threads take consecutive chunks of a row: a warp's request to a peer's shared
       // memory is one contiguous piece (scattered 16-byte requests crawl), and so is its store.
       constexpr int kStride = 32 * Cfg::kEpiWarps, kBatch = 1;  // (more chunks in flight per thread measured slower)
-      for (int idx0 = tid - 64; idx0 < Cfg::kBM * cpr; idx0 += kBatch * kStride) {
+      const int live = min(Cfg::kBM, M - tc.m0) * cpr;  // rows beyond M hold zeros nobody wants
+      for (int idx0 = tid - 64; idx0 < live; idx0 += kBatch * kStride) {
         float4 a[kBatch][kMaxClusterSegments];  // every value is requested before the first is used
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
           const int idx = idx0 + u * kStride;
-          if (idx < Cfg::kBM * cpr) {
+          if (idx < live) {
             const int row = idx / cpr, ch = idx - row * cpr;
             const uint32_t local = base + row * kPartRow + g_lo * 32 + ch * 16;
 #pragma unroll
@@ -368,7 +370,7 @@ linear_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
           const int idx = idx0 + u * kStride;
-          if (idx < Cfg::kBM * cpr) {
+          if (idx < live) {
             const int row = idx / cpr, ch = idx - row * cpr;
             float4 t = a[u][0];
 #pragma unroll
